@@ -1,0 +1,20 @@
+"""B200-native (sm_100a) implementation of the LAGA per-rank attention hot path.
+
+One sequence-parallel rank's compute after the latent all-gather (Algorithm 1 steps 4-5 of the
+paper, and the backward of Section 5.2): head-shard up-projection of the gathered MLA latent,
+key assembly with the shared rope band, explicit causal softmax attention, forward and backward.
+
+The work is done by hand-written CUDA kernels behind a C ABI (``include/laga.h``); ``laga`` is the
+ctypes binding (argument marshalling only).  The shared library is loaded on first use and its
+absence is an error: there is no CPU or eager fallback.
+"""
+from .inputs import CONFIGS, CONFIG_SEEDS, LagaShape, make_inputs  # noqa: F401
+
+__all__ = ["CONFIGS", "CONFIG_SEEDS", "LagaShape", "make_inputs", "laga"]
+
+
+def __getattr__(name):
+    if name == "laga":
+        import importlib
+        return importlib.import_module(".laga", __name__)
+    raise AttributeError(name)
