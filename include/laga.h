@@ -1,0 +1,121 @@
+/*
+ * laga.h -- C ABI of the B200 (sm_100a) LAGA per-rank attention hot path.
+ *
+ * What the library computes.  One sequence-parallel rank's work after the latent all-gather of
+ * LAGA (paper Algorithm 1, steps 4 and 5) and its backward (paper Section 5.2):
+ *
+ *   step 4   KV = c_kv . W_kv_b[H_r]                (head-shard up-projection of the gathered latent)
+ *            K_nope[t,i,:] = KV[t, i*(d_nope+d_v) + 0 .. d_nope)
+ *            V[t,i,:]      = KV[t, i*(d_nope+d_v) + d_nope .. d_nope+d_v)
+ *   step 5   K[t,i,:] = K_nope[t,i,:] || k_pe[t,:]   (the rope key band is shared by all heads, Sec. 2.1)
+ *            scores = softmax_scale * q K^T, masked to t <= s when causal
+ *            O = softmax(scores) V,   LSE = natural-log-sum-exp of the masked scaled scores
+ *   backward dQ, dc_kv (partial sum over this head shard), dk_pe (sum over this head shard) and
+ *            dW_kv_b[H_r] (complete for these heads: the "(full_seq, H_r)" gradient shard of Sec. 5.2)
+ *
+ * Conventions common to every call
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library allocates nothing,
+ *     frees nothing and keeps no pointer after the call returns.  Buffers must stay valid until the
+ *     work enqueued on `stream` has finished.  All base pointers must be 16-byte aligned.
+ *   - All tensors are dense row-major ("C order") with the shapes given below; bf16 tensors are
+ *     passed as `const void*` / `void*` pointing at 16-bit brain-float elements.
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL is the default
+ *     stream) and return without synchronising, except laga_query_status.
+ *   - Return value: LAGA_OK (0) or a negative LAGA_ERR_* code.  Argument errors are detected before
+ *     anything is enqueued.  Nothing throws, aborts or traps.
+ *   - This build is tuned for the DeepSeek-V3 head geometry: d_c = 512, d_nope = 128, d_rope = 64,
+ *     d_v = 128.  Other values return LAGA_ERR_UNSUPPORTED.  S >= 1 and h >= 1 are arbitrary (S need
+ *     not be a multiple of any tile).  Batch is a caller loop.
+ *   - `workspace` is caller-provided scratch of at least laga_*_workspace_bytes(...) bytes, 1024-byte
+ *     aligned.  Its first word is the launch status word read by laga_query_status.  Two calls that
+ *     may overlap on the GPU must not share a workspace.
+ */
+#ifndef LAGA_H_
+#define LAGA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LAGA_OK 0
+#define LAGA_ERR_INVALID_ARG (-1)         /* NULL or misaligned pointer, S < 1, h < 1, bad flag     */
+#define LAGA_ERR_UNSUPPORTED (-2)         /* head geometry other than 512/128/64/128, or not sm_100 */
+#define LAGA_ERR_WORKSPACE_TOO_SMALL (-3)
+#define LAGA_ERR_CUDA (-4)                /* a CUDA runtime/driver call or a launch failed          */
+#define LAGA_ERR_DEVICE_TIMEOUT (-5)      /* only from laga_query_status: a bounded device wait ran out */
+
+#define LAGA_FLAG_ACCUM_DW 1u             /* laga_bwd: add into dw_kv_b instead of overwriting it   */
+
+/* Library version (major*10000 + minor*100 + patch). */
+int laga_version(void);
+
+/* Static, human-readable name of a status code. */
+const char* laga_status_string(int status);
+
+/* Scratch sizes in bytes for the calls below (0 if the geometry is unsupported). */
+size_t laga_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v);
+size_t laga_bwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v, unsigned flags);
+
+/*
+ * Forward: Algorithm 1 steps 4-5.
+ *   q       bf16 [S, h, d_nope+d_rope]   queries of this head shard, nope band first, rope band last
+ *                                        (already rotated)
+ *   c_kv    bf16 [S, d_c]                gathered, already-normalised latent
+ *   k_pe    bf16 [S, d_rope]             gathered, already-rotated shared rope key
+ *   w_kv_b  bf16 [d_c, h*(d_nope+d_v)]   head shard of W_kv_b; column i*(d_nope+d_v)+j is K_nope
+ *                                        channel j of head i for j < d_nope, else V channel j-d_nope
+ *   out     bf16 [S, h, d_v]             written
+ *   lse     fp32 [S, h]                  written
+ * `causal` != 0 masks keys t > s.  The per-head K_nope/V are materialised in bf16 inside `workspace`
+ * (the explicit form's own footprint); nothing else of size S x S or S x h x d_c exists.
+ */
+int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
+             int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out, float* lse,
+             void* workspace, size_t workspace_bytes, unsigned flags, void* stream);
+
+/*
+ * Backward: Section 5.2 (chain rule through step 5, then back through step 4).
+ *   q, c_kv, k_pe, w_kv_b   as in laga_fwd
+ *   out, lse                what laga_fwd produced for the same inputs
+ *   dout    bf16 [S, h, d_v]             upstream gradient of out
+ *   dq      bf16 [S, h, d_nope+d_rope]   written
+ *   dc_kv   bf16 [S, d_c]                written: this head shard's contribution (ranks reduce-scatter it)
+ *   dk_pe   bf16 [S, d_rope]             written: summed over this shard's heads
+ *   dw_kv_b fp32 [d_c, h*(d_nope+d_v)]   overwritten, or accumulated into with LAGA_FLAG_ACCUM_DW
+ * K_nope/V are recomputed from c_kv (the forward keeps only out and lse).  All accumulation is fp32.
+ * dw_kv_b is reduced over the sequence with floating-point atomics: its low-order bits may differ
+ * from run to run.
+ */
+int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
+             const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
+             float softmax_scale, int causal, void* dq, void* dc_kv, void* dk_pe, float* dw_kv_b,
+             void* workspace, size_t workspace_bytes, unsigned flags, void* stream);
+
+/*
+ * Step entry points (the same kernels laga_fwd / laga_bwd launch, callable on their own).
+ *
+ * laga_up_project: Algorithm 1 step 4.   kv bf16 [S, h*(d_nope+d_v)] = c_kv . w_kv_b  (fp32 accumulate).
+ * laga_kv_backward: Section 5.2, back through step 4.  Given dkv bf16 [S, h*(d_nope+d_v)] (per head:
+ *   dK_nope then dV), writes dc_kv bf16 [S, d_c] = dkv . w_kv_b^T and dw_kv_b fp32 = c_kv^T . dkv.
+ * `status_word` is a device pointer to one 32-bit word (zeroed by the call) that receives the
+ * device status; pass it to laga_query_status.
+ */
+int laga_up_project(const void* c_kv, const void* w_kv_b, int S, int h, int d_c, int d_nope, int d_v,
+                    void* kv, void* status_word, void* stream);
+int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int S, int h, int d_c,
+                     int d_nope, int d_v, void* dc_kv, float* dw_kv_b, unsigned flags, void* status_word,
+                     void* stream);
+
+/*
+ * Synchronises `stream`, reads the status word at the start of `workspace` (or a `status_word`
+ * given to a step entry point) and returns LAGA_OK, LAGA_ERR_DEVICE_TIMEOUT or LAGA_ERR_CUDA.
+ * If `detail` is not NULL it receives the raw device word (which wait gave up).
+ */
+int laga_query_status(const void* workspace, void* stream, unsigned* detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAGA_H_ */

@@ -1,0 +1,261 @@
+// Forward attention of Algorithm 1 step 5 for the DeepSeek-V3 head geometry (d_qk = 128 nope + 64
+// rope, d_v = 128): O = softmax(scale * q (K_nope || k_pe)^T) V, with LSE, never materialising the
+// S x S scores.  K_nope and V are read from the bf16 up-projection KV[S, h*256]; the shared rope
+// band k_pe[S, 64] is a separate TMA box, so the 192-wide key is never assembled in memory.
+//
+// One CTA owns 128 query rows of one head and walks the key tiles (128 keys each).
+//   warp 0      TMA producer: Q once, then K (2 stages) and V (1 stage) tiles
+//   warp 1      MMA issuer:   S = Q K^T (12 tcgen05.mma of K=16) into a double-buffered TMEM tile,
+//                             O += P V  (8 tcgen05.mma) into a TMEM accumulator
+//   warps 2..5  softmax: one thread per query row; online max / sum in registers, P written to
+//               shared memory as the bf16 A operand of the second contraction, lazy rescale of O
+#pragma once
+#include "sm100_ptx.cuh"
+
+namespace laga {
+
+struct AttnFwdArgs {
+    int S, h;
+    float scale_log2;       // softmax_scale * log2(e)
+    __nv_bfloat16* out;     // [S, h, 128]
+    float* lse;             // [S, h]
+    unsigned int* status;
+};
+
+struct AttnFwdSmem {
+    static constexpr int kSlab = 128 * 128;             // 128 rows x 128 bytes
+    static constexpr int kQ = 0;                        // 3 slabs
+    static constexpr int kK = kQ + 3 * kSlab;           // 2 stages x 3 slabs (nope lo, nope hi, rope)
+    static constexpr int kV = kK + 2 * 3 * kSlab;       // 1 stage x 2 slabs
+    static constexpr int kP = kV + 2 * kSlab;           // 2 slabs
+    static constexpr int kBar = kP + 2 * kSlab;
+    static constexpr int kTotalBytes = kBar + 256 + 1024;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <bool kCausal>
+__global__ void __launch_bounds__(192, 1)
+attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
+                      const __grid_constant__ CUtensorMap tmap_kpe, const AttnFwdArgs args) {
+    using L = AttnFwdSmem;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
+    uint64_t* q_full = bars + 0;
+    uint64_t* k_full = bars + 1;     // [2]
+    uint64_t* k_empty = bars + 3;    // [2]
+    uint64_t* v_full = bars + 5;
+    uint64_t* v_empty = bars + 6;
+    uint64_t* s_full = bars + 7;     // [2]
+    uint64_t* s_free = bars + 9;     // [2]
+    uint64_t* p_full = bars + 11;
+    uint64_t* pv_done = bars + 12;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+    AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_q_tiles = (args.S + 127) / 128;
+    const int q_tile = n_q_tiles - 1 - static_cast<int>(blockIdx.x);   // longest rows first
+    const int head = blockIdx.y;
+    const int q0 = q_tile * 128;
+    const int n_kv = kCausal ? q_tile + 1 : n_q_tiles;
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+            mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 128);
+        }
+        mbar_init(v_full, 1); mbar_init(v_empty, 1);
+        mbar_init(p_full, 128); mbar_init(pv_done, 1);
+        abort_flag->value = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
+    }
+    if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base + 256;
+
+    if (warp == 0) {
+        if (elect_one()) {
+            mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
+            for (int c = 0; c < 3; ++c)
+                tma_load_2d(smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
+            auto load_k = [&](int j) -> bool {
+                const int s = j & 1;
+                if (!mbar_wait(&k_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, args.status, 0x10)) return false;
+                uint8_t* dst = smem + L::kK + s * 3 * L::kSlab;
+                mbar_arrive_expect_tx(&k_full[s], 3 * L::kSlab);
+                tma_load_2d(dst, &tmap_kv, &k_full[s], head * 256, j * 128);
+                tma_load_2d(dst + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * 128);
+                tma_load_2d(dst + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * 128);
+                return true;
+            };
+            bool ok = load_k(0);
+            for (int j = 0; j < n_kv && ok; ++j) {
+                if (j + 1 < n_kv) ok = load_k(j + 1);
+                if (!ok) break;
+                ok = mbar_wait(v_empty, (j & 1) ^ 1, abort_flag, args.status, 0x11);
+                if (!ok) break;
+                mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
+                tma_load_2d(smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
+                tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
+            }
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);
+            const uint32_t sq = smem_u32(smem + L::kQ);
+            const uint32_t sv = smem_u32(smem + L::kV);
+            const uint32_t sp = smem_u32(smem + L::kP);
+            auto issue_pv = [&](int j) -> bool {
+                if (!mbar_wait(v_full, j & 1, abort_flag, args.status, 0x20)) return false;
+                if (!mbar_wait(p_full, j & 1, abort_flag, args.status, 0x21)) return false;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint64_t da = desc_k_major(sp + (kk >> 2) * L::kSlab + (kk & 3) * 32);
+                    const uint64_t db = desc_mn_major(sv + kk * 2048, L::kSlab);
+                    mma_ss(tmem_o, da, db, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(v_empty);
+                mma_commit(pv_done);
+                return true;
+            };
+            bool ok = mbar_wait(q_full, 0, abort_flag, args.status, 0x22);
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int s = j & 1;
+                const uint32_t ph = (j >> 1) & 1;
+                ok = mbar_wait(&k_full[s], ph, abort_flag, args.status, 0x23) &&
+                     mbar_wait(&s_free[s], ph ^ 1, abort_flag, args.status, 0x24);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t sk = smem_u32(smem + L::kK + s * 3 * L::kSlab);
+#pragma unroll
+                for (int kk = 0; kk < 12; ++kk) {
+                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
+                    mma_ss(tmem_base + s * 128, desc_k_major(sq + off), desc_k_major(sk + off), idesc_qk,
+                           kk > 0 ? 1u : 0u);
+                }
+                mma_commit(&k_empty[s]);
+                mma_commit(&s_full[s]);
+                if (j > 0) ok = issue_pv(j - 1);
+            }
+            if (ok) issue_pv(n_kv - 1);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;          // row inside the tile == TMEM lane
+        const int sq_idx = q0 + row;                  // global query index
+        const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+        uint8_t* p_smem = smem + L::kP;
+        float m_run = -INFINITY, l_run = 0.f;         // running max (scaled, log2 domain) and sum
+        bool ok = true;
+        for (int j = 0; j < n_kv; ++j) {
+            const int s = j & 1;
+            ok = mbar_wait_warp(&s_full[s], (j >> 1) & 1, abort_flag, args.status, 0x30);
+            if (!ok) break;
+            tc_fence_after_sync();
+            uint32_t sv[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld_x32(tmem_base + lane_addr + s * 128 + c * 32, sv + c * 32);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            mbar_arrive(&s_free[s]);
+
+            const bool edge = (j == n_kv - 1);
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 128; ++c) {
+                float x = __uint_as_float(sv[c]);
+                if (edge) {
+                    const int t = j * 128 + c;
+                    if ((kCausal && t > sq_idx) || t >= args.S) x = -INFINITY;
+                }
+                sv[c] = __float_as_uint(x);
+                mx = fmaxf(mx, x);
+            }
+            const float m_new = fmaxf(m_run, mx * args.scale_log2);
+            // Lazy rescale: keep the old reference max unless it fell behind by more than 2^8.
+            const bool move = (m_new - m_run) > 8.0f;
+            const float alpha = move ? fast_exp2(m_run - m_new) : 1.0f;
+            if (move) m_run = m_new;
+            float sum = 0.f;
+            uint32_t pk[64];
+#pragma unroll
+            for (int c = 0; c < 64; ++c) {
+                const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * c]), args.scale_log2, -m_run));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * c + 1]), args.scale_log2, -m_run));
+                sum += p0 + p1;
+                pk[c] = pack_bf16x2(p0, p1);
+            }
+            l_run = l_run * alpha + sum;
+
+            if (j > 0) {
+                ok = mbar_wait_warp(pv_done, (j - 1) & 1, abort_flag, args.status, 0x31);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (__any_sync(0xffffffffu, move)) {
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int v = 0; v < 32; ++v) o[v] = __float_as_uint(__uint_as_float(o[v]) * alpha);
+                        tmem_st_x32(tmem_o + lane_addr + c * 32, o);
+                    }
+                    tmem_st_wait();
+                }
+            }
+#pragma unroll
+            for (int c16 = 0; c16 < 16; ++c16) {
+                uint4 val = make_uint4(pk[c16 * 4], pk[c16 * 4 + 1], pk[c16 * 4 + 2], pk[c16 * 4 + 3]);
+                *reinterpret_cast<uint4*>(p_smem + (c16 >> 3) * L::kSlab + swz128_offset(row, c16 & 7)) = val;
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(p_full);
+        }
+        if (ok) ok = mbar_wait_warp(pv_done, (n_kv - 1) & 1, abort_flag, args.status, 0x32);
+        if (ok) {
+            tc_fence_after_sync();
+            const float inv_l = 1.0f / l_run;
+            const bool valid = sq_idx < args.S;
+            __nv_bfloat16* dst = args.out + (static_cast<size_t>(sq_idx) * args.h + head) * 128;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
+                tmem_ld_wait();
+                if (valid) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(o[v * 8 + 0]) * inv_l, __uint_as_float(o[v * 8 + 1]) * inv_l);
+                        w.y = pack_bf16x2(__uint_as_float(o[v * 8 + 2]) * inv_l, __uint_as_float(o[v * 8 + 3]) * inv_l);
+                        w.z = pack_bf16x2(__uint_as_float(o[v * 8 + 4]) * inv_l, __uint_as_float(o[v * 8 + 5]) * inv_l);
+                        w.w = pack_bf16x2(__uint_as_float(o[v * 8 + 6]) * inv_l, __uint_as_float(o[v * 8 + 7]) * inv_l);
+                        reinterpret_cast<uint4*>(dst + c * 32)[v] = w;
+                    }
+                }
+            }
+            if (valid)
+                args.lse[static_cast<size_t>(sq_idx) * args.h + head] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+}
+
+}  // namespace laga

@@ -1,0 +1,273 @@
+// C ABI of the LAGA hot path (see include/laga.h): argument validation, TMA tensor-map
+// construction, workspace carving and kernel launches on the caller's stream.
+#include "../../include/laga.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "attn_fwd_sm100.cuh"
+#include "gemm_sm100.cuh"
+
+namespace {
+
+using namespace laga;
+
+constexpr int kDc = 512, kDn = 128, kDr = 64, kDv = 128;
+constexpr size_t kStatusBytes = 1024;   // the status word's slot; keeps what follows 1024-aligned
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool geometry_supported(int d_c, int d_nope, int d_rope, int d_v) {
+    return d_c == kDc && d_nope == kDn && d_rope == kDr && d_v == kDv;
+}
+
+// cuTensorMapEncodeTiled is resolved through the runtime so the library has no link-time
+// dependency on the driver library (it must load on machines without a GPU).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor map, 128-byte swizzle, box of 64 contiguous elements x box_rows rows,
+// out-of-range elements read as zero.
+bool make_tmap_bf16(CUtensorMap* map, const void* base, uint64_t inner_elems, uint64_t rows,
+                    uint64_t row_stride_bytes, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner_elems, rows};
+    cuuint64_t strides[1] = {row_stride_bytes};
+    cuuint32_t box[2] = {64u, box_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int check_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LAGA_ERR_CUDA;
+    static int cached_dev = -1, cached_major = 0;
+    if (cached_dev != dev) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return LAGA_ERR_CUDA;
+        cached_dev = dev;
+        cached_major = major;
+    }
+    return cached_major == 10 ? LAGA_OK : LAGA_ERR_UNSUPPORTED;
+}
+
+template <typename Kernel>
+int set_smem(Kernel kernel, int bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
+               ? LAGA_OK
+               : LAGA_ERR_CUDA;
+}
+
+int launch_status() { return cudaGetLastError() == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA; }
+
+// ---- Algorithm 1 step 4: KV[S, N] = c_kv[S, d_c] . W[d_c, N] ------------------------------------
+int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
+                      cudaStream_t stream) {
+    constexpr int BN = 256, STAGES = 4;
+    auto kernel = gemm_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
+    using L = GemmSmem<BN, STAGES>;
+    CUtensorMap ta, tb;
+    if (!make_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
+    if (!make_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
+    if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
+    GemmArgs a{S, N, kDc, kDc / 64, kv, N, status};
+    dim3 grid(N / BN, (S + 127) / 128, 1);
+    kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a);
+    return launch_status();
+}
+
+// ---- Section 5.2, back through step 4 -----------------------------------------------------------
+// dc_kv[S, d_c] = dKV[S, N] . W^T          (A = dKV K-major, B = W rows d_c / inner N: K-major)
+int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, unsigned* status,
+                cudaStream_t stream) {
+    constexpr int BN = 256, STAGES = 4;
+    auto kernel = gemm_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
+    using L = GemmSmem<BN, STAGES>;
+    CUtensorMap ta, tb;
+    if (!make_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
+    if (!make_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN)) return LAGA_ERR_CUDA;
+    if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
+    GemmArgs a{S, kDc, N, (N + 63) / 64, dc_kv, kDc, status};
+    dim3 grid(kDc / BN, (S + 127) / 128, 1);
+    kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a);
+    return launch_status();
+}
+
+// dW[d_c, N] (+)= c_kv^T . dKV   (both operands read with the token index as K: MN-major), split over
+// the sequence with fp32 atomic accumulation.
+int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool accumulate, unsigned* status,
+              cudaStream_t stream) {
+    constexpr int BN = 256, STAGES = 4;
+    auto kernel = gemm_sm100_kernel<BN, STAGES, true, true, EPI_ATOMIC_F32>;
+    using L = GemmSmem<BN, STAGES>;
+    CUtensorMap ta, tb;
+    if (!make_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 64)) return LAGA_ERR_CUDA;
+    if (!make_tmap_bf16(&tb, dkv, N, S, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;
+    if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
+    if (!accumulate &&
+        cudaMemsetAsync(dw, 0, sizeof(float) * static_cast<size_t>(kDc) * N, stream) != cudaSuccess)
+        return LAGA_ERR_CUDA;
+    const int tiles = (kDc / 128) * (N / BN);
+    const int k_tiles = (S + 63) / 64;
+    int splits = (2 * 148 + tiles - 1) / tiles;
+    if (splits > k_tiles) splits = k_tiles;
+    if (splits < 1) splits = 1;
+    const int per_split = (k_tiles + splits - 1) / splits;
+    splits = (k_tiles + per_split - 1) / per_split;
+    GemmArgs a{kDc, N, S, per_split, dw, N, status};
+    dim3 grid(N / BN, kDc / 128, splits);
+    kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a);
+    return launch_status();
+}
+
+// ---- Algorithm 1 step 5 -------------------------------------------------------------------------
+int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int h, float softmax_scale,
+                    int causal, void* out, float* lse, unsigned* status, cudaStream_t stream) {
+    using L = AttnFwdSmem;
+    const int N = h * (kDn + kDv);
+    CUtensorMap tq, tkv, tpe;
+    if (!make_tmap_bf16(&tq, q, static_cast<uint64_t>(h) * 192, S, static_cast<uint64_t>(h) * 192 * 2, 128))
+        return LAGA_ERR_CUDA;
+    if (!make_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
+    if (!make_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, 128)) return LAGA_ERR_CUDA;
+    AttnFwdArgs a{S, h, softmax_scale * 1.4426950408889634f, reinterpret_cast<__nv_bfloat16*>(out), lse, status};
+    dim3 grid((S + 127) / 128, h, 1);
+    if (causal) {
+        auto kernel = attn_fwd_sm100_kernel<true>;
+        if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
+        kernel<<<grid, 192, L::kTotalBytes, stream>>>(tq, tkv, tpe, a);
+    } else {
+        auto kernel = attn_fwd_sm100_kernel<false>;
+        if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
+        kernel<<<grid, 192, L::kTotalBytes, stream>>>(tq, tkv, tpe, a);
+    }
+    return launch_status();
+}
+
+int zero_status(void* status_word, cudaStream_t stream) {
+    return cudaMemsetAsync(status_word, 0, sizeof(unsigned), stream) == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int laga_version(void) { return 100; }
+
+const char* laga_status_string(int status) {
+    switch (status) {
+        case LAGA_OK: return "LAGA_OK";
+        case LAGA_ERR_INVALID_ARG: return "LAGA_ERR_INVALID_ARG";
+        case LAGA_ERR_UNSUPPORTED: return "LAGA_ERR_UNSUPPORTED";
+        case LAGA_ERR_WORKSPACE_TOO_SMALL: return "LAGA_ERR_WORKSPACE_TOO_SMALL";
+        case LAGA_ERR_CUDA: return "LAGA_ERR_CUDA";
+        case LAGA_ERR_DEVICE_TIMEOUT: return "LAGA_ERR_DEVICE_TIMEOUT";
+        default: return "LAGA_ERR_UNKNOWN";
+    }
+}
+
+size_t laga_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v) {
+    if (S < 1 || h < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
+    return kStatusBytes + align_up(static_cast<size_t>(S) * h * (d_nope + d_v) * 2, 1024);
+}
+
+size_t laga_bwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v, unsigned flags) {
+    (void)flags;
+    if (S < 1 || h < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
+    return 0;   // backward kernels not built yet
+}
+
+int laga_up_project(const void* c_kv, const void* w_kv_b, int S, int h, int d_c, int d_nope, int d_v, void* kv,
+                    void* status_word, void* stream) {
+    if (!c_kv || !w_kv_b || !kv || !status_word || S < 1 || h < 1) return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(c_kv) || !aligned16(w_kv_b) || !aligned16(kv)) return LAGA_ERR_INVALID_ARG;
+    if (!geometry_supported(d_c, d_nope, kDr, d_v)) return LAGA_ERR_UNSUPPORTED;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = zero_status(status_word, st)) != LAGA_OK) return rc;
+    return launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, static_cast<unsigned*>(status_word), st);
+}
+
+int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int S, int h, int d_c, int d_nope,
+                     int d_v, void* dc_kv, float* dw_kv_b, unsigned flags, void* status_word, void* stream) {
+    if (!dkv || !c_kv || !w_kv_b || !dc_kv || !dw_kv_b || !status_word || S < 1 || h < 1)
+        return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(dkv) || !aligned16(c_kv) || !aligned16(w_kv_b) || !aligned16(dc_kv) || !aligned16(dw_kv_b))
+        return LAGA_ERR_INVALID_ARG;
+    if (flags & ~LAGA_FLAG_ACCUM_DW) return LAGA_ERR_INVALID_ARG;
+    if (!geometry_supported(d_c, d_nope, kDr, d_v)) return LAGA_ERR_UNSUPPORTED;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned* status = static_cast<unsigned*>(status_word);
+    const int N = h * (kDn + kDv);
+    if ((rc = zero_status(status_word, st)) != LAGA_OK) return rc;
+    if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, status, st);
+}
+
+int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
+             int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out, float* lse,
+             void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+    if (!q || !c_kv || !k_pe || !w_kv_b || !out || !lse || !workspace || S < 1 || h < 1)
+        return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(c_kv) || !aligned16(k_pe) || !aligned16(w_kv_b) || !aligned16(out) ||
+        !aligned16(lse) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return LAGA_ERR_INVALID_ARG;
+    if (flags != 0 || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
+    if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
+    if (workspace_bytes < laga_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v))
+        return LAGA_ERR_WORKSPACE_TOO_SMALL;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned* status = static_cast<unsigned*>(workspace);
+    void* kv = static_cast<uint8_t*>(workspace) + kStatusBytes;
+    if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
+    if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
+    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st);
+}
+
+int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
+             const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
+             float softmax_scale, int causal, void* dq, void* dc_kv, void* dk_pe, float* dw_kv_b, void* workspace,
+             size_t workspace_bytes, unsigned flags, void* stream) {
+    (void)q; (void)c_kv; (void)k_pe; (void)w_kv_b; (void)out; (void)lse; (void)dout; (void)S; (void)h;
+    (void)d_c; (void)d_nope; (void)d_rope; (void)d_v; (void)softmax_scale; (void)causal; (void)dq; (void)dc_kv;
+    (void)dk_pe; (void)dw_kv_b; (void)workspace; (void)workspace_bytes; (void)flags; (void)stream;
+    return LAGA_ERR_UNSUPPORTED;   // backward kernels not built yet
+}
+
+int laga_query_status(const void* workspace, void* stream, unsigned* detail) {
+    if (!workspace) return LAGA_ERR_INVALID_ARG;
+    unsigned word = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return LAGA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return LAGA_ERR_CUDA;
+    if (detail) *detail = word;
+    if (word == 0) return LAGA_OK;
+    return (word & 0xff000000u) == kStatusTimeout ? LAGA_ERR_DEVICE_TIMEOUT : LAGA_ERR_CUDA;
+}
+
+}  // extern "C"

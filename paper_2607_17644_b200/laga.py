@@ -1,0 +1,215 @@
+"""ctypes binding of the LAGA C ABI (``include/laga.h``): argument marshalling only.
+
+PyTorch appears here for device memory and the current CUDA stream; every step of the path runs in
+the library's CUDA kernels.  The shared library must exist (``python -m paper_2607_17644_b200.build``):
+there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED = -2
+ERR_WORKSPACE_TOO_SMALL = -3
+ERR_CUDA = -4
+ERR_DEVICE_TIMEOUT = -5
+FLAG_ACCUM_DW = 1
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblaga.so")
+_lib = None
+
+# name -> (restype, argtypes); mirrors include/laga.h one to one
+_vp, _ci, _cf, _cu, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_uint, ctypes.c_size_t
+SIGNATURES = {
+    "laga_version": (_ci, []),
+    "laga_status_string": (ctypes.c_char_p, [_ci]),
+    "laga_fwd_workspace_bytes": (_sz, [_ci] * 6),
+    "laga_bwd_workspace_bytes": (_sz, [_ci] * 6 + [_cu]),
+    "laga_fwd": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
+    "laga_bwd": (_ci, [_vp] * 7 + [_ci] * 6 + [_cf, _ci] + [_vp] * 4 + [_vp, _sz, _cu, _vp]),
+    "laga_up_project": (_ci, [_vp, _vp] + [_ci] * 5 + [_vp, _vp, _vp]),
+    "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
+    "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
+}
+
+
+class LagaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+def lib():
+    """Load liblaga.so once.  Raises if it has not been built: the product has no other path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_17644_b200.build`")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (restype, argtypes) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = restype, argtypes
+        _lib = handle
+    return _lib
+
+
+def version() -> int:
+    return int(lib().laga_version())
+
+
+def status_string(code: int) -> str:
+    return lib().laga_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise LagaError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, shape, name):
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous() and tuple(t.shape) == tuple(shape)):
+        raise ValueError(f"{name}: expected contiguous CUDA {dtype} tensor of shape {tuple(shape)}, "
+                         f"got {t.dtype} {tuple(t.shape)} on {t.device}")
+    return t
+
+
+def _geometry(q, c_kv, k_pe, w_kv_b, d_v):
+    S, h, d_qk = q.shape
+    d_c, d_rope = c_kv.shape[1], k_pe.shape[1]
+    d_nope = d_qk - d_rope
+    _dev(c_kv, torch.bfloat16, (S, d_c), "c_kv")
+    _dev(k_pe, torch.bfloat16, (S, d_rope), "k_pe")
+    _dev(w_kv_b, torch.bfloat16, (d_c, h * (d_nope + d_v)), "w_kv_b")
+    _dev(q, torch.bfloat16, (S, h, d_qk), "q")
+    return S, h, d_c, d_nope, d_rope
+
+
+def fwd_workspace_bytes(S, h, d_c=512, d_nope=128, d_rope=64, d_v=128) -> int:
+    return int(lib().laga_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v))
+
+
+def bwd_workspace_bytes(S, h, d_c=512, d_nope=128, d_rope=64, d_v=128, flags=0) -> int:
+    return int(lib().laga_bwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v, flags))
+
+
+def alloc_workspace(n_bytes: int, device="cuda") -> torch.Tensor:
+    """A 1024-byte aligned byte buffer (torch's caching allocator aligns to at least 512; over-allocate)."""
+    buf = torch.empty(n_bytes + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + n_bytes]
+
+
+def fwd(q, c_kv, k_pe, w_kv_b, d_v=128, softmax_scale=None, causal=True, out=None, lse=None, workspace=None,
+        stream=None):
+    """laga_fwd: returns (out bf16 [S,h,d_v], lse fp32 [S,h], workspace).  Enqueues only."""
+    S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
+    if softmax_scale is None:
+        softmax_scale = (d_nope + d_rope) ** -0.5
+    if out is None:
+        out = torch.empty(S, h, d_v, dtype=torch.bfloat16, device=q.device)
+    if lse is None:
+        lse = torch.empty(S, h, dtype=torch.float32, device=q.device)
+    _dev(out, torch.bfloat16, (S, h, d_v), "out")
+    _dev(lse, torch.float32, (S, h), "lse")
+    need = fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v)
+    if need == 0:
+        raise LagaError(ERR_UNSUPPORTED, "laga_fwd_workspace_bytes")
+    if workspace is None:
+        workspace = alloc_workspace(need, q.device)
+    rc = lib().laga_fwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope, d_v,
+                        float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse), _ptr(workspace),
+                        workspace.numel(), 0, _stream(stream))
+    _check(rc, "laga_fwd")
+    return out, lse, workspace
+
+
+def bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout, d_v=128, softmax_scale=None, causal=True, dq=None, dc_kv=None,
+        dk_pe=None, dw_kv_b=None, workspace=None, flags=0, stream=None):
+    """laga_bwd: returns (dq, dc_kv, dk_pe, dw_kv_b, workspace).  Enqueues only."""
+    S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
+    if softmax_scale is None:
+        softmax_scale = (d_nope + d_rope) ** -0.5
+    _dev(out, torch.bfloat16, (S, h, d_v), "out")
+    _dev(lse, torch.float32, (S, h), "lse")
+    _dev(dout, torch.bfloat16, (S, h, d_v), "dout")
+    dev = q.device
+    dq = torch.empty_like(q) if dq is None else _dev(dq, torch.bfloat16, q.shape, "dq")
+    dc_kv = torch.empty_like(c_kv) if dc_kv is None else _dev(dc_kv, torch.bfloat16, c_kv.shape, "dc_kv")
+    dk_pe = torch.empty_like(k_pe) if dk_pe is None else _dev(dk_pe, torch.bfloat16, k_pe.shape, "dk_pe")
+    if dw_kv_b is None:
+        if flags & FLAG_ACCUM_DW:
+            raise ValueError("LAGA_FLAG_ACCUM_DW needs an existing dw_kv_b to add into")
+        dw_kv_b = torch.empty(w_kv_b.shape, dtype=torch.float32, device=dev)
+    _dev(dw_kv_b, torch.float32, w_kv_b.shape, "dw_kv_b")
+    need = bwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v, flags)
+    if need == 0:
+        raise LagaError(ERR_UNSUPPORTED, "laga_bwd_workspace_bytes")
+    if workspace is None:
+        workspace = alloc_workspace(need, dev)
+    rc = lib().laga_bwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), _ptr(out), _ptr(lse), _ptr(dout), S, h,
+                        d_c, d_nope, d_rope, d_v, float(softmax_scale), int(bool(causal)), _ptr(dq), _ptr(dc_kv),
+                        _ptr(dk_pe), _ptr(dw_kv_b), _ptr(workspace), workspace.numel(), flags, _stream(stream))
+    _check(rc, "laga_bwd")
+    return dq, dc_kv, dk_pe, dw_kv_b, workspace
+
+
+def up_project(c_kv, w_kv_b, h, d_nope=128, d_v=128, kv=None, status_word=None, stream=None):
+    """laga_up_project: kv bf16 [S, h*(d_nope+d_v)] = c_kv . w_kv_b.  Returns (kv, status_word)."""
+    S, d_c = c_kv.shape
+    n = h * (d_nope + d_v)
+    _dev(c_kv, torch.bfloat16, (S, d_c), "c_kv")
+    _dev(w_kv_b, torch.bfloat16, (d_c, n), "w_kv_b")
+    kv = torch.empty(S, n, dtype=torch.bfloat16, device=c_kv.device) if kv is None else kv
+    _dev(kv, torch.bfloat16, (S, n), "kv")
+    if status_word is None:
+        status_word = torch.zeros(1, dtype=torch.int32, device=c_kv.device)
+    rc = lib().laga_up_project(_ptr(c_kv), _ptr(w_kv_b), S, h, d_c, d_nope, d_v, _ptr(kv), _ptr(status_word),
+                               _stream(stream))
+    _check(rc, "laga_up_project")
+    return kv, status_word
+
+
+def kv_backward(dkv, c_kv, w_kv_b, h, d_nope=128, d_v=128, dc_kv=None, dw_kv_b=None, flags=0, status_word=None,
+                stream=None):
+    """laga_kv_backward: dc_kv = dkv . w_kv_b^T (bf16), dw_kv_b (+)= c_kv^T . dkv (fp32)."""
+    S, d_c = c_kv.shape
+    n = h * (d_nope + d_v)
+    _dev(dkv, torch.bfloat16, (S, n), "dkv")
+    _dev(c_kv, torch.bfloat16, (S, d_c), "c_kv")
+    _dev(w_kv_b, torch.bfloat16, (d_c, n), "w_kv_b")
+    dc_kv = torch.empty_like(c_kv) if dc_kv is None else _dev(dc_kv, torch.bfloat16, c_kv.shape, "dc_kv")
+    if dw_kv_b is None:
+        dw_kv_b = torch.empty(d_c, n, dtype=torch.float32, device=c_kv.device)
+    _dev(dw_kv_b, torch.float32, (d_c, n), "dw_kv_b")
+    if status_word is None:
+        status_word = torch.zeros(1, dtype=torch.int32, device=c_kv.device)
+    rc = lib().laga_kv_backward(_ptr(dkv), _ptr(c_kv), _ptr(w_kv_b), S, h, d_c, d_nope, d_v, _ptr(dc_kv),
+                                _ptr(dw_kv_b), flags, _ptr(status_word), _stream(stream))
+    _check(rc, "laga_kv_backward")
+    return dc_kv, dw_kv_b, status_word
+
+
+def query_status(workspace_or_word, stream=None) -> tuple[int, int]:
+    """laga_query_status: synchronises the stream; returns (status code, raw device word)."""
+    detail = ctypes.c_uint(0)
+    rc = lib().laga_query_status(_ptr(workspace_or_word), _stream(stream), ctypes.byref(detail))
+    return int(rc), int(detail.value)
+
+
+def check_status(workspace_or_word, stream=None, where="laga"):
+    rc, detail = query_status(workspace_or_word, stream)
+    if rc != OK:
+        raise LagaError(rc, f"{where} (device word 0x{detail:08x})")
