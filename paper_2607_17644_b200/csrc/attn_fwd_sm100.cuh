@@ -235,6 +235,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
+                __syncwarp();
                 tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
                 tmem_ld_wait();
                 if (valid) {

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "attn_bwd_sm100.cuh"
 #include "attn_fwd_sm100.cuh"
 #include "gemm_sm100.cuh"
 
@@ -163,6 +164,80 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
     return launch_status();
 }
 
+// ---- Section 5.2: backward of step 5 ------------------------------------------------------------
+struct BwdWorkspace {
+    size_t kv, dkv, stat_l2, stat_delta, dk_rope, total;
+    int S_pad;
+};
+
+BwdWorkspace bwd_workspace_layout(int S, int h) {
+    BwdWorkspace w;
+    const size_t kv_bytes = align_up(static_cast<size_t>(S) * h * (kDn + kDv) * 2, 1024);
+    w.S_pad = (S + 127) / 128 * 128;
+    const size_t stat_bytes = align_up(static_cast<size_t>(h) * w.S_pad * sizeof(float), 1024);
+    w.kv = kStatusBytes;
+    w.dkv = w.kv + kv_bytes;
+    w.stat_l2 = w.dkv + kv_bytes;
+    w.stat_delta = w.stat_l2 + stat_bytes;
+    w.dk_rope = w.stat_delta + stat_bytes;
+    w.total = w.dk_rope + align_up(static_cast<size_t>(h) * S * kDr * sizeof(float), 1024);
+    return w;
+}
+
+int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void* out, const float* lse,
+                    const void* dout, int S, int h, float softmax_scale, int causal, void* dq, void* dkv,
+                    void* dk_pe, float* stat_l2, float* stat_delta, float* dk_rope, int S_pad, unsigned* status,
+                    cudaStream_t stream) {
+    const int N = h * (kDn + kDv);
+    const float scale_log2 = softmax_scale * 1.4426950408889634f;
+    {   // delta and the transposed, padded softmax statistics
+        const long long warps = static_cast<long long>(S_pad) * h;
+        const unsigned blocks = static_cast<unsigned>((warps * 32 + 255) / 256);
+        bwd_delta_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(out),
+                                                     reinterpret_cast<const __nv_bfloat16*>(dout), lse, S, h, S_pad,
+                                                     stat_l2, stat_delta);
+        if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+    }
+    const uint64_t q_row = static_cast<uint64_t>(h) * 192, do_row = static_cast<uint64_t>(h) * 128;
+    CUtensorMap tq64, tdo64, tkv128, tpe128, tq128, tdo128, tkv64, tpe64;
+    if (!make_tmap_bf16(&tq64, q, q_row, S, q_row * 2, 64) || !make_tmap_bf16(&tdo64, dout, do_row, S, do_row * 2, 64) ||
+        !make_tmap_bf16(&tkv128, kv, N, S, static_cast<uint64_t>(N) * 2, 128) ||
+        !make_tmap_bf16(&tpe128, k_pe, kDr, S, kDr * 2, 128) || !make_tmap_bf16(&tq128, q, q_row, S, q_row * 2, 128) ||
+        !make_tmap_bf16(&tdo128, dout, do_row, S, do_row * 2, 128) ||
+        !make_tmap_bf16(&tkv64, kv, N, S, static_cast<uint64_t>(N) * 2, 64) ||
+        !make_tmap_bf16(&tpe64, k_pe, kDr, S, kDr * 2, 64))
+        return LAGA_ERR_CUDA;
+    dim3 grid((S + 127) / 128, h, 1);
+    AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
+                     reinterpret_cast<__nv_bfloat16*>(dkv), dk_rope, status};
+    AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad, reinterpret_cast<__nv_bfloat16*>(dq),
+                    status};
+    if (causal) {
+        auto k1 = attn_bwd_dkv_sm100_kernel<true>;
+        auto k2 = attn_bwd_dq_sm100_kernel<true>;
+        if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
+            return LAGA_ERR_CUDA;
+        k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a);
+        if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+        k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b);
+    } else {
+        auto k1 = attn_bwd_dkv_sm100_kernel<false>;
+        auto k2 = attn_bwd_dq_sm100_kernel<false>;
+        if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
+            return LAGA_ERR_CUDA;
+        k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a);
+        if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+        k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b);
+    }
+    if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+    {
+        const size_t n = static_cast<size_t>(S) * kDr;
+        bwd_dkpe_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
+            dk_rope, S, h, reinterpret_cast<__nv_bfloat16*>(dk_pe));
+    }
+    return launch_status();
+}
+
 int zero_status(void* status_word, cudaStream_t stream) {
     return cudaMemsetAsync(status_word, 0, sizeof(unsigned), stream) == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA;
 }
@@ -193,7 +268,7 @@ size_t laga_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, i
 size_t laga_bwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v, unsigned flags) {
     (void)flags;
     if (S < 1 || h < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
-    return 0;   // backward kernels not built yet
+    return bwd_workspace_layout(S, h).total;
 }
 
 int laga_up_project(const void* c_kv, const void* w_kv_b, int S, int h, int d_c, int d_nope, int d_v, void* kv,
@@ -252,10 +327,34 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
              const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
              float softmax_scale, int causal, void* dq, void* dc_kv, void* dk_pe, float* dw_kv_b, void* workspace,
              size_t workspace_bytes, unsigned flags, void* stream) {
-    (void)q; (void)c_kv; (void)k_pe; (void)w_kv_b; (void)out; (void)lse; (void)dout; (void)S; (void)h;
-    (void)d_c; (void)d_nope; (void)d_rope; (void)d_v; (void)softmax_scale; (void)causal; (void)dq; (void)dc_kv;
-    (void)dk_pe; (void)dw_kv_b; (void)workspace; (void)workspace_bytes; (void)flags; (void)stream;
-    return LAGA_ERR_UNSUPPORTED;   // backward kernels not built yet
+    if (!q || !c_kv || !k_pe || !w_kv_b || !out || !lse || !dout || !dq || !dc_kv || !dk_pe || !dw_kv_b ||
+        !workspace || S < 1 || h < 1)
+        return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(c_kv) || !aligned16(k_pe) || !aligned16(w_kv_b) || !aligned16(out) ||
+        !aligned16(lse) || !aligned16(dout) || !aligned16(dq) || !aligned16(dc_kv) || !aligned16(dk_pe) ||
+        !aligned16(dw_kv_b) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return LAGA_ERR_INVALID_ARG;
+    if ((flags & ~LAGA_FLAG_ACCUM_DW) || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
+    if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
+    const BwdWorkspace w = bwd_workspace_layout(S, h);
+    if (workspace_bytes < w.total) return LAGA_ERR_WORKSPACE_TOO_SMALL;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    unsigned* status = reinterpret_cast<unsigned*>(base);
+    void* kv = base + w.kv;
+    void* dkv = base + w.dkv;
+    const int N = h * (kDn + kDv);
+    if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
+    // K_nope / V are recomputed from the latent: the forward keeps only out and lse.
+    if ((rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
+    if ((rc = launch_attn_bwd(q, kv, k_pe, out, lse, dout, S, h, softmax_scale, causal, dq, dkv, dk_pe,
+                              reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
+                              reinterpret_cast<float*>(base + w.dk_rope), w.S_pad, status, st)) != LAGA_OK)
+        return rc;
+    if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, status, st);
 }
 
 int laga_query_status(const void* workspace, void* stream, unsigned* detail) {
