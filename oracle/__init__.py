@@ -153,3 +153,59 @@ def bwd(q, c_kv, k_pe, w_kv_b, dout, d_v, softmax_scale, causal=True, kv_round_b
     if return_dkv:
         res["dk"], res["dv"] = torch.from_numpy(dk), torch.from_numpy(dv)
     return res
+
+
+def _int_list(values, upper):
+    arr = np.ascontiguousarray(np.asarray(values, dtype=np.int32))
+    assert arr.ndim == 1 and arr.size > 0 and (arr >= 0).all() and (arr < upper).all()
+    return arr, arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int))
+
+
+def bwd_rows(q, c_kv, k_pe, w_kv_b, dout, d_v, softmax_scale, rows, causal=True, kv_round_bf16=False):
+    """dQ for the listed query rows (a dQ row depends on its own query row only), with the forward
+    values it used.  Returns dict: dq [R,h,d_qk], out [R,h,d_v], lse [R,h]."""
+    lib = _load()
+    lib.laga_oracle_bwd_rows.argtypes = ([ctypes.POINTER(ctypes.c_uint16)] * 5 + [ctypes.c_int] * 6
+                                         + [ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                            ctypes.POINTER(ctypes.c_int), ctypes.c_int]
+                                         + [ctypes.POINTER(ctypes.c_double)] * 3)
+    lib.laga_oracle_bwd_rows.restype = ctypes.c_int
+    S, h, d_c, d_nope, d_rope = _dims(q, c_kv, k_pe, w_kv_b, d_v)
+    rows_arr, rows_p = _int_list(rows, S)
+    n = rows_arr.shape[0]
+    dq = np.empty((n, h, d_nope + d_rope), dtype=np.float64)
+    out = np.empty((n, h, d_v), dtype=np.float64)
+    lse = np.empty((n, h), dtype=np.float64)
+    qb, cb, kb, wb, db = _bits(q), _bits(c_kv), _bits(k_pe), _bits(w_kv_b), _bits(dout)
+    rc = lib.laga_oracle_bwd_rows(_u16(qb), _u16(cb), _u16(kb), _u16(wb), _u16(db), S, h, d_c, d_nope, d_rope,
+                                  d_v, float(softmax_scale), int(bool(causal)), int(bool(kv_round_bf16)),
+                                  rows_p, n, _f64(dq), _f64(out), _f64(lse))
+    if rc != 0:
+        raise RuntimeError(f"laga_oracle_bwd_rows failed with code {rc}")
+    return {"dq": torch.from_numpy(dq), "out": torch.from_numpy(out), "lse": torch.from_numpy(lse)}
+
+
+def bwd_keys(q, c_kv, k_pe, w_kv_b, dout, d_v, softmax_scale, keys, causal=True, kv_round_bf16=False):
+    """Key-side gradients for the listed key positions only.  Returns dict: dk [T,h,d_qk],
+    dv [T,h,d_v], dk_pe [T,d_rope], dc_kv [T,d_c] (the same numbers the full backward gives there)."""
+    lib = _load()
+    lib.laga_oracle_bwd_keys.argtypes = ([ctypes.POINTER(ctypes.c_uint16)] * 5 + [ctypes.c_int] * 6
+                                         + [ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                            ctypes.POINTER(ctypes.c_int), ctypes.c_int]
+                                         + [ctypes.POINTER(ctypes.c_double)] * 4)
+    lib.laga_oracle_bwd_keys.restype = ctypes.c_int
+    S, h, d_c, d_nope, d_rope = _dims(q, c_kv, k_pe, w_kv_b, d_v)
+    keys_arr, keys_p = _int_list(keys, S)
+    n = keys_arr.shape[0]
+    dk = np.empty((n, h, d_nope + d_rope), dtype=np.float64)
+    dv = np.empty((n, h, d_v), dtype=np.float64)
+    dkpe = np.empty((n, d_rope), dtype=np.float64)
+    dc = np.empty((n, d_c), dtype=np.float64)
+    qb, cb, kb, wb, db = _bits(q), _bits(c_kv), _bits(k_pe), _bits(w_kv_b), _bits(dout)
+    rc = lib.laga_oracle_bwd_keys(_u16(qb), _u16(cb), _u16(kb), _u16(wb), _u16(db), S, h, d_c, d_nope, d_rope,
+                                  d_v, float(softmax_scale), int(bool(causal)), int(bool(kv_round_bf16)),
+                                  keys_p, n, _f64(dk), _f64(dv), _f64(dkpe), _f64(dc))
+    if rc != 0:
+        raise RuntimeError(f"laga_oracle_bwd_keys failed with code {rc}")
+    return {"dk": torch.from_numpy(dk), "dv": torch.from_numpy(dv), "dk_pe": torch.from_numpy(dkpe),
+            "dc_kv": torch.from_numpy(dc)}

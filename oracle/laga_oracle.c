@@ -179,6 +179,166 @@ int laga_oracle_fwd(const uint16_t* q, const uint16_t* c_kv, const uint16_t* k_p
                                 causal, kv_round_bf16, NULL, 0, out, lse, NULL, NULL);
 }
 
+/* Backward restricted to a list of query rows: dq [n_rows][h][d_n+d_r] (a row of dQ depends on that
+ * query row only), plus the forward values out [n_rows][h][d_v] and lse [n_rows][h] it used. */
+int laga_oracle_bwd_rows(const uint16_t* q, const uint16_t* c_kv, const uint16_t* k_pe,
+                         const uint16_t* w_kv_b, const uint16_t* dout, int S, int h, int d_c, int d_nope,
+                         int d_rope, int d_v, double softmax_scale, int causal, int kv_round_bf16,
+                         const int* rows, int n_rows, double* dq, double* out, double* lse) {
+    if (!q || !c_kv || !k_pe || !w_kv_b || !dout || !rows || !dq || !out || !lse) return -1;
+    if (S < 1 || h < 1 || d_c < 1 || d_nope < 1 || d_rope < 0 || d_v < 1 || n_rows < 1) return -1;
+    for (int r = 0; r < n_rows; ++r) if (rows[r] < 0 || rows[r] >= S) return -1;
+    const int d_qk = d_nope + d_rope;
+    double* K = (double*)malloc(sizeof(double) * (size_t)h * S * d_qk);
+    double* V = (double*)malloc(sizeof(double) * (size_t)h * S * d_v);
+    int fail = (!K || !V);
+    if (fail) goto done;
+    up_project(c_kv, k_pe, w_kv_b, S, h, d_c, d_nope, d_rope, d_v, kv_round_bf16, K, V);
+#pragma omp parallel
+    {
+        double* x = (double*)malloc(sizeof(double) * (size_t)S);
+        if (!x) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for collapse(2) schedule(dynamic, 1)
+            for (int r = 0; r < n_rows; ++r) {
+                for (int i = 0; i < h; ++i) {
+                    const int s = rows[r];
+                    const int n_allowed = causal ? s + 1 : S;
+                    const double* Kh = K + (size_t)i * S * d_qk;
+                    const double* Vh = V + (size_t)i * S * d_v;
+                    const uint16_t* do_row = dout + ((size_t)s * h + i) * d_v;
+                    double* o = out + ((size_t)r * h + i) * d_v;
+                    double* dq_row = dq + ((size_t)r * h + i) * d_qk;
+                    lse[(size_t)r * h + i] =
+                        softmax_row(q + ((size_t)s * h + i) * d_qk, Kh, n_allowed, d_qk, softmax_scale, x);
+                    for (int j = 0; j < d_v; ++j) o[j] = 0.0;
+                    for (int t = 0; t < n_allowed; ++t)
+                        for (int j = 0; j < d_v; ++j) o[j] += x[t] * Vh[(size_t)t * d_v + j];
+                    double delta = 0.0;
+                    for (int j = 0; j < d_v; ++j) delta += bf16_bits_to_f64(do_row[j]) * o[j];
+                    for (int d = 0; d < d_qk; ++d) dq_row[d] = 0.0;
+                    for (int t = 0; t < n_allowed; ++t) {
+                        double dp = 0.0;
+                        for (int j = 0; j < d_v; ++j) dp += bf16_bits_to_f64(do_row[j]) * Vh[(size_t)t * d_v + j];
+                        double ds = x[t] * (dp - delta);
+                        for (int d = 0; d < d_qk; ++d) dq_row[d] += softmax_scale * ds * Kh[(size_t)t * d_qk + d];
+                    }
+                }
+            }
+        }
+        free(x);
+    }
+done:
+    free(K); free(V);
+    return fail ? -2 : 0;
+}
+
+/* Backward restricted to a list of key positions (for spot checks at sizes where the full backward
+ * takes minutes).  For each listed key t it returns the same numbers the full backward would:
+ * dk [n_keys][h][d_n+d_r], dv [n_keys][h][d_v], dk_pe [n_keys][d_r], dc_kv [n_keys][d_c].
+ * Only the query rows that can attend to a listed key are visited (s >= min key when causal). */
+int laga_oracle_bwd_keys(const uint16_t* q, const uint16_t* c_kv, const uint16_t* k_pe,
+                         const uint16_t* w_kv_b, const uint16_t* dout, int S, int h, int d_c, int d_nope,
+                         int d_rope, int d_v, double softmax_scale, int causal, int kv_round_bf16,
+                         const int* keys, int n_keys, double* dk, double* dv, double* dk_pe,
+                         double* dc_kv) {
+    if (!q || !c_kv || !k_pe || !w_kv_b || !dout || !keys || !dk || !dv || !dk_pe || !dc_kv) return -1;
+    if (S < 1 || h < 1 || d_c < 1 || d_nope < 1 || d_rope < 0 || d_v < 1 || n_keys < 1) return -1;
+    const int d_qk = d_nope + d_rope, per_head = d_nope + d_v, N = h * per_head;
+    int s_first = 0;
+    if (causal) {
+        s_first = keys[0];
+        for (int k = 1; k < n_keys; ++k) if (keys[k] < s_first) s_first = keys[k];
+    }
+    for (int k = 0; k < n_keys; ++k) if (keys[k] < 0 || keys[k] >= S) return -1;
+    double* K = (double*)malloc(sizeof(double) * (size_t)h * S * d_qk);
+    double* V = (double*)malloc(sizeof(double) * (size_t)h * S * d_v);
+    double* L = (double*)malloc(sizeof(double) * (size_t)h * S);
+    double* D = (double*)malloc(sizeof(double) * (size_t)h * S);
+    int fail = (!K || !V || !L || !D);
+    if (fail) goto done;
+    up_project(c_kv, k_pe, w_kv_b, S, h, d_c, d_nope, d_rope, d_v, kv_round_bf16, K, V);
+#pragma omp parallel
+    {
+        double* x = (double*)malloc(sizeof(double) * (size_t)S);
+        double* o = (double*)malloc(sizeof(double) * (size_t)d_v);
+        if (!x || !o) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for collapse(2) schedule(dynamic, 4)
+            for (int s = s_first; s < S; ++s) {
+                for (int i = 0; i < h; ++i) {
+                    const int n_allowed = causal ? s + 1 : S;
+                    const double* Kh = K + (size_t)i * S * d_qk;
+                    const double* Vh = V + (size_t)i * S * d_v;
+                    const uint16_t* do_row = dout + ((size_t)s * h + i) * d_v;
+                    L[(size_t)i * S + s] =
+                        softmax_row(q + ((size_t)s * h + i) * d_qk, Kh, n_allowed, d_qk, softmax_scale, x);
+                    for (int j = 0; j < d_v; ++j) o[j] = 0.0;
+                    for (int t = 0; t < n_allowed; ++t)
+                        for (int j = 0; j < d_v; ++j) o[j] += x[t] * Vh[(size_t)t * d_v + j];
+                    double delta = 0.0;
+                    for (int j = 0; j < d_v; ++j) delta += bf16_bits_to_f64(do_row[j]) * o[j];
+                    D[(size_t)i * S + s] = delta;
+                }
+            }
+        }
+        free(x); free(o);
+    }
+    if (fail) goto done;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int k = 0; k < n_keys; ++k) {
+        for (int i = 0; i < h; ++i) {
+            const int t = keys[k];
+            const double* Kh = K + (size_t)i * S * d_qk;
+            const double* Vh = V + (size_t)i * S * d_v;
+            double* dk_row = dk + ((size_t)k * h + i) * d_qk;
+            double* dv_row = dv + ((size_t)k * h + i) * d_v;
+            for (int d = 0; d < d_qk; ++d) dk_row[d] = 0.0;
+            for (int j = 0; j < d_v; ++j) dv_row[j] = 0.0;
+            for (int s = causal ? t : 0; s < S; ++s) {
+                const uint16_t* q_row = q + ((size_t)s * h + i) * d_qk;
+                const uint16_t* do_row = dout + ((size_t)s * h + i) * d_v;
+                double acc = 0.0;
+                for (int d = 0; d < d_qk; ++d) acc += bf16_bits_to_f64(q_row[d]) * Kh[(size_t)t * d_qk + d];
+                double p = exp(softmax_scale * acc - L[(size_t)i * S + s]);
+                double dp = 0.0;
+                for (int j = 0; j < d_v; ++j) dp += bf16_bits_to_f64(do_row[j]) * Vh[(size_t)t * d_v + j];
+                double ds = p * (dp - D[(size_t)i * S + s]);
+                for (int d = 0; d < d_qk; ++d) dk_row[d] += softmax_scale * ds * bf16_bits_to_f64(q_row[d]);
+                for (int j = 0; j < d_v; ++j) dv_row[j] += p * bf16_bits_to_f64(do_row[j]);
+            }
+        }
+    }
+    for (int k = 0; k < n_keys; ++k) {
+        for (int r = 0; r < d_rope; ++r) {
+            double acc = 0.0;
+            for (int i = 0; i < h; ++i) acc += dk[((size_t)k * h + i) * d_qk + d_nope + r];
+            dk_pe[(size_t)k * d_rope + r] = acc;
+        }
+        for (int c = 0; c < d_c; ++c) {
+            double acc = 0.0;
+            for (int i = 0; i < h; ++i)
+                for (int j = 0; j < per_head; ++j) {
+                    double g = (j < d_nope) ? dk[((size_t)k * h + i) * d_qk + j]
+                                            : dv[((size_t)k * h + i) * d_v + (j - d_nope)];
+                    acc += g * bf16_bits_to_f64(w_kv_b[(size_t)c * N + (size_t)i * per_head + j]);
+                }
+            dc_kv[(size_t)k * d_c + c] = acc;
+        }
+    }
+done:
+    free(K); free(V); free(L); free(D);
+    return fail ? -2 : 0;
+}
+
 /* Backward.  Outputs: dq [S][h][d_n+d_r], dc_kv [S][d_c], dk_pe [S][d_r], dw [d_c][h*(d_n+d_v)].
  * Optional (NULL to skip): out [S][h][d_v], lse [S][h] (the forward it differentiates), and
  * dk_full [S][h][d_n+d_r], dv_full [S][h][d_v] (the per-head K/V gradients before they are

@@ -1,0 +1,169 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
+seeded bf16 inputs.  Small cases are compared element by element (several tiles, ragged tails,
+degenerate sizes); the benchmark configurations are run at full size in the launch configuration
+bench.py times and compared on sampled query rows / key positions / heads the oracle can afford,
+plus identities that hold at any size.
+"""
+import pytest
+import torch
+
+from paper_2607_17644_b200.inputs import CONFIGS, CONFIG_SEEDS, LagaShape, make_inputs
+from parity import (TOL_LSE, TOL_LSE_UNROUNDED, check_dw, check_row_bands, check_tensor, f64, max_abs)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def laga():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2607_17644_b200 import laga as _laga
+    _laga.lib()          # must load: there is no fallback
+    return _laga
+
+
+def run_gpu(laga, tensors, causal, backward=True):
+    q, c_kv, k_pe, w, dout = (t.cuda() if t is not None else None for t in tensors)
+    out, lse, ws = laga.fwd(q, c_kv, k_pe, w, causal=causal)
+    laga.check_status(ws, where="laga_fwd")
+    res = {"out": out, "lse": lse}
+    if backward:
+        dq, dc_kv, dk_pe, dw, ws2 = laga.bwd(q, c_kv, k_pe, w, out, lse, dout, causal=causal)
+        laga.check_status(ws2, where="laga_bwd")
+        res.update(dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw=dw)
+    return {k: v.cpu() for k, v in res.items()}
+
+
+SMALL_CASES = [
+    # S, h, causal
+    (512, 2, True),      # benchmark config 0
+    (300, 3, True),      # ragged tail, odd head count
+    (300, 3, False),     # non-causal with a ragged last key tile
+    (1, 1, True),        # single token
+    (64, 1, True),
+    (129, 2, True),      # one row past a tile boundary
+    (1024, 4, True),     # eight key tiles
+    (200, 1, False),
+]
+
+
+@pytest.mark.parametrize("S,h,causal", SMALL_CASES)
+def test_forward_backward_elementwise(laga, oracle, S, h, causal):
+    sh = LagaShape(S=S, h=h)
+    tensors = make_inputs(sh, 1000 + S + h)
+    g = run_gpu(laga, tensors, causal)
+    q, c_kv, k_pe, w, dout = tensors
+    for rounded in (True, False):
+        r = oracle.bwd(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, causal=causal, kv_round_bf16=rounded,
+                       return_fwd=True)
+        check_tensor("out", g["out"], r["out"])
+        lse_err = max_abs(g["lse"], r["lse"])
+        assert lse_err <= (TOL_LSE if rounded else TOL_LSE_UNROUNDED), f"lse max-abs {lse_err:.3e}"
+        if S > 1:
+            check_tensor("dq", g["dq"], r["dq"])
+            check_tensor("dk_pe", g["dk_pe"], r["dk_pe"])
+        else:
+            # One token: the exact dq and dk_pe are zero (dP equals delta).  The GPU forms delta from
+            # the bf16-rounded O, so it returns rounding residue (~1e-7) instead: absolute check only.
+            assert max_abs(g["dq"], r["dq"]) <= 1e-5 and max_abs(g["dk_pe"], r["dk_pe"]) <= 1e-5
+        check_tensor("dc_kv", g["dc_kv"], r["dc_kv"])
+        check_dw(g["dw"], r["dw"])
+        if S >= 64:
+            check_row_bands("out", g["out"], r["out"])
+            check_row_bands("dq", g["dq"], r["dq"])
+
+
+def test_row_zero_and_head_shard_invariance(laga):
+    """Properties that need no oracle: causal row 0 of O is V[0] (here: the bf16 up-projection row the
+    library itself materialises), and a head shard's outputs do not depend on which other heads run
+    with it (paper Prop. 1), bit for bit."""
+    sh = LagaShape(S=384, h=4)
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in make_inputs(sh, 7))
+    out, lse, ws = laga.fwd(q, c_kv, k_pe, w)
+    laga.check_status(ws)
+    kv, word = laga.up_project(c_kv, w, sh.h)
+    laga.check_status(word)
+    v0 = kv[0].view(sh.h, 256)[:, 128:]
+    assert torch.equal(out[0], v0)
+    per = 256
+    out_a, lse_a, ws_a = laga.fwd(q[:, :1].contiguous(), c_kv, k_pe, w[:, :per].contiguous())
+    out_b, lse_b, ws_b = laga.fwd(q[:, 1:].contiguous(), c_kv, k_pe, w[:, per:].contiguous())
+    laga.check_status(ws_a), laga.check_status(ws_b)
+    assert torch.equal(torch.cat([out_a, out_b], 1), out) and torch.equal(torch.cat([lse_a, lse_b], 1), lse)
+
+
+def test_forward_is_repeatable_and_accum_flag(laga):
+    sh = LagaShape(S=640, h=2)
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in make_inputs(sh, 8))
+    out1, lse1, ws = laga.fwd(q, c_kv, k_pe, w)
+    out2, lse2, _ = laga.fwd(q, c_kv, k_pe, w, workspace=ws)
+    laga.check_status(ws)
+    assert torch.equal(out1, out2) and torch.equal(lse1, lse2)
+    dq, dc, dk, dw, ws2 = laga.bwd(q, c_kv, k_pe, w, out1, lse1, dout)
+    dq2, dc2, dk2, dw2, _ = laga.bwd(q, c_kv, k_pe, w, out1, lse1, dout, dw_kv_b=dw.clone(),
+                                     flags=laga.FLAG_ACCUM_DW, workspace=ws2)
+    laga.check_status(ws2)
+    assert torch.equal(dq, dq2) and torch.equal(dc, dc2) and torch.equal(dk, dk2)
+    assert (dw2 - 2 * dw).abs().max() <= 1e-3 * dw.abs().max()   # accumulated on top, up to atomic order
+
+
+def test_step_entry_points(laga):
+    """laga_up_project and laga_kv_backward against plain fp64 matmuls of the same bf16 bits."""
+    sh = LagaShape(S=333, h=3)
+    _, c_kv, _, w, _ = make_inputs(sh, 9)
+    g = torch.Generator().manual_seed(3)
+    dkv = torch.randn(sh.S, sh.n_cols, generator=g).to(torch.bfloat16)
+    kv, word = laga.up_project(c_kv.cuda(), w.cuda(), sh.h)
+    laga.check_status(word)
+    ref = f64(c_kv) @ f64(w)
+    assert max_abs(kv, ref) <= 2.0 ** -8 * float(ref.abs().max()) + 1e-6      # one bf16 rounding of the fp32 sum
+    dc, dw, word = laga.kv_backward(dkv.cuda(), c_kv.cuda(), w.cuda(), sh.h)
+    laga.check_status(word)
+    ref_dc = f64(dkv) @ f64(w).T
+    assert max_abs(dc, ref_dc) <= 2.0 ** -8 * float(ref_dc.abs().max()) + 1e-6
+    ref_dw = f64(c_kv).T @ f64(dkv)
+    assert max_abs(dw, ref_dw) <= 1e-5 * float(ref_dw.abs().max())            # fp32 accumulation only
+
+
+def _sample_rows(S, n, seed):
+    g = torch.Generator().manual_seed(seed)
+    edges = [0, 1, 7, 63, 64, 127, 128, 129, S - 129, S - 128, S - 1]
+    rnd = torch.randint(0, S, (n,), generator=g).tolist()
+    return sorted({r for r in edges + rnd if 0 <= r < S})
+
+
+@pytest.mark.parametrize("name", ["c1", "c2"])
+def test_benchmark_configs_sampled(laga, oracle, name):
+    """Full-size run of the benchmark shard (h=16; S=4096 and S=16384), checked on what the oracle can
+    compute one by one: sampled query rows (O, LSE, dQ), sampled key positions (dk_pe, dc_kv), one or
+    two whole heads of dW, and bilinear trace identities over the complete GPU outputs."""
+    sh = CONFIGS[name]
+    tensors = make_inputs(sh, CONFIG_SEEDS[name])
+    q, c_kv, k_pe, w, dout = tensors
+    g = run_gpu(laga, tensors, True)
+    rows = _sample_rows(sh.S, 24, 1)
+    r = oracle.bwd_rows(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, rows, kv_round_bf16=True)
+    check_tensor("out[rows]", g["out"][rows], r["out"])
+    assert max_abs(g["lse"][rows], r["lse"]) <= TOL_LSE
+    check_tensor("dq[rows]", g["dq"][rows], r["dq"])
+    check_row_bands("out[rows]", g["out"][rows], r["out"], row_index=rows)
+    check_row_bands("dq[rows]", g["dq"][rows], r["dq"], row_index=rows)
+    # key side: late keys are cheap for the oracle (few query rows attend to them)
+    keys = sorted({sh.S - 1, sh.S - 2, sh.S - 64, sh.S - 65, sh.S - 128, sh.S - 129, sh.S - 200})
+    if name == "c1":
+        keys = sorted(set(keys) | {0, 1, 63, 64, 127, 128, 1000, 2047, 2048, 3000})
+    k = oracle.bwd_keys(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, keys, kv_round_bf16=True)
+    check_tensor("dk_pe[keys]", g["dk_pe"][keys], k["dk_pe"])
+    check_tensor("dc_kv[keys]", g["dc_kv"][keys], k["dc_kv"])
+    # dW: whole heads via the head-shard property (a head's dW columns depend on that head only)
+    for head in ([3, 15] if name == "c1" else [9]):
+        cols = slice(head * 256, (head + 1) * 256)
+        rh = oracle.bwd(q[:, head:head + 1].contiguous(), c_kv, k_pe, w[:, cols].contiguous(),
+                        dout[:, head:head + 1].contiguous(), sh.d_v, sh.softmax_scale, kv_round_bf16=True)
+        check_dw(g["dw"][:, cols], rh["dw"])
+        check_tensor(f"dq[head {head}]", g["dq"][:, head:head + 1], rh["dq"])
+    # identities over the complete outputs: <W, dW> = <c_kv, dc_kv> (both equal <KV, dKV>)
+    a = float((f64(w) * f64(g["dw"])).sum())
+    b = float((f64(c_kv) * f64(g["dc_kv"])).sum())
+    scale = float(f64(w).norm() * f64(g["dw"]).norm())
+    assert abs(a - b) <= 1e-3 * scale, (a, b, scale)

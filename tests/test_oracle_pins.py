@@ -317,3 +317,21 @@ def test_config_distribution_statistics(oracle):
     assert 0.9 < float(kn.std()) < 1.1 and 0.9 < float(v.std()) < 1.1
     excess = lse - torch.tensor(rows, dtype=torch.float64).add(1).log()[:, None]
     assert 0.4 < float(excess.mean()) < 0.6
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_row_and_key_subsets_match_full_backward(oracle, causal):
+    """The spot-check entry points return exactly what the (autograd-pinned) full backward returns."""
+    sh = LagaShape(S=70, h=3, d_c=16, d_nope=8, d_rope=4, d_v=8)
+    q, c_kv, k_pe, w, dout = make_inputs(sh, 26)
+    full = oracle.bwd(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, causal=causal, return_fwd=True,
+                      return_dkv=True)
+    rows = [0, 69, 17, 40]
+    r = oracle.bwd_rows(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, rows, causal=causal)
+    assert torch.equal(r["dq"], full["dq"][rows]) and torch.equal(r["out"], full["out"][rows])
+    assert torch.equal(r["lse"], full["lse"][rows])
+    keys = [69, 33, 50, 68]
+    k = oracle.bwd_keys(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, keys, causal=causal)
+    assert (k["dk"] - full["dk"][keys]).abs().max() < 1e-13 and (k["dv"] - full["dv"][keys]).abs().max() < 1e-13
+    assert (k["dk_pe"] - full["dk_pe"][keys]).abs().max() < 1e-13
+    assert (k["dc_kv"] - full["dc_kv"][keys]).abs().max() < 1e-12
