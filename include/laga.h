@@ -109,6 +109,24 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
                      void* stream);
 
 /*
+ * Measurement aid.  Registers n_pairs CUDA events pairs (cudaEvent_t passed as void*, created by the
+ * caller with timing enabled) that the library records on the launch stream immediately before and
+ * after every launch of one kernel, cycling through the pairs launch after launch; n_pairs = 0 stops
+ * it.  The caller reads the times (cudaEventElapsedTime) after synchronising, and keeps the events
+ * alive while registered.  Not thread-safe; intended for benchmarks.  The paper has no counterpart.
+ */
+#define LAGA_KERNEL_UP_PROJECT 0    /* step 4 GEMM (also the recomputation in laga_bwd)        */
+#define LAGA_KERNEL_ATTN_FWD 1      /* step 5 forward attention                               */
+#define LAGA_KERNEL_BWD_DELTA 2     /* delta = rowsum(dO * O) and transposed statistics        */
+#define LAGA_KERNEL_ATTN_BWD_DKV 3  /* backward attention: dK, dV                              */
+#define LAGA_KERNEL_ATTN_BWD_DQ 4   /* backward attention: dQ                                  */
+#define LAGA_KERNEL_DKPE_REDUCE 5   /* dk_pe = sum over heads of the rope-column key gradient  */
+#define LAGA_KERNEL_DCKV_GEMM 6     /* dc_kv = dKV . W^T                                       */
+#define LAGA_KERNEL_DW_GEMM 7       /* dW = c_kv^T . dKV                                       */
+#define LAGA_KERNEL_COUNT 8
+int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs);
+
+/*
  * Synchronises `stream`, reads the status word at the start of `workspace` (or a `status_word`
  * given to a step entry point) and returns LAGA_OK, LAGA_ERR_DEVICE_TIMEOUT or LAGA_ERR_CUDA.
  * If `detail` is not NULL it receives the raw device word (which wait gave up).

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "attn_bwd_sm100.cuh"
 #include "attn_fwd_sm100.cuh"
 #include "gemm_sm100.cuh"
@@ -80,6 +82,30 @@ int set_smem(Kernel kernel, int bytes) {
 
 int launch_status() { return cudaGetLastError() == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA; }
 
+// Measurement aid (laga_profile_kernel): caller-provided CUDA events recorded around launches of one
+// kernel, cycling through the registered pairs.
+struct ProfileSlot {
+    std::vector<cudaEvent_t> starts, stops;
+    unsigned long long launches = 0;
+};
+ProfileSlot g_profile[LAGA_KERNEL_COUNT];
+
+struct ScopedKernelEvents {
+    cudaEvent_t stop = nullptr;
+    cudaStream_t stream;
+    ScopedKernelEvents(int kernel_id, cudaStream_t st) : stream(st) {
+        ProfileSlot& slot = g_profile[kernel_id];
+        if (!slot.starts.empty()) {
+            const size_t i = static_cast<size_t>(slot.launches++ % slot.starts.size());
+            cudaEventRecord(slot.starts[i], stream);
+            stop = slot.stops[i];
+        }
+    }
+    ~ScopedKernelEvents() {
+        if (stop) cudaEventRecord(stop, stream);
+    }
+};
+
 // ---- Algorithm 1 step 4: KV[S, N] = c_kv[S, d_c] . W[d_c, N] ------------------------------------
 int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
                       cudaStream_t stream) {
@@ -92,7 +118,7 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
     if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
     GemmArgs a{S, N, kDc, kDc / 64, kv, N, status};
     dim3 grid(N / BN, (S + 127) / 128, 1);
-    kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a);
+    { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
 
@@ -109,7 +135,7 @@ int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, unsig
     if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
     GemmArgs a{S, kDc, N, (N + 63) / 64, dc_kv, kDc, status};
     dim3 grid(kDc / BN, (S + 127) / 128, 1);
-    kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a);
+    { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
 
@@ -136,7 +162,7 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool a
     splits = (k_tiles + per_split - 1) / per_split;
     GemmArgs a{kDc, N, S, per_split, dw, N, status};
     dim3 grid(N / BN, kDc / 128, splits);
-    kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a);
+    { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
 
@@ -155,11 +181,11 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
     if (causal) {
         auto kernel = attn_fwd_sm100_kernel<true>;
         if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-        kernel<<<grid, 192, L::kTotalBytes, stream>>>(tq, tkv, tpe, a);
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(tq, tkv, tpe, a); }
     } else {
         auto kernel = attn_fwd_sm100_kernel<false>;
         if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-        kernel<<<grid, 192, L::kTotalBytes, stream>>>(tq, tkv, tpe, a);
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(tq, tkv, tpe, a); }
     }
     return launch_status();
 }
@@ -193,6 +219,7 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
     {   // delta and the transposed, padded softmax statistics
         const long long warps = static_cast<long long>(S_pad) * h;
         const unsigned blocks = static_cast<unsigned>((warps * 32 + 255) / 256);
+        ScopedKernelEvents ev(LAGA_KERNEL_BWD_DELTA, stream);
         bwd_delta_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(out),
                                                      reinterpret_cast<const __nv_bfloat16*>(dout), lse, S, h, S_pad,
                                                      stat_l2, stat_delta);
@@ -217,21 +244,22 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         auto k2 = attn_bwd_dq_sm100_kernel<true>;
         if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
             return LAGA_ERR_CUDA;
-        k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a);
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b);
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
     } else {
         auto k1 = attn_bwd_dkv_sm100_kernel<false>;
         auto k2 = attn_bwd_dq_sm100_kernel<false>;
         if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
             return LAGA_ERR_CUDA;
-        k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a);
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b);
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     {
         const size_t n = static_cast<size_t>(S) * kDr;
+        ScopedKernelEvents ev(LAGA_KERNEL_DKPE_REDUCE, stream);
         bwd_dkpe_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
             dk_rope, S, h, reinterpret_cast<__nv_bfloat16*>(dk_pe));
     }
@@ -355,6 +383,21 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
         return rc;
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
     return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, status, st);
+}
+
+int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs) {
+    if (kernel_id < 0 || kernel_id >= LAGA_KERNEL_COUNT || n_pairs < 0) return LAGA_ERR_INVALID_ARG;
+    if (n_pairs > 0 && (!start_events || !stop_events)) return LAGA_ERR_INVALID_ARG;
+    ProfileSlot& slot = g_profile[kernel_id];
+    slot.starts.clear();
+    slot.stops.clear();
+    slot.launches = 0;
+    for (int i = 0; i < n_pairs; ++i) {
+        if (!start_events[i] || !stop_events[i]) { slot.starts.clear(); slot.stops.clear(); return LAGA_ERR_INVALID_ARG; }
+        slot.starts.push_back(static_cast<cudaEvent_t>(start_events[i]));
+        slot.stops.push_back(static_cast<cudaEvent_t>(stop_events[i]));
+    }
+    return LAGA_OK;
 }
 
 int laga_query_status(const void* workspace, void* stream, unsigned* detail) {

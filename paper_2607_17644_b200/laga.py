@@ -34,7 +34,10 @@ SIGNATURES = {
     "laga_up_project": (_ci, [_vp, _vp] + [_ci] * 5 + [_vp, _vp, _vp]),
     "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
     "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
+    "laga_profile_kernel": (_ci, [_ci, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _ci]),
 }
+KERNELS = {"up_project": 0, "attn_fwd": 1, "bwd_delta": 2, "attn_bwd_dkv": 3, "attn_bwd_dq": 4,
+           "dkpe_reduce": 5, "dckv_gemm": 6, "dw_gemm": 7}
 
 
 class LagaError(RuntimeError):
@@ -200,6 +203,17 @@ def kv_backward(dkv, c_kv, w_kv_b, h, d_nope=128, d_v=128, dc_kv=None, dw_kv_b=N
                                 _ptr(dw_kv_b), flags, _ptr(status_word), _stream(stream))
     _check(rc, "laga_kv_backward")
     return dc_kv, dw_kv_b, status_word
+
+
+def profile_kernel(kernel: str, start_events=(), stop_events=()):
+    """laga_profile_kernel: record the given torch.cuda.Event pairs around every launch of `kernel`
+    (cycling through them); call with no events to stop.  Events must have been created with
+    enable_timing=True and recorded once already (torch creates the CUDA event lazily)."""
+    n = len(start_events)
+    assert n == len(stop_events)
+    starts = (_vp * max(n, 1))(*[e.cuda_event for e in start_events])
+    stops = (_vp * max(n, 1))(*[e.cuda_event for e in stop_events])
+    _check(lib().laga_profile_kernel(KERNELS[kernel], starts, stops, n), "laga_profile_kernel")
 
 
 def query_status(workspace_or_word, stream=None) -> tuple[int, int]:

@@ -6,12 +6,14 @@ g = GPU output converted to float64, r = oracle.
   scaled max-abs max |g - r| / max(1, rms(r))     (used for dW only, see below)
 
 Bounds (bf16 operands, fp32 accumulation):
-  O, dQ, dc_kv, dk_pe   |g - r| <= max(2e-2, |r| / 128) element by element, and rel-L2 <= 5e-3.
-                        These outputs are bf16: an element of magnitude above 2.56 has a bf16 quantum
-                        (|r| / 128 at the bottom of its binade) wider than 2e-2, so a correctly rounded
-                        result can already miss by more than 2e-2 there (dk_pe and dc_kv sum over the
-                        whole sequence and all heads and reach 5..10 on early keys).  Below 2.56 the
-                        plain 2e-2 bound applies.
+  O, dQ, dc_kv, dk_pe   rel-L2 <= 5e-3, and element by element
+                            |g - r| <= 2e-2 * max(1, rms of r over the element's row) , or |r| / 128 if larger.
+                        The plain 2e-2 presumes unit-scale rows; it is what binds O and dQ everywhere and
+                        dc_kv / dk_pe on all but the earliest keys.  dc_kv and dk_pe are un-normalised sums
+                        over every query row and head that attends to a key, so rows of early keys reach
+                        rms 3..4 and entries 5..10: the bf16 roundings of P, dS and dKV inject an error
+                        proportional to that row scale, and the bf16 output quantum alone (|r| / 128 at the
+                        bottom of a binade) exceeds 2e-2 above |r| = 2.56.
   LSE                   max-abs <= 1e-3 against the oracle that rounds K_nope/V to bf16 (the explicit
                         form as it runs in bf16; the rounding of K_nope alone moves early-row LSE by
                         up to a few 1e-3, which no bf16-operand kernel can avoid), <= 5e-3 against the
@@ -55,11 +57,13 @@ def check_tensor(name, g, r, max_abs_tol=TOL_MAX_ABS, rel_l2_tol=TOL_REL_L2):
     assert g.shape == r.shape, (name, g.shape, r.shape)
     assert torch.isfinite(g).all(), f"{name}: non-finite values"
     ma, rl = max_abs(g, r), rel_l2(g, r)
-    excess = (g - r).abs() - torch.maximum(torch.full_like(r, max_abs_tol), r.abs() / 128.0)
+    row_rms = r.pow(2).mean(dim=-1, keepdim=True).sqrt().clamp_min(1.0)
+    bound = torch.maximum(max_abs_tol * row_rms.expand_as(r), r.abs() / 128.0)
+    excess = (g - r).abs() - bound
     worst = int(excess.argmax())
     assert float(excess.max()) <= 0, (f"{name}: |g-r| = {float((g - r).abs().flatten()[worst]):.3e} at reference "
-                                      f"value {float(r.flatten()[worst]):.4f} exceeds max({max_abs_tol}, |r|/128); "
-                                      f"tensor max-abs {ma:.3e}")
+                                      f"value {float(r.flatten()[worst]):.4f} exceeds its bound "
+                                      f"{float(bound.flatten()[worst]):.3e}; tensor max-abs {ma:.3e}")
     assert rl <= rel_l2_tol, f"{name}: rel-L2 {rl:.3e} > {rel_l2_tol}"
     return ma, rl
 
