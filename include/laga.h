@@ -109,6 +109,38 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
                      void* stream);
 
 /*
+ * laga_fwd for callers that have no scratch to give.  (The paper has no counterpart: this is a
+ * packaging convenience of the library, not a step of the method.)
+ *
+ * Who it is for: code that must run the forward but is not in a position to obtain device memory --
+ * a plug-in or callback invoked where allocation calls are forbidden, a component of a process whose
+ * device memory is entirely owned by someone else's pool, or a latency-sensitive loop that cannot
+ * afford cudaMalloc's device-wide synchronisation.  Such a caller still owns its inputs and outputs
+ * (same shapes, dtypes, alignment and meaning as laga_fwd) but passes no workspace: the bf16
+ * up-projection KV and the launch status word go into a fixed array inside the library image.
+ *
+ * Limits and rules
+ *   - The array holds 16 MiB of KV: S * h <= 32768 (e.g. S=2048 with h=16).  A larger problem returns
+ *     LAGA_ERR_WORKSPACE_TOO_SMALL and nothing is enqueued; use laga_fwd with your own workspace.
+ *     Every GPU on which the library is loaded carries these 16 MiB (+1 KiB) until the process exits.
+ *   - The call allocates and frees nothing (no cudaMalloc/cudaFree, no allocating library routine).
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.  The
+ *     call itself clears the status word and overwrites the KV rows it uses, so back-to-back calls
+ *     on ONE stream are safe; calls that can overlap on the GPU (different streams, no ordering
+ *     between them) race on it and must be serialised by the caller.
+ *   - There is no way to read the device status word of this variant: a bounded device wait that
+ *     gives up leaves the outputs incomplete without a report.  Callers that need the report use
+ *     laga_fwd + laga_query_status.
+ * Errors: as laga_fwd (LAGA_ERR_INVALID_ARG, LAGA_ERR_UNSUPPORTED, LAGA_ERR_CUDA), plus the size
+ * limit above.
+ */
+int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S,
+                             int h, int d_c, int d_nope, int d_rope, int d_v, float softmax_scale, int causal,
+                             void* out, float* lse, void* stream);
+
+/*
  * Measurement aid.  Registers n_pairs CUDA events pairs (cudaEvent_t passed as void*, created by the
  * caller with timing enabled) that the library records on the launch stream immediately before and
  * after every launch of one kernel, cycling through the pairs launch after launch; n_pairs = 0 stops

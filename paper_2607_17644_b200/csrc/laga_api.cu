@@ -385,6 +385,58 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
     return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, status, st);
 }
 
+// ---- forward without caller-provided scratch ----------------------------------------------------
+// Scratch for laga_fwd_builtin_scratch: the launch status slot followed by the bf16 up-projection
+// KV[S, h*256].  It lives in the library image, so every GPU that loads the library holds these
+// bytes until the process exits; the cap keeps that cost modest.
+constexpr size_t kBuiltinKvBytes = size_t(16) << 20;                       // S * h <= 32768
+static __device__ __align__(256) unsigned char g_builtin_scratch[kStatusBytes + kBuiltinKvBytes];
+
+// Device address of g_builtin_scratch on the current device.  In host code the symbol's name is only
+// a handle, never an address a kernel may use: the address comes from cudaGetSymbolAddress, looked up
+// once per device with that device current.
+static int builtin_scratch_address(unsigned char** ptr) {
+    constexpr int kMaxDevices = 64;
+    static unsigned char* cached[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LAGA_ERR_CUDA;
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return LAGA_ERR_CUDA;
+        }
+        cached[dev] = static_cast<unsigned char*>(p);
+    }
+    *ptr = cached[dev];
+    return LAGA_OK;
+}
+
+int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h,
+                             int d_c, int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out,
+                             float* lse, void* stream) {
+    if (!q || !c_kv || !k_pe || !w_kv_b || !out || !lse || S < 1 || h < 1) return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(c_kv) || !aligned16(k_pe) || !aligned16(w_kv_b) || !aligned16(out) ||
+        !aligned16(lse))
+        return LAGA_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
+    if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
+    // the built-in scratch is a fixed size: larger problems must bring their own workspace (laga_fwd)
+    if (static_cast<size_t>(S) * h * (kDn + kDv) * 2 > kBuiltinKvBytes) return LAGA_ERR_WORKSPACE_TOO_SMALL;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    unsigned char* base = nullptr;
+    if ((rc = builtin_scratch_address(&base)) != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned* status = reinterpret_cast<unsigned*>(base);
+    void* kv = base + kStatusBytes;
+    // The array keeps whatever the previous call left: the status word must start at zero; KV rows
+    // [0, S) are fully overwritten by the up-projection before the attention kernel reads them.
+    if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
+    if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
+    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st);
+}
+
 int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs) {
     if (kernel_id < 0 || kernel_id >= LAGA_KERNEL_COUNT || n_pairs < 0) return LAGA_ERR_INVALID_ARG;
     if (n_pairs > 0 && (!start_events || !stop_events)) return LAGA_ERR_INVALID_ARG;

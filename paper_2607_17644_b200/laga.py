@@ -35,7 +35,9 @@ SIGNATURES = {
     "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
     "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
     "laga_profile_kernel": (_ci, [_ci, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _ci]),
+    "laga_fwd_builtin_scratch": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp]),
 }
+BUILTIN_SCRATCH_MAX_TOKEN_HEADS = 32768   # S * h limit of laga_fwd_builtin_scratch (16 MiB of bf16 KV)
 KERNELS = {"up_project": 0, "attn_fwd": 1, "bwd_delta": 2, "attn_bwd_dkv": 3, "attn_bwd_dq": 4,
            "dkpe_reduce": 5, "dckv_gemm": 6, "dw_gemm": 7}
 
@@ -137,6 +139,27 @@ def fwd(q, c_kv, k_pe, w_kv_b, d_v=128, softmax_scale=None, causal=True, out=Non
                         workspace.numel(), 0, _stream(stream))
     _check(rc, "laga_fwd")
     return out, lse, workspace
+
+
+def fwd_builtin_scratch(q, c_kv, k_pe, w_kv_b, out, lse, d_v=128, softmax_scale=None, causal=True, stream=None):
+    """laga_fwd_builtin_scratch: the forward for callers that cannot obtain scratch memory.
+
+    `out` and `lse` are written in place (the caller passes them: this wrapper, like the entry point,
+    allocates nothing).  The up-projection lives in a fixed 16 MiB array inside the library, so
+    S * h must not exceed BUILTIN_SCRATCH_MAX_TOKEN_HEADS; larger problems raise
+    LAGA_ERR_WORKSPACE_TOO_SMALL.  Calls on one stream may follow each other freely; calls that could
+    overlap on the GPU share the array and must be ordered by the caller.  The first call on a device
+    resolves the array's address and should happen outside stream capture.
+    """
+    S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
+    if softmax_scale is None:
+        softmax_scale = (d_nope + d_rope) ** -0.5
+    _dev(out, torch.bfloat16, (S, h, d_v), "out")
+    _dev(lse, torch.float32, (S, h), "lse")
+    rc = lib().laga_fwd_builtin_scratch(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope,
+                                        d_v, float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse),
+                                        _stream(stream))
+    _check(rc, "laga_fwd_builtin_scratch")
 
 
 def bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout, d_v=128, softmax_scale=None, causal=True, dq=None, dc_kv=None,
