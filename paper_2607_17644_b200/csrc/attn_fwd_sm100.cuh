@@ -173,31 +173,36 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             mbar_arrive(&s_free[s]);
 
             const bool edge = (j == n_kv - 1);
-            float mx = -INFINITY;
+            if (edge) {
 #pragma unroll
-            for (int c = 0; c < 128; ++c) {
-                float x = __uint_as_float(sv[c]);
-                if (edge) {
+                for (int c = 0; c < 128; ++c) {
                     const int t = j * 128 + c;
-                    if ((kCausal && t > sq_idx) || t >= args.S) x = -INFINITY;
+                    if ((kCausal && t > sq_idx) || t >= args.S) sv[c] = __float_as_uint(-INFINITY);
                 }
-                sv[c] = __float_as_uint(x);
-                mx = fmaxf(mx, x);
             }
+            // eight independent chains: a single warp per scheduler cannot hide a 128-deep dependency
+            float mxs[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) mxs[e] = __uint_as_float(sv[e]);
+#pragma unroll
+            for (int c = 8; c < 128; ++c) mxs[c & 7] = fmaxf(mxs[c & 7], __uint_as_float(sv[c]));
+            const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                   fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
             const float m_new = fmaxf(m_run, mx * args.scale_log2);
             // Lazy rescale: keep the old reference max unless it fell behind by more than 2^8.
             const bool move = (m_new - m_run) > 8.0f;
             const float alpha = move ? fast_exp2(m_run - m_new) : 1.0f;
             if (move) m_run = m_new;
-            float sum = 0.f;
+            float sums[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             uint32_t pk[64];
 #pragma unroll
             for (int c = 0; c < 64; ++c) {
                 const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * c]), args.scale_log2, -m_run));
                 const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * c + 1]), args.scale_log2, -m_run));
-                sum += p0 + p1;
+                sums[c & 7] += p0 + p1;
                 pk[c] = pack_bf16x2(p0, p1);
             }
+            const float sum = ((sums[0] + sums[1]) + (sums[2] + sums[3])) + ((sums[4] + sums[5]) + (sums[6] + sums[7]));
             l_run = l_run * alpha + sum;
 
             if (j > 0) {
