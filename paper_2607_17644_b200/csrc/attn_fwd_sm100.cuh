@@ -4,11 +4,14 @@
 // band k_pe[S, 64] is a separate TMA box, so the 192-wide key is never assembled in memory.
 //
 // One CTA owns 128 query rows of one head and walks the key tiles (128 keys each).
-//   warp 0      TMA producer: Q once, then K (2 stages) and V (1 stage) tiles
-//   warp 1      MMA issuer:   S = Q K^T (12 tcgen05.mma of K=16) into a double-buffered TMEM tile,
-//                             O += P V  (8 tcgen05.mma) into a TMEM accumulator
-//   warps 2..5  softmax: one thread per query row; online max / sum in registers, P written to
-//               shared memory as the bf16 A operand of the second contraction, lazy rescale of O
+//   warp 0      TMA producer: Q once, then K and V tiles, two stages each
+//   warp 1      MMA issuer:   S = Q K^T (12 tcgen05.mma of K=16) into one of two TMEM tiles;
+//                             O += P V  (8 tcgen05.mma, A operand read from TMEM) into a TMEM accumulator
+//   warps 2..5  softmax: one thread per query row; online max / sum in registers; P is written back as
+//               packed bf16 over the first 64 columns of the S tile it came from and consumed from
+//               there by the second contraction; lazy rescale of O
+// The score tile for key tile j+2 reuses the TMEM columns of tile j; it is issued after P_j V_j by the
+// same thread, and the tensor pipe executes a thread's MMAs in order, so no extra barrier guards it.
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -26,9 +29,8 @@ struct AttnFwdSmem {
     static constexpr int kSlab = 128 * 128;             // 128 rows x 128 bytes
     static constexpr int kQ = 0;                        // 3 slabs
     static constexpr int kK = kQ + 3 * kSlab;           // 2 stages x 3 slabs (nope lo, nope hi, rope)
-    static constexpr int kV = kK + 2 * 3 * kSlab;       // 1 stage x 2 slabs
-    static constexpr int kP = kV + 2 * kSlab;           // 2 slabs
-    static constexpr int kBar = kP + 2 * kSlab;
+    static constexpr int kV = kK + 2 * 3 * kSlab;       // 2 stages x 2 slabs
+    static constexpr int kBar = kV + 2 * 2 * kSlab;
     static constexpr int kTotalBytes = kBar + 256 + 1024;
 };
 
@@ -49,10 +51,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     uint64_t* q_full = bars + 0;
     uint64_t* k_full = bars + 1;     // [2]
     uint64_t* k_empty = bars + 3;    // [2]
-    uint64_t* v_full = bars + 5;
-    uint64_t* v_empty = bars + 6;
-    uint64_t* s_full = bars + 7;     // [2]
-    uint64_t* s_free = bars + 9;     // [2]
+    uint64_t* v_full = bars + 5;     // [2]
+    uint64_t* v_empty = bars + 7;    // [2]
+    uint64_t* s_full = bars + 9;     // [2]
     uint64_t* p_full = bars + 11;
     uint64_t* pv_done = bars + 12;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
@@ -69,9 +70,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         mbar_init(q_full, 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
-            mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 128);
+            mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+            mbar_init(&s_full[s], 1);
         }
-        mbar_init(v_full, 1); mbar_init(v_empty, 1);
         mbar_init(p_full, 128); mbar_init(pv_done, 1);
         abort_flag->value = 0;
         mbar_fence_init();
@@ -89,25 +90,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
             for (int c = 0; c < 3; ++c)
                 tma_load_2d(smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
-            auto load_k = [&](int j) -> bool {
+            for (int j = 0; j < n_kv; ++j) {
                 const int s = j & 1;
-                if (!mbar_wait(&k_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, args.status, 0x10)) return false;
-                uint8_t* dst = smem + L::kK + s * 3 * L::kSlab;
+                const uint32_t ph_free = ((j >> 1) & 1) ^ 1;
+                if (!mbar_wait(&k_empty[s], ph_free, abort_flag, args.status, 0x10)) break;
+                uint8_t* dk = smem + L::kK + s * 3 * L::kSlab;
                 mbar_arrive_expect_tx(&k_full[s], 3 * L::kSlab);
-                tma_load_2d(dst, &tmap_kv, &k_full[s], head * 256, j * 128);
-                tma_load_2d(dst + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * 128);
-                tma_load_2d(dst + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * 128);
-                return true;
-            };
-            bool ok = load_k(0);
-            for (int j = 0; j < n_kv && ok; ++j) {
-                if (j + 1 < n_kv) ok = load_k(j + 1);
-                if (!ok) break;
-                ok = mbar_wait(v_empty, (j & 1) ^ 1, abort_flag, args.status, 0x11);
-                if (!ok) break;
-                mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
-                tma_load_2d(smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
-                tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
+                tma_load_2d(dk, &tmap_kv, &k_full[s], head * 256, j * 128);
+                tma_load_2d(dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * 128);
+                tma_load_2d(dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * 128);
+                if (!mbar_wait(&v_empty[s], ph_free, abort_flag, args.status, 0x11)) break;
+                uint8_t* dv = smem + L::kV + s * 2 * L::kSlab;
+                mbar_arrive_expect_tx(&v_full[s], 2 * L::kSlab);
+                tma_load_2d(dv, &tmap_kv, &v_full[s], head * 256 + 128, j * 128);
+                tma_load_2d(dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * 128);
             }
         }
     } else if (warp == 1) {
@@ -115,29 +111,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);
             const uint32_t sq = smem_u32(smem + L::kQ);
-            const uint32_t sv = smem_u32(smem + L::kV);
-            const uint32_t sp = smem_u32(smem + L::kP);
-            auto issue_pv = [&](int j) -> bool {
-                if (!mbar_wait(v_full, j & 1, abort_flag, args.status, 0x20)) return false;
-                if (!mbar_wait(p_full, j & 1, abort_flag, args.status, 0x21)) return false;
-                tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t da = desc_k_major(sp + (kk >> 2) * L::kSlab + (kk & 3) * 32);
-                    const uint64_t db = desc_mn_major(sv + kk * 2048, L::kSlab);
-                    mma_ss(tmem_o, da, db, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
-                }
-                mma_commit(v_empty);
-                mma_commit(pv_done);
-                return true;
-            };
-            bool ok = mbar_wait(q_full, 0, abort_flag, args.status, 0x22);
-            for (int j = 0; j < n_kv && ok; ++j) {
+            auto issue_qk = [&](int j) -> bool {
                 const int s = j & 1;
-                const uint32_t ph = (j >> 1) & 1;
-                ok = mbar_wait(&k_full[s], ph, abort_flag, args.status, 0x23) &&
-                     mbar_wait(&s_free[s], ph ^ 1, abort_flag, args.status, 0x24);
-                if (!ok) break;
+                if (!mbar_wait(&k_full[s], (j >> 1) & 1, abort_flag, args.status, 0x23)) return false;
                 tc_fence_after_sync();
                 const uint32_t sk = smem_u32(smem + L::kK + s * 3 * L::kSlab);
 #pragma unroll
@@ -148,16 +124,32 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 }
                 mma_commit(&k_empty[s]);
                 mma_commit(&s_full[s]);
-                if (j > 0) ok = issue_pv(j - 1);
+                return true;
+            };
+            bool ok = mbar_wait(q_full, 0, abort_flag, args.status, 0x22);
+            if (ok) ok = issue_qk(0);
+            if (ok && n_kv > 1) ok = issue_qk(1);
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int s = j & 1;
+                ok = mbar_wait(&v_full[s], (j >> 1) & 1, abort_flag, args.status, 0x20) &&
+                     mbar_wait(p_full, j & 1, abort_flag, args.status, 0x21);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t sv = smem_u32(smem + L::kV + s * 2 * L::kSlab);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)   // A = P_j: packed bf16, 8 TMEM columns per 16 keys
+                    mma_ts(tmem_o, tmem_base + s * 128 + kk * 8, desc_mn_major(sv + kk * 2048, L::kSlab), idesc_pv,
+                           (j > 0 || kk > 0) ? 1u : 0u);
+                mma_commit(&v_empty[s]);
+                mma_commit(pv_done);
+                if (j + 2 < n_kv) ok = issue_qk(j + 2);
             }
-            if (ok) issue_pv(n_kv - 1);
         }
     } else {
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;          // row inside the tile == TMEM lane
         const int sq_idx = q0 + row;                  // global query index
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-        uint8_t* p_smem = smem + L::kP;
         float m_run = -INFINITY, l_run = 0.f;         // running max (scaled, log2 domain) and sum
         bool ok = true;
         for (int j = 0; j < n_kv; ++j) {
@@ -169,8 +161,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld_x32(tmem_base + lane_addr + s * 128 + c * 32, sv + c * 32);
             tmem_ld_wait();
-            tc_fence_before_sync();
-            mbar_arrive(&s_free[s]);
 
             const bool edge = (j == n_kv - 1);
             if (edge) {
@@ -205,29 +195,24 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             const float sum = ((sums[0] + sums[1]) + (sums[2] + sums[3])) + ((sums[4] + sums[5]) + (sums[6] + sums[7]));
             l_run = l_run * alpha + sum;
 
-            if (j > 0) {
+            if (j > 0 && __any_sync(0xffffffffu, move)) {
+                // O must be at rest: P_{j-1} V_{j-1} finished, P_j V_j not issued before p_full below.
                 ok = mbar_wait_warp(pv_done, (j - 1) & 1, abort_flag, args.status, 0x31);
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (__any_sync(0xffffffffu, move)) {
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
-                        tmem_ld_wait();
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int v = 0; v < 32; ++v) o[v] = __float_as_uint(__uint_as_float(o[v]) * alpha);
-                        tmem_st_x32(tmem_o + lane_addr + c * 32, o);
-                    }
-                    tmem_st_wait();
+                    for (int v = 0; v < 32; ++v) o[v] = __float_as_uint(__uint_as_float(o[v]) * alpha);
+                    tmem_st_x32(tmem_o + lane_addr + c * 32, o);
                 }
             }
-#pragma unroll
-            for (int c16 = 0; c16 < 16; ++c16) {
-                uint4 val = make_uint4(pk[c16 * 4], pk[c16 * 4 + 1], pk[c16 * 4 + 2], pk[c16 * 4 + 3]);
-                *reinterpret_cast<uint4*>(p_smem + (c16 >> 3) * L::kSlab + swz128_offset(row, c16 & 7)) = val;
-            }
-            fence_proxy_async_smem();
+            tmem_st_x32(tmem_base + lane_addr + s * 128, pk);
+            tmem_st_x32(tmem_base + lane_addr + s * 128 + 32, pk + 32);
+            tmem_st_wait();
             tc_fence_before_sync();
             mbar_arrive(p_full);
         }
