@@ -10,6 +10,13 @@
 //
 // Both read K_nope / V from the recomputed bf16 up-projection KV[S, h*256] and the shared rope band
 // from k_pe[S, 64]; both keep every accumulator in TMEM and never materialise S x S.
+//
+// Roles (320 threads): warp 0 TMA producer (3 stages), warp 1 MMA issuer, warps 2..5 and 6..9 two
+// consumer warpgroups that take alternate tiles, so one warpgroup's exponentials and dS arithmetic
+// overlap the other's MMAs.  P^T / dS^T (dkv) and dS (dq) never touch shared memory: the consumers
+// write them back to TMEM as packed bf16 and the accumulating MMAs read their A operand from there.
+// A tile's scratch columns are reused two tiles later by an MMA that the same thread issues after the
+// MMAs that read them; the tensor pipe runs one thread's MMAs in order, so that reuse needs no barrier.
 #pragma once
 #include "attn_fwd_sm100.cuh"
 #include "sm100_ptx.cuh"
@@ -74,6 +81,9 @@ bwd_dkpe_reduce_kernel(const float* __restrict__ dk_rope, int S, int h, __nv_bfl
     dk_pe[idx] = __float2bfloat16_rn(acc);
 }
 
+constexpr int kBwdThreads = 320;
+constexpr int kBwdStages = 3;
+
 // ================================================================================================
 // dK / dV kernel
 // ================================================================================================
@@ -90,19 +100,17 @@ struct AttnBwdDkvArgs {
 struct AttnBwdDkvSmem {
     static constexpr int kSlab128 = 128 * 128;                 // 128 rows x 128 B
     static constexpr int kSlab64 = 64 * 128;                   // 64 rows x 128 B
+    static constexpr int kStage = 5 * kSlab64;                 // Q (3 slabs) + dO (2 slabs), 64 rows each
     static constexpr int kK = 0;                               // 3 slabs of 128 rows
     static constexpr int kV = kK + 3 * kSlab128;               // 2 slabs of 128 rows
-    static constexpr int kQ = kV + 2 * kSlab128;               // 2 stages x 3 slabs of 64 rows
-    static constexpr int kDO = kQ + 2 * 3 * kSlab64;           // 2 stages x 2 slabs of 64 rows
-    static constexpr int kPt = kDO + 2 * 2 * kSlab64;          // P^T  [128 keys x 64 q]
-    static constexpr int kDSt = kPt + kSlab128;                // dS^T [128 keys x 64 q]
-    static constexpr int kStat = kDSt + kSlab128;              // 2 stages x (64 l2 + 64 delta) floats
-    static constexpr int kBar = kStat + 2 * 512;
+    static constexpr int kQdO = kV + 2 * kSlab128;             // kBwdStages stages
+    static constexpr int kStat = kQdO + kBwdStages * kStage;   // per stage: 64 l2 + 64 delta floats
+    static constexpr int kBar = kStat + kBwdStages * 512;
     static constexpr int kTotalBytes = kBar + 256 + 1024;
 };
 
 template <bool kCausal>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_do,
                           const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
                           const AttnBwdDkvArgs args) {
@@ -111,16 +119,15 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
     uint64_t* kv_full = bars + 0;
-    uint64_t* qdo_full = bars + 1;    // [2]
-    uint64_t* qdo_empty = bars + 3;   // [2]
-    uint64_t* st_full = bars + 5;     // [2]
-    uint64_t* st_free = bars + 7;     // [2]
-    uint64_t* dp_full = bars + 9;
-    uint64_t* dp_free = bars + 10;
-    uint64_t* pds_full = bars + 11;
-    uint64_t* pds_free = bars + 12;
-    uint64_t* acc_done = bars + 13;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+    uint64_t* qdo_full = bars + 1;    // [3]
+    uint64_t* qdo_empty = bars + 4;   // [3]
+    uint64_t* st_full = bars + 7;     // [2]  S^T of the group's tile is in TMEM
+    uint64_t* st_read = bars + 9;     // [2]  the group has loaded it: the columns may take dP^T
+    uint64_t* p_full = bars + 11;     // [2]  P^T (bf16) is in TMEM
+    uint64_t* dp_full = bars + 13;    // [2]  dP^T is in TMEM
+    uint64_t* ds_full = bars + 15;    // [2]  dS^T (bf16) is in TMEM
+    uint64_t* acc_done = bars + 17;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -132,12 +139,11 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&qdo_full[s], 1); mbar_init(&qdo_empty[s], 1);
-            mbar_init(&st_full[s], 1); mbar_init(&st_free[s], 128);
+        for (int s = 0; s < kBwdStages; ++s) { mbar_init(&qdo_full[s], 1); mbar_init(&qdo_empty[s], 1); }
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(&st_full[g], 1); mbar_init(&st_read[g], 128); mbar_init(&p_full[g], 128);
+            mbar_init(&dp_full[g], 1); mbar_init(&ds_full[g], 128);
         }
-        mbar_init(dp_full, 1); mbar_init(dp_free, 128);
-        mbar_init(pds_full, 128); mbar_init(pds_free, 1);
         mbar_init(acc_done, 1);
         abort_flag->value = 0;
         mbar_fence_init();
@@ -149,10 +155,11 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_st = tmem_base;            // 2 x 64 columns
-    const uint32_t tmem_dp = tmem_base + 128;      // 64 columns
-    const uint32_t tmem_dk = tmem_base + 192;      // 192 columns
-    const uint32_t tmem_dv = tmem_base + 384;      // 128 columns
+    // columns: [0,64) group 0 scratch (S^T, then dP^T, then dS^T bf16) | [64,128) group 1 scratch |
+    //          [128,160) P^T group 0 | [160,192) P^T group 1 | [192,384) dK | [384,512) dV
+    const uint32_t tmem_pt = tmem_base + 128;
+    const uint32_t tmem_dk = tmem_base + 192;
+    const uint32_t tmem_dv = tmem_base + 384;
 
     if (warp == 0) {
         if (elect_one()) {
@@ -163,98 +170,109 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             tma_load_2d(smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, t0);
             tma_load_2d(smem + L::kV + L::kSlab128, &tmap_kv, kv_full, head * 256 + 192, t0);
             for (int j = 0; j < n_iter; ++j) {
-                const int s = j & 1;
-                if (!mbar_wait(&qdo_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, args.status, 0x40)) break;
+                const int st = j % kBwdStages;
+                if (!mbar_wait(&qdo_empty[st], ((j / kBwdStages) & 1) ^ 1, abort_flag, args.status, 0x40)) break;
                 const int q0 = (j_begin + j) * 64;
-                mbar_arrive_expect_tx(&qdo_full[s], 5 * L::kSlab64 + 512);
-                uint8_t* sq = smem + L::kQ + s * 3 * L::kSlab64;
-                uint8_t* sdo = smem + L::kDO + s * 2 * L::kSlab64;
+                mbar_arrive_expect_tx(&qdo_full[st], L::kStage + 512);
+                uint8_t* sq = smem + L::kQdO + st * L::kStage;
+                uint8_t* sdo = sq + 3 * L::kSlab64;
                 for (int c = 0; c < 3; ++c)
-                    tma_load_2d(sq + c * L::kSlab64, &tmap_q, &qdo_full[s], head * 192 + c * 64, q0);
+                    tma_load_2d(sq + c * L::kSlab64, &tmap_q, &qdo_full[st], head * 192 + c * 64, q0);
                 for (int c = 0; c < 2; ++c)
-                    tma_load_2d(sdo + c * L::kSlab64, &tmap_do, &qdo_full[s], head * 128 + c * 64, q0);
-                float* stat = reinterpret_cast<float*>(smem + L::kStat + s * 512);
-                bulk_load_1d(stat, args.stat_l2 + static_cast<size_t>(head) * args.S_pad + q0, 256, &qdo_full[s]);
+                    tma_load_2d(sdo + c * L::kSlab64, &tmap_do, &qdo_full[st], head * 128 + c * 64, q0);
+                float* stat = reinterpret_cast<float*>(smem + L::kStat + st * 512);
+                bulk_load_1d(stat, args.stat_l2 + static_cast<size_t>(head) * args.S_pad + q0, 256, &qdo_full[st]);
                 bulk_load_1d(stat + 64, args.stat_delta + static_cast<size_t>(head) * args.S_pad + q0, 256,
-                             &qdo_full[s]);
+                             &qdo_full[st]);
             }
         }
     } else if (warp == 1) {
         if (elect_one()) {
             constexpr uint32_t idesc_st = make_idesc_bf16(128, 64, 0, 0);    // S^T, dP^T: both K-major
-            constexpr uint32_t idesc_dv = make_idesc_bf16(128, 128, 0, 1);   // dV: A = P^T K-major, B = dO MN-major
-            constexpr uint32_t idesc_dk = make_idesc_bf16(128, 192, 0, 1);   // dK: A = dS^T,     B = Q  MN-major
+            constexpr uint32_t idesc_dv = make_idesc_bf16(128, 128, 0, 1);   // dV: A = P^T (TMEM), B = dO MN-major
+            constexpr uint32_t idesc_dk = make_idesc_bf16(128, 192, 0, 1);   // dK: A = dS^T (TMEM), B = Q MN-major
             const uint32_t sk = smem_u32(smem + L::kK), sv = smem_u32(smem + L::kV);
-            const uint32_t spt = smem_u32(smem + L::kPt), sdst = smem_u32(smem + L::kDSt);
-            auto issue_acc = [&](int j) -> bool {   // dV += P^T dO_j, dK += dS^T Q_j
-                if (!mbar_wait(pds_full, j & 1, abort_flag, args.status, 0x50)) return false;
+            auto stage_q = [&](int j) { return smem_u32(smem + L::kQdO + (j % kBwdStages) * L::kStage); };
+            auto issue_st = [&](int j) -> bool {     // S^T(j) = K Q_j^T into the group's scratch columns
+                const int g = j & 1;
+                if (!mbar_wait(&qdo_full[j % kBwdStages], (j / kBwdStages) & 1, abort_flag, args.status, 0x52))
+                    return false;
                 tc_fence_after_sync();
-                const int s = j & 1;
-                const uint32_t sq = smem_u32(smem + L::kQ + s * 3 * L::kSlab64);
-                const uint32_t sdo = smem_u32(smem + L::kDO + s * 2 * L::kSlab64);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ss(tmem_dv, desc_k_major(spt + kk * 32), desc_mn_major(sdo + kk * 2048, L::kSlab64), idesc_dv,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ss(tmem_dk, desc_k_major(sdst + kk * 32), desc_mn_major(sq + kk * 2048, L::kSlab64), idesc_dk,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-                mma_commit(&qdo_empty[s]);
-                mma_commit(pds_free);
-                return true;
-            };
-            bool ok = mbar_wait(kv_full, 0, abort_flag, args.status, 0x51);
-            for (int j = 0; j < n_iter && ok; ++j) {
-                const int s = j & 1;
-                const uint32_t ph = (j >> 1) & 1;
-                ok = mbar_wait(&qdo_full[s], ph, abort_flag, args.status, 0x52) &&
-                     mbar_wait(&st_free[s], ph ^ 1, abort_flag, args.status, 0x53);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t sq = smem_u32(smem + L::kQ + s * 3 * L::kSlab64);
-                const uint32_t sdo = smem_u32(smem + L::kDO + s * 2 * L::kSlab64);
+                const uint32_t sq = stage_q(j);
 #pragma unroll
                 for (int kk = 0; kk < 12; ++kk)
-                    mma_ss(tmem_st + s * 64, desc_k_major(sk + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
+                    mma_ss(tmem_base + g * 64, desc_k_major(sk + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
                            desc_k_major(sq + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_st, kk > 0 ? 1u : 0u);
-                mma_commit(&st_full[s]);
-                ok = mbar_wait(dp_free, (j & 1) ^ 1, abort_flag, args.status, 0x54);
-                if (!ok) break;
+                mma_commit(&st_full[g]);
+                return true;
+            };
+            auto issue_dp = [&](int j) -> bool {     // dP^T(j) = V dO_j^T over the same columns once S^T was read
+                const int g = j & 1;
+                if (!mbar_wait(&st_read[g], (j >> 1) & 1, abort_flag, args.status, 0x53)) return false;
                 tc_fence_after_sync();
+                const uint32_t sdo = stage_q(j) + 3 * L::kSlab64;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    mma_ss(tmem_dp, desc_k_major(sv + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
+                    mma_ss(tmem_base + g * 64, desc_k_major(sv + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
                            desc_k_major(sdo + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_st, kk > 0 ? 1u : 0u);
-                mma_commit(dp_full);
-                if (j > 0) ok = issue_acc(j - 1);
+                mma_commit(&dp_full[g]);
+                return true;
+            };
+            auto issue_acc = [&](int j) -> bool {    // dV += P^T dO_j, dK += dS^T Q_j (A operands from TMEM)
+                const int g = j & 1;
+                const uint32_t ph = (j >> 1) & 1;
+                if (!mbar_wait(&p_full[g], ph, abort_flag, args.status, 0x50)) return false;
+                if (!mbar_wait(&ds_full[g], ph, abort_flag, args.status, 0x51)) return false;
+                tc_fence_after_sync();
+                const uint32_t sq = stage_q(j);
+                const uint32_t sdo = sq + 3 * L::kSlab64;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts(tmem_dv, tmem_pt + g * 32 + kk * 8, desc_mn_major(sdo + kk * 2048, L::kSlab64), idesc_dv,
+                           (j > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts(tmem_dk, tmem_base + g * 64 + kk * 8, desc_mn_major(sq + kk * 2048, L::kSlab64), idesc_dk,
+                           (j > 0 || kk > 0) ? 1u : 0u);
+                mma_commit(&qdo_empty[j % kBwdStages]);
+                return true;
+            };
+            bool ok = mbar_wait(kv_full, 0, abort_flag, args.status, 0x54);
+            if (ok) ok = issue_st(0);
+            for (int j = 0; j < n_iter && ok; ++j) {
+                ok = issue_dp(j);
+                if (ok && j > 0) ok = issue_acc(j - 1);
+                if (ok && j + 1 < n_iter) ok = issue_st(j + 1);
             }
             if (ok) ok = issue_acc(n_iter - 1);
             if (ok) mma_commit(acc_done);
         }
     } else {
+        const int g = (warp - 2) >> 2;               // consumer warpgroup 0 or 1
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;         // key row inside the tile == TMEM lane
         const int t_idx = t0 + row;
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+        const uint32_t tmem_scr = tmem_base + g * 64 + lane_addr;
         bool ok = true;
-        for (int j = 0; j < n_iter; ++j) {
-            const int s = j & 1;
+        for (int j = g; j < n_iter; j += 2) {
+            const uint32_t ph = (j >> 1) & 1;
+            const int st = j % kBwdStages;
             const int q0 = (j_begin + j) * 64;
-            ok = mbar_wait_warp(&st_full[s], (j >> 1) & 1, abort_flag, args.status, 0x60);
+            ok = mbar_wait_warp(&st_full[g], ph, abort_flag, args.status, 0x60);
             if (!ok) break;
             tc_fence_after_sync();
             uint32_t sv[64];
-            tmem_ld_x32(tmem_st + lane_addr + s * 64, sv);
-            tmem_ld_x32(tmem_st + lane_addr + s * 64 + 32, sv + 32);
+            tmem_ld_x32(tmem_scr, sv);
+            tmem_ld_x32(tmem_scr + 32, sv + 32);
             tmem_ld_wait();
             tc_fence_before_sync();
-            mbar_arrive(&st_free[s]);
-            // stat tile was delivered with Q/dO on qdo_full[s], which the MMA warp waited for before
-            // S^T could complete; this wait makes those bulk-copy writes visible to this thread too.
-            ok = mbar_wait_warp(&qdo_full[s], (j >> 1) & 1, abort_flag, args.status, 0x61);
+            mbar_arrive(&st_read[g]);
+            // The statistics arrived with Q/dO on qdo_full[st]; waiting on it here makes those
+            // bulk-copy writes visible to this thread as well.
+            ok = mbar_wait_warp(&qdo_full[st], (j / kBwdStages) & 1, abort_flag, args.status, 0x61);
             if (!ok) break;
-            const float* stat = reinterpret_cast<const float*>(smem + L::kStat + s * 512);
+            const float* stat = reinterpret_cast<const float*>(smem + L::kStat + st * 512);
             const bool diag = kCausal && (q0 < t0 + 128);
             float p[64];
 #pragma unroll
@@ -269,45 +287,36 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     p[c] = v;
                 }
             }
-            if (j > 0) {
-                ok = mbar_wait_warp(pds_free, (j - 1) & 1, abort_flag, args.status, 0x62);
-                if (!ok) break;
-            }
+            uint32_t pk[32];
 #pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-                uint4 val;
-                val.x = pack_bf16x2(p[c16 * 8 + 0], p[c16 * 8 + 1]);
-                val.y = pack_bf16x2(p[c16 * 8 + 2], p[c16 * 8 + 3]);
-                val.z = pack_bf16x2(p[c16 * 8 + 4], p[c16 * 8 + 5]);
-                val.w = pack_bf16x2(p[c16 * 8 + 6], p[c16 * 8 + 7]);
-                *reinterpret_cast<uint4*>(smem + L::kPt + swz128_offset(row, c16)) = val;
-            }
-            ok = mbar_wait_warp(dp_full, j & 1, abort_flag, args.status, 0x63);
+            for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
+            tmem_st_x32(tmem_pt + g * 32 + lane_addr, pk);
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(&p_full[g]);
+
+            ok = mbar_wait_warp(&dp_full[g], ph, abort_flag, args.status, 0x63);
             if (!ok) break;
             tc_fence_after_sync();
-            tmem_ld_x32(tmem_dp + lane_addr, sv);
-            tmem_ld_x32(tmem_dp + lane_addr + 32, sv + 32);
+            tmem_ld_x32(tmem_scr, sv);
+            tmem_ld_x32(tmem_scr + 32, sv + 32);
             tmem_ld_wait();
-            tc_fence_before_sync();
-            mbar_arrive(dp_free);
 #pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-                const float4 d0 = *reinterpret_cast<const float4*>(stat + 64 + c16 * 8);
-                const float4 d1 = *reinterpret_cast<const float4*>(stat + 64 + c16 * 8 + 4);
+            for (int c8 = 0; c8 < 8; ++c8) {
+                const float4 d0 = *reinterpret_cast<const float4*>(stat + 64 + c8 * 8);
+                const float4 d1 = *reinterpret_cast<const float4*>(stat + 64 + c8 * 8 + 4);
                 const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-                float ds[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    ds[e] = p[c16 * 8 + e] * (__uint_as_float(sv[c16 * 8 + e]) - dl[e]);
-                uint4 val;
-                val.x = pack_bf16x2(ds[0], ds[1]);
-                val.y = pack_bf16x2(ds[2], ds[3]);
-                val.z = pack_bf16x2(ds[4], ds[5]);
-                val.w = pack_bf16x2(ds[6], ds[7]);
-                *reinterpret_cast<uint4*>(smem + L::kDSt + swz128_offset(row, c16)) = val;
+                for (int e = 0; e < 4; ++e) {
+                    const int c = c8 * 8 + 2 * e;
+                    pk[c8 * 4 + e] = pack_bf16x2(p[c] * (__uint_as_float(sv[c]) - dl[2 * e]),
+                                                 p[c + 1] * (__uint_as_float(sv[c + 1]) - dl[2 * e + 1]));
+                }
             }
-            fence_proxy_async_smem();
-            mbar_arrive(pds_full);
+            tmem_st_x32(tmem_scr, pk);               // dS^T over the first 32 of the columns dP^T occupied
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(&ds_full[g]);
         }
         if (ok) ok = mbar_wait_warp(acc_done, 0, abort_flag, args.status, 0x64);
         if (ok) {
@@ -315,11 +324,13 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             const bool valid = t_idx < args.S;
             __nv_bfloat16* dkv_row = args.dkv + static_cast<size_t>(t_idx) * args.h * 256 + head * 256;
             float* dkr_row = args.dk_rope + (static_cast<size_t>(head) * args.S + t_idx) * 64;
+            // 10 chunks of 32 columns: dK nope (0..3), dK rope (4..5), dV (6..9; dV follows dK in TMEM).
+            // Group 0 drains chunks 0..4, group 1 chunks 5..9.
 #pragma unroll 1
-            for (int c = 0; c < 10; ++c) {            // 6 chunks of dK (4 nope + 2 rope), 4 chunks of dV
+            for (int c = g * 5; c < g * 5 + 5; ++c) {
                 uint32_t r[32];
                 __syncwarp();
-                tmem_ld_x32(tmem_dk + lane_addr + c * 32, r);   // dV follows dK in TMEM
+                tmem_ld_x32(tmem_dk + lane_addr + c * 32, r);
                 tmem_ld_wait();
                 if (!valid) continue;
                 if (c == 4 || c == 5) {
@@ -366,17 +377,16 @@ struct AttnBwdDqArgs {
 struct AttnBwdDqSmem {
     static constexpr int kSlab128 = 128 * 128;
     static constexpr int kSlab64 = 64 * 128;
+    static constexpr int kStage = 5 * kSlab64;                 // K (3 slabs) + V (2 slabs), 64 keys each
     static constexpr int kQ = 0;                               // 3 slabs of 128 rows
     static constexpr int kDO = kQ + 3 * kSlab128;              // 2 slabs of 128 rows
-    static constexpr int kK = kDO + 2 * kSlab128;              // 2 stages x 3 slabs of 64 rows
-    static constexpr int kV = kK + 2 * 3 * kSlab64;            // 2 stages x 2 slabs of 64 rows
-    static constexpr int kDS = kV + 2 * 2 * kSlab64;           // dS [128 q x 64 keys]
-    static constexpr int kBar = kDS + kSlab128;
+    static constexpr int kKV = kDO + 2 * kSlab128;             // kBwdStages stages
+    static constexpr int kBar = kKV + kBwdStages * kStage;
     static constexpr int kTotalBytes = kBar + 256 + 1024;
 };
 
 template <bool kCausal>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_do,
                          const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
                          const AttnBwdDqArgs args) {
@@ -385,12 +395,10 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
     uint64_t* qdo_full = bars + 0;
-    uint64_t* kv_full = bars + 1;     // [2]
-    uint64_t* kv_empty = bars + 3;    // [2]
-    uint64_t* sdp_full = bars + 5;    // [2]
-    uint64_t* sdp_free = bars + 7;    // [2]
-    uint64_t* ds_full = bars + 9;
-    uint64_t* ds_free = bars + 10;
+    uint64_t* kv_full = bars + 1;     // [3]
+    uint64_t* kv_empty = bars + 4;    // [3]
+    uint64_t* sdp_full = bars + 7;    // [2]  S and dP of the group's tile are in TMEM
+    uint64_t* ds_full = bars + 9;     // [2]  dS (bf16) is in TMEM
     uint64_t* acc_done = bars + 11;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
@@ -405,11 +413,8 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
 
     if (threadIdx.x == 0) {
         mbar_init(qdo_full, 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1);
-            mbar_init(&sdp_full[s], 1); mbar_init(&sdp_free[s], 128);
-        }
-        mbar_init(ds_full, 128); mbar_init(ds_free, 1);
+        for (int s = 0; s < kBwdStages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        for (int g = 0; g < 2; ++g) { mbar_init(&sdp_full[g], 1); mbar_init(&ds_full[g], 128); }
         mbar_init(acc_done, 1);
         abort_flag->value = 0;
         mbar_fence_init();
@@ -421,9 +426,9 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_s = tmem_base;             // 2 x 64 columns
-    const uint32_t tmem_dp = tmem_base + 128;      // 2 x 64 columns
-    const uint32_t tmem_dq = tmem_base + 256;      // 192 columns
+    // columns: group g scratch at [128g, 128g+128): S in the first 64, dP in the last 64, then dS (bf16)
+    //          over the first 32 | [256,448) dQ
+    const uint32_t tmem_dq = tmem_base + 256;
 
     if (warp == 0) {
         if (elect_one()) {
@@ -433,84 +438,82 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             for (int c = 0; c < 2; ++c)
                 tma_load_2d(smem + L::kDO + c * L::kSlab128, &tmap_do, qdo_full, head * 128 + c * 64, q0);
             for (int j = 0; j < n_iter; ++j) {
-                const int s = j & 1;
-                if (!mbar_wait(&kv_empty[s], ((j >> 1) & 1) ^ 1, abort_flag, args.status, 0x70)) break;
-                mbar_arrive_expect_tx(&kv_full[s], 5 * L::kSlab64);
-                uint8_t* sk = smem + L::kK + s * 3 * L::kSlab64;
-                uint8_t* sv = smem + L::kV + s * 2 * L::kSlab64;
-                tma_load_2d(sk, &tmap_kv, &kv_full[s], head * 256, j * 64);
-                tma_load_2d(sk + L::kSlab64, &tmap_kv, &kv_full[s], head * 256 + 64, j * 64);
-                tma_load_2d(sk + 2 * L::kSlab64, &tmap_kpe, &kv_full[s], 0, j * 64);
-                tma_load_2d(sv, &tmap_kv, &kv_full[s], head * 256 + 128, j * 64);
-                tma_load_2d(sv + L::kSlab64, &tmap_kv, &kv_full[s], head * 256 + 192, j * 64);
+                const int st = j % kBwdStages;
+                if (!mbar_wait(&kv_empty[st], ((j / kBwdStages) & 1) ^ 1, abort_flag, args.status, 0x70)) break;
+                mbar_arrive_expect_tx(&kv_full[st], L::kStage);
+                uint8_t* sk = smem + L::kKV + st * L::kStage;
+                uint8_t* sv = sk + 3 * L::kSlab64;
+                tma_load_2d(sk, &tmap_kv, &kv_full[st], head * 256, j * 64);
+                tma_load_2d(sk + L::kSlab64, &tmap_kv, &kv_full[st], head * 256 + 64, j * 64);
+                tma_load_2d(sk + 2 * L::kSlab64, &tmap_kpe, &kv_full[st], 0, j * 64);
+                tma_load_2d(sv, &tmap_kv, &kv_full[st], head * 256 + 128, j * 64);
+                tma_load_2d(sv + L::kSlab64, &tmap_kv, &kv_full[st], head * 256 + 192, j * 64);
             }
         }
     } else if (warp == 1) {
         if (elect_one()) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);     // S, dP: both K-major
-            constexpr uint32_t idesc_dq = make_idesc_bf16(128, 192, 0, 1);   // dQ: A = dS K-major, B = K MN-major
+            constexpr uint32_t idesc_dq = make_idesc_bf16(128, 192, 0, 1);   // dQ: A = dS (TMEM), B = K MN-major
             const uint32_t sq = smem_u32(smem + L::kQ), sdo = smem_u32(smem + L::kDO);
-            const uint32_t sds = smem_u32(smem + L::kDS);
-            auto issue_dq = [&](int j) -> bool {
-                if (!mbar_wait(ds_full, j & 1, abort_flag, args.status, 0x80)) return false;
+            auto stage_k = [&](int j) { return smem_u32(smem + L::kKV + (j % kBwdStages) * L::kStage); };
+            auto issue_sdp = [&](int j) -> bool {
+                const int g = j & 1;
+                if (!mbar_wait(&kv_full[j % kBwdStages], (j / kBwdStages) & 1, abort_flag, args.status, 0x82))
+                    return false;
                 tc_fence_after_sync();
-                const int s = j & 1;
-                const uint32_t sk = smem_u32(smem + L::kK + s * 3 * L::kSlab64);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ss(tmem_dq, desc_k_major(sds + kk * 32), desc_mn_major(sk + kk * 2048, L::kSlab64), idesc_dq,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-                mma_commit(&kv_empty[s]);
-                mma_commit(ds_free);
-                return true;
-            };
-            bool ok = mbar_wait(qdo_full, 0, abort_flag, args.status, 0x81);
-            for (int j = 0; j < n_iter && ok; ++j) {
-                const int s = j & 1;
-                const uint32_t ph = (j >> 1) & 1;
-                ok = mbar_wait(&kv_full[s], ph, abort_flag, args.status, 0x82) &&
-                     mbar_wait(&sdp_free[s], ph ^ 1, abort_flag, args.status, 0x83);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t sk = smem_u32(smem + L::kK + s * 3 * L::kSlab64);
-                const uint32_t sv = smem_u32(smem + L::kV + s * 2 * L::kSlab64);
+                const uint32_t sk = stage_k(j);
+                const uint32_t sv = sk + 3 * L::kSlab64;
 #pragma unroll
                 for (int kk = 0; kk < 12; ++kk)
-                    mma_ss(tmem_s + s * 64, desc_k_major(sq + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
+                    mma_ss(tmem_base + g * 128, desc_k_major(sq + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
                            desc_k_major(sk + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    mma_ss(tmem_dp + s * 64, desc_k_major(sdo + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
+                    mma_ss(tmem_base + g * 128 + 64, desc_k_major(sdo + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
                            desc_k_major(sv + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
-                mma_commit(&sdp_full[s]);
-                if (j > 0) ok = issue_dq(j - 1);
+                mma_commit(&sdp_full[g]);
+                return true;
+            };
+            bool ok = mbar_wait(qdo_full, 0, abort_flag, args.status, 0x81);
+            if (ok) ok = issue_sdp(0);
+            if (ok && n_iter > 1) ok = issue_sdp(1);
+            for (int j = 0; j < n_iter && ok; ++j) {
+                const int g = j & 1;
+                ok = mbar_wait(&ds_full[g], (j >> 1) & 1, abort_flag, args.status, 0x80);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t sk = stage_k(j);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts(tmem_dq, tmem_base + g * 128 + kk * 8, desc_mn_major(sk + kk * 2048, L::kSlab64), idesc_dq,
+                           (j > 0 || kk > 0) ? 1u : 0u);
+                mma_commit(&kv_empty[j % kBwdStages]);
+                if (j + 2 < n_iter) ok = issue_sdp(j + 2);
             }
-            if (ok) ok = issue_dq(n_iter - 1);
             if (ok) mma_commit(acc_done);
         }
     } else {
+        const int g = (warp - 2) >> 2;
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const int s_idx = q0 + row;
         const bool valid = s_idx < args.S;
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+        const uint32_t tmem_scr = tmem_base + g * 128 + lane_addr;
         // Rows past the end of the sequence get LSE = +inf so that their P is exactly zero.
         const float l2 = valid ? args.lse[static_cast<size_t>(s_idx) * args.h + head] * 1.4426950408889634f : INFINITY;
         const float delta = valid ? args.stat_delta[static_cast<size_t>(head) * args.S_pad + s_idx] : 0.f;
         bool ok = true;
-        for (int j = 0; j < n_iter; ++j) {
-            const int s = j & 1;
-            ok = mbar_wait_warp(&sdp_full[s], (j >> 1) & 1, abort_flag, args.status, 0x90);
+        for (int j = g; j < n_iter; j += 2) {
+            ok = mbar_wait_warp(&sdp_full[g], (j >> 1) & 1, abort_flag, args.status, 0x90);
             if (!ok) break;
             tc_fence_after_sync();
             uint32_t sv[64], dpv[64];
-            tmem_ld_x32(tmem_s + lane_addr + s * 64, sv);
-            tmem_ld_x32(tmem_s + lane_addr + s * 64 + 32, sv + 32);
-            tmem_ld_x32(tmem_dp + lane_addr + s * 64, dpv);
-            tmem_ld_x32(tmem_dp + lane_addr + s * 64 + 32, dpv + 32);
+            tmem_ld_x32(tmem_scr, sv);
+            tmem_ld_x32(tmem_scr + 32, sv + 32);
+            tmem_ld_x32(tmem_scr + 64, dpv);
+            tmem_ld_x32(tmem_scr + 96, dpv + 32);
             tmem_ld_wait();
-            tc_fence_before_sync();
-            mbar_arrive(&sdp_free[s]);
             const int tk0 = j * 64;
             const bool edge = (kCausal && tk0 + 63 > q0) || (tk0 + 64 > args.S);
             uint32_t pk[32];
@@ -529,24 +532,17 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 }
                 pk[c] = pack_bf16x2(d[0], d[1]);
             }
-            if (j > 0) {
-                ok = mbar_wait_warp(ds_free, (j - 1) & 1, abort_flag, args.status, 0x91);
-                if (!ok) break;
-            }
-#pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-                uint4 val = make_uint4(pk[c16 * 4], pk[c16 * 4 + 1], pk[c16 * 4 + 2], pk[c16 * 4 + 3]);
-                *reinterpret_cast<uint4*>(smem + L::kDS + swz128_offset(row, c16)) = val;
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(ds_full);
+            tmem_st_x32(tmem_scr, pk);
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(&ds_full[g]);
         }
         if (ok) ok = mbar_wait_warp(acc_done, 0, abort_flag, args.status, 0x92);
         if (ok) {
             tc_fence_after_sync();
             __nv_bfloat16* dst = args.dq + (static_cast<size_t>(s_idx) * args.h + head) * 192;
 #pragma unroll 1
-            for (int c = 0; c < 6; ++c) {
+            for (int c = g * 3; c < g * 3 + 3; ++c) {   // six 32-column chunks, three per group
                 uint32_t r[32];
                 __syncwarp();
                 tmem_ld_x32(tmem_dq + lane_addr + c * 32, r);

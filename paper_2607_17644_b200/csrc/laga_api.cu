@@ -244,17 +244,17 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         auto k2 = attn_bwd_dq_sm100_kernel<true>;
         if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
             return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
     } else {
         auto k1 = attn_bwd_dkv_sm100_kernel<false>;
         auto k2 = attn_bwd_dq_sm100_kernel<false>;
         if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
             return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, 192, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, 192, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     {
