@@ -5,18 +5,22 @@
 //                 S^T = K Q^T, dP^T = V dO^T, P^T = exp(scale S^T - LSE), dS^T = P^T (dP^T - delta),
 //                 dV += P^T dO, dK += dS^T Q  (dK 192 wide: 128 nope columns + 64 rope columns).
 //                 TMEM lanes are keys, so LSE and delta are per-column vectors staged in shared memory.
-//   attn_bwd_dq   one CTA per (128-query tile, head), sweeping 64-key tiles:
+//   attn_bwd_dq   one CTA per (128-query tile, head), sweeping 128-key tiles:
 //                 S = Q K^T, dP = dO V^T, dS = P (dP - delta), dQ += dS K.  TMEM lanes are queries.
 //
 // Both read K_nope / V from the recomputed bf16 up-projection KV[S, h*256] and the shared rope band
 // from k_pe[S, 64]; both keep every accumulator in TMEM and never materialise S x S.
 //
-// Roles (320 threads): warp 0 TMA producer (3 stages), warp 1 MMA issuer, warps 2..5 and 6..9 two
-// consumer warpgroups that take alternate tiles, so one warpgroup's exponentials and dS arithmetic
-// overlap the other's MMAs.  P^T / dS^T (dkv) and dS (dq) never touch shared memory: the consumers
-// write them back to TMEM as packed bf16 and the accumulating MMAs read their A operand from there.
-// A tile's scratch columns are reused two tiles later by an MMA that the same thread issues after the
+// Roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 and 6..9 two consumer
+// warpgroups (every thread owns one TMEM lane).  P^T / dS^T (dkv) and dS (dq) never touch shared
+// memory: the consumers write them back to TMEM as packed bf16 and the accumulating MMAs read their
+// A operand from there.  Scratch columns are reused by an MMA that the same thread issues after the
 // MMAs that read them; the tensor pipe runs one thread's MMAs in order, so that reuse needs no barrier.
+//   dkv: dK (192) + dV (128) leave 192 TMEM columns, so query tiles are 64 rows and the two groups
+//        take alternate tiles (scratch 2 x 64 columns + P^T 2 x 32): one group's exponentials overlap
+//        the other's MMAs.  A 64-wide N costs 48 cycles per MMA against 32 ideal.
+//   dq:  128-key tiles, all MMAs 128 wide; the two groups take 64 key columns each.  dO (the A
+//        operand of dP) lives in TMEM, which frees shared memory for a third K stage.
 #pragma once
 #include "attn_fwd_sm100.cuh"
 #include "sm100_ptx.cuh"
@@ -237,12 +241,14 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 mma_commit(&qdo_empty[j % kBwdStages]);
                 return true;
             };
+            // Issue order per tile: S^T(j), then the accumulations of tile j-1, then dP^T(j).  Each wait
+            // has about one MMA group of slack: the other warpgroup finishes dS^T(j-1) while S^T(j)
+            // runs, and this tile's warpgroup has loaded S^T(j) long before dP^T(j) is due.
             bool ok = mbar_wait(kv_full, 0, abort_flag, args.status, 0x54);
-            if (ok) ok = issue_st(0);
             for (int j = 0; j < n_iter && ok; ++j) {
-                ok = issue_dp(j);
+                ok = issue_st(j);
                 if (ok && j > 0) ok = issue_acc(j - 1);
-                if (ok && j + 1 < n_iter) ok = issue_st(j + 1);
+                if (ok) ok = issue_dp(j);
             }
             if (ok) ok = issue_acc(n_iter - 1);
             if (ok) mma_commit(acc_done);
@@ -361,6 +367,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
 }
 
+
 // ================================================================================================
 // dQ kernel
 // ================================================================================================
@@ -370,37 +377,45 @@ struct AttnBwdDqArgs {
     const float* lse;            // [S, h]
     const float* stat_delta;     // [h][S_pad]
     int S_pad;
+    const __nv_bfloat16* dout;   // [S, h, 128]
     __nv_bfloat16* dq;           // [S, h, 192]
     unsigned int* status;
 };
 
+constexpr int kDqKStages = 3;
+
 struct AttnBwdDqSmem {
-    static constexpr int kSlab128 = 128 * 128;
-    static constexpr int kSlab64 = 64 * 128;
-    static constexpr int kStage = 5 * kSlab64;                 // K (3 slabs) + V (2 slabs), 64 keys each
-    static constexpr int kQ = 0;                               // 3 slabs of 128 rows
-    static constexpr int kDO = kQ + 3 * kSlab128;              // 2 slabs of 128 rows
-    static constexpr int kKV = kDO + 2 * kSlab128;             // kBwdStages stages
-    static constexpr int kBar = kKV + kBwdStages * kStage;
+    static constexpr int kSlab = 128 * 128;
+    static constexpr int kQ = 0;                               // 3 slabs
+    static constexpr int kK = kQ + 3 * kSlab;                  // 3 stages x 3 slabs
+    static constexpr int kV = kK + kDqKStages * 3 * kSlab;     // 1 stage x 2 slabs
+    static constexpr int kBar = kV + 2 * kSlab;
     static constexpr int kTotalBytes = kBar + 256 + 1024;
 };
 
+// dO of the query tile is the A operand of dP = dO V^T for every key tile.  It is kept in TMEM as
+// packed bf16 (64 columns) instead of 32 KB of shared memory, which is what leaves room for a third
+// stage of K: a K tile lives from its score MMA to its dQ MMA, a whole tile period later.
 template <bool kCausal>
 __global__ void __launch_bounds__(kBwdThreads, 1)
-attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_do,
-                         const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
-                         const AttnBwdDqArgs args) {
+attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
+                         const __grid_constant__ CUtensorMap tmap_kpe, const AttnBwdDqArgs args) {
     using L = AttnBwdDqSmem;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
-    uint64_t* qdo_full = bars + 0;
-    uint64_t* kv_full = bars + 1;     // [3]
-    uint64_t* kv_empty = bars + 4;    // [3]
-    uint64_t* sdp_full = bars + 7;    // [2]  S and dP of the group's tile are in TMEM
-    uint64_t* ds_full = bars + 9;     // [2]  dS (bf16) is in TMEM
-    uint64_t* acc_done = bars + 11;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+    uint64_t* q_full = bars + 0;
+    uint64_t* k_full = bars + 1;      // [3]
+    uint64_t* k_empty = bars + 4;     // [3]
+    uint64_t* v_full = bars + 7;
+    uint64_t* v_empty = bars + 8;
+    uint64_t* do_ready = bars + 9;    // dO is in TMEM
+    uint64_t* s_full = bars + 10;     // S is in TMEM
+    uint64_t* s_read = bars + 11;     // both groups have loaded it
+    uint64_t* dp_full = bars + 12;    // dP is in TMEM
+    uint64_t* ds_full = bars + 13;    // dS (bf16) is in TMEM
+    uint64_t* acc_done = bars + 14;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -408,134 +423,174 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     const int q_tile = n_q_tiles - 1 - static_cast<int>(blockIdx.x);
     const int head = blockIdx.y;
     const int q0 = q_tile * 128;
-    const int k_end = kCausal ? min(args.S, q0 + 128) : args.S;
-    const int n_iter = (k_end + 63) / 64;
+    const int n_iter = kCausal ? q_tile + 1 : n_q_tiles;
 
     if (threadIdx.x == 0) {
-        mbar_init(qdo_full, 1);
-        for (int s = 0; s < kBwdStages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
-        for (int g = 0; g < 2; ++g) { mbar_init(&sdp_full[g], 1); mbar_init(&ds_full[g], 128); }
+        mbar_init(q_full, 1);
+        for (int s = 0; s < kDqKStages; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); }
+        mbar_init(v_full, 1); mbar_init(v_empty, 1);
+        mbar_init(do_ready, 256);
+        mbar_init(s_full, 1); mbar_init(s_read, 256); mbar_init(dp_full, 1); mbar_init(ds_full, 256);
         mbar_init(acc_done, 1);
         abort_flag->value = 0;
         mbar_fence_init();
-        tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_do);
-        tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
+        tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
     }
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    // columns: group g scratch at [128g, 128g+128): S in the first 64, dP in the last 64, then dS (bf16)
-    //          over the first 32 | [256,448) dQ
-    const uint32_t tmem_dq = tmem_base + 256;
+    // columns: [0,128) S | [128,256) dP, then dS as bf16 (keys 0..63 in [128,160), 64..127 in [192,224)) |
+    //          [256,320) dO as bf16 | [320,512) dQ
+    const uint32_t tmem_dp = tmem_base + 128;
+    const uint32_t tmem_do = tmem_base + 256;
+    const uint32_t tmem_dq = tmem_base + 320;
 
     if (warp == 0) {
         if (elect_one()) {
-            mbar_arrive_expect_tx(qdo_full, 5 * L::kSlab128);
+            mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
             for (int c = 0; c < 3; ++c)
-                tma_load_2d(smem + L::kQ + c * L::kSlab128, &tmap_q, qdo_full, head * 192 + c * 64, q0);
-            for (int c = 0; c < 2; ++c)
-                tma_load_2d(smem + L::kDO + c * L::kSlab128, &tmap_do, qdo_full, head * 128 + c * 64, q0);
-            for (int j = 0; j < n_iter; ++j) {
-                const int st = j % kBwdStages;
-                if (!mbar_wait(&kv_empty[st], ((j / kBwdStages) & 1) ^ 1, abort_flag, args.status, 0x70)) break;
-                mbar_arrive_expect_tx(&kv_full[st], L::kStage);
-                uint8_t* sk = smem + L::kKV + st * L::kStage;
-                uint8_t* sv = sk + 3 * L::kSlab64;
-                tma_load_2d(sk, &tmap_kv, &kv_full[st], head * 256, j * 64);
-                tma_load_2d(sk + L::kSlab64, &tmap_kv, &kv_full[st], head * 256 + 64, j * 64);
-                tma_load_2d(sk + 2 * L::kSlab64, &tmap_kpe, &kv_full[st], 0, j * 64);
-                tma_load_2d(sv, &tmap_kv, &kv_full[st], head * 256 + 128, j * 64);
-                tma_load_2d(sv + L::kSlab64, &tmap_kv, &kv_full[st], head * 256 + 192, j * 64);
+                tma_load_2d(smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
+            auto load_k = [&](int j) -> bool {
+                const int st = j % kDqKStages;
+                if (!mbar_wait(&k_empty[st], ((j / kDqKStages) & 1) ^ 1, abort_flag, args.status, 0x70)) return false;
+                mbar_arrive_expect_tx(&k_full[st], 3 * L::kSlab);
+                uint8_t* sk = smem + L::kK + st * 3 * L::kSlab;
+                tma_load_2d(sk, &tmap_kv, &k_full[st], head * 256, j * 128);
+                tma_load_2d(sk + L::kSlab, &tmap_kv, &k_full[st], head * 256 + 64, j * 128);
+                tma_load_2d(sk + 2 * L::kSlab, &tmap_kpe, &k_full[st], 0, j * 128);
+                return true;
+            };
+            bool ok = load_k(0);
+            for (int j = 0; j < n_iter && ok; ++j) {
+                if (j + 1 < n_iter) ok = load_k(j + 1);
+                if (!ok) break;
+                ok = mbar_wait(v_empty, (j & 1) ^ 1, abort_flag, args.status, 0x71);
+                if (!ok) break;
+                mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
+                tma_load_2d(smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
+                tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
             }
         }
     } else if (warp == 1) {
         if (elect_one()) {
-            constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);     // S, dP: both K-major
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);    // S: both K-major; dP: A from TMEM
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, 192, 0, 1);   // dQ: A = dS (TMEM), B = K MN-major
-            const uint32_t sq = smem_u32(smem + L::kQ), sdo = smem_u32(smem + L::kDO);
-            auto stage_k = [&](int j) { return smem_u32(smem + L::kKV + (j % kBwdStages) * L::kStage); };
-            auto issue_sdp = [&](int j) -> bool {
-                const int g = j & 1;
-                if (!mbar_wait(&kv_full[j % kBwdStages], (j / kBwdStages) & 1, abort_flag, args.status, 0x82))
-                    return false;
+            const uint32_t sq = smem_u32(smem + L::kQ);
+            const uint32_t sv = smem_u32(smem + L::kV);
+            auto stage_k = [&](int j) { return smem_u32(smem + L::kK + (j % kDqKStages) * 3 * L::kSlab); };
+            auto issue_s = [&](int j) -> bool {      // S(j) = Q K_j^T
+                if (!mbar_wait(&k_full[j % kDqKStages], (j / kDqKStages) & 1, abort_flag, args.status, 0x82)) return false;
+                if (j > 0 && !mbar_wait(s_read, (j - 1) & 1, abort_flag, args.status, 0x83)) return false;
                 tc_fence_after_sync();
                 const uint32_t sk = stage_k(j);
-                const uint32_t sv = sk + 3 * L::kSlab64;
 #pragma unroll
-                for (int kk = 0; kk < 12; ++kk)
-                    mma_ss(tmem_base + g * 128, desc_k_major(sq + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
-                           desc_k_major(sk + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    mma_ss(tmem_base + g * 128 + 64, desc_k_major(sdo + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
-                           desc_k_major(sv + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
-                mma_commit(&sdp_full[g]);
+                for (int kk = 0; kk < 12; ++kk) {
+                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
+                    mma_ss(tmem_base, desc_k_major(sq + off), desc_k_major(sk + off), idesc_s, kk > 0 ? 1u : 0u);
+                }
+                mma_commit(s_full);
                 return true;
             };
-            bool ok = mbar_wait(qdo_full, 0, abort_flag, args.status, 0x81);
-            if (ok) ok = issue_sdp(0);
-            if (ok && n_iter > 1) ok = issue_sdp(1);
+            auto issue_dp = [&](int j) -> bool {     // dP(j) = dO V_j^T; overwrites dS(j-1), whose reader was issued earlier
+                if (!mbar_wait(v_full, j & 1, abort_flag, args.status, 0x84)) return false;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    mma_ts(tmem_dp, tmem_do + kk * 8, desc_k_major(sv + (kk >> 2) * L::kSlab + (kk & 3) * 32), idesc_s,
+                           kk > 0 ? 1u : 0u);
+                mma_commit(v_empty);
+                mma_commit(dp_full);
+                return true;
+            };
+            bool ok = mbar_wait(q_full, 0, abort_flag, args.status, 0x81) &&
+                      mbar_wait(do_ready, 0, abort_flag, args.status, 0x85);
+            if (ok) ok = issue_s(0);
+            if (ok) ok = issue_dp(0);
             for (int j = 0; j < n_iter && ok; ++j) {
-                const int g = j & 1;
-                ok = mbar_wait(&ds_full[g], (j >> 1) & 1, abort_flag, args.status, 0x80);
+                if (j + 1 < n_iter) ok = issue_s(j + 1);
+                if (!ok) break;
+                ok = mbar_wait(ds_full, j & 1, abort_flag, args.status, 0x80);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t sk = stage_k(j);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ts(tmem_dq, tmem_base + g * 128 + kk * 8, desc_mn_major(sk + kk * 2048, L::kSlab64), idesc_dq,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-                mma_commit(&kv_empty[j % kBwdStages]);
-                if (j + 2 < n_iter) ok = issue_sdp(j + 2);
+                for (int kk = 0; kk < 8; ++kk)
+                    mma_ts(tmem_dq, tmem_dp + (kk >> 2) * 64 + (kk & 3) * 8, desc_mn_major(sk + kk * 2048, L::kSlab),
+                           idesc_dq, (j > 0 || kk > 0) ? 1u : 0u);
+                mma_commit(&k_empty[j % kDqKStages]);
+                if (j + 1 < n_iter) ok = issue_dp(j + 1);
             }
             if (ok) mma_commit(acc_done);
         }
     } else {
-        const int g = (warp - 2) >> 2;
+        const int g = (warp - 2) >> 2;               // consumer group: key columns [64g, 64g+64) of the tile
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const int s_idx = q0 + row;
         const bool valid = s_idx < args.S;
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-        const uint32_t tmem_scr = tmem_base + g * 128 + lane_addr;
+        {   // this thread's dO row, channels [64g, 64g+64), as 32 packed words into TMEM
+            uint32_t w[32];
+            if (valid) {
+                const uint4* src = reinterpret_cast<const uint4*>(args.dout + (static_cast<size_t>(s_idx) * args.h + head) * 128 + g * 64);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const uint4 x = src[v];
+                    w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
+                }
+            } else {
+#pragma unroll
+                for (int v = 0; v < 32; ++v) w[v] = 0u;
+            }
+            __syncwarp();
+            tmem_st_x32(tmem_do + lane_addr + g * 32, w);
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(do_ready);
+        }
         // Rows past the end of the sequence get LSE = +inf so that their P is exactly zero.
         const float l2 = valid ? args.lse[static_cast<size_t>(s_idx) * args.h + head] * 1.4426950408889634f : INFINITY;
         const float delta = valid ? args.stat_delta[static_cast<size_t>(head) * args.S_pad + s_idx] : 0.f;
         bool ok = true;
-        for (int j = g; j < n_iter; j += 2) {
-            ok = mbar_wait_warp(&sdp_full[g], (j >> 1) & 1, abort_flag, args.status, 0x90);
+        for (int j = 0; j < n_iter; ++j) {
+            ok = mbar_wait_warp(s_full, j & 1, abort_flag, args.status, 0x90);
             if (!ok) break;
             tc_fence_after_sync();
-            uint32_t sv[64], dpv[64];
-            tmem_ld_x32(tmem_scr, sv);
-            tmem_ld_x32(tmem_scr + 32, sv + 32);
-            tmem_ld_x32(tmem_scr + 64, dpv);
-            tmem_ld_x32(tmem_scr + 96, dpv + 32);
+            uint32_t sv[64];
+            tmem_ld_x32(tmem_base + lane_addr + g * 64, sv);
+            tmem_ld_x32(tmem_base + lane_addr + g * 64 + 32, sv + 32);
             tmem_ld_wait();
-            const int tk0 = j * 64;
+            tc_fence_before_sync();
+            mbar_arrive(s_read);
+            const int tk0 = j * 128 + g * 64;
             const bool edge = (kCausal && tk0 + 63 > q0) || (tk0 + 64 > args.S);
+            float p[64];
+#pragma unroll
+            for (int c = 0; c < 64; ++c) {
+                float v = fast_exp2(fmaf(__uint_as_float(sv[c]), args.scale_log2, -l2));
+                if (edge) {
+                    const int t = tk0 + c;
+                    if ((kCausal && t > s_idx) || t >= args.S) v = 0.f;
+                }
+                p[c] = v;
+            }
+            ok = mbar_wait_warp(dp_full, j & 1, abort_flag, args.status, 0x91);
+            if (!ok) break;
+            tc_fence_after_sync();
+            tmem_ld_x32(tmem_dp + lane_addr + g * 64, sv);
+            tmem_ld_x32(tmem_dp + lane_addr + g * 64 + 32, sv + 32);
+            tmem_ld_wait();
             uint32_t pk[32];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                float d[2];
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int cc = 2 * c + e;
-                    float p = fast_exp2(fmaf(__uint_as_float(sv[cc]), args.scale_log2, -l2));
-                    if (edge) {
-                        const int t = tk0 + cc;
-                        if ((kCausal && t > s_idx) || t >= args.S) p = 0.f;
-                    }
-                    d[e] = p * (__uint_as_float(dpv[cc]) - delta);
-                }
-                pk[c] = pack_bf16x2(d[0], d[1]);
-            }
-            tmem_st_x32(tmem_scr, pk);
+            for (int c = 0; c < 32; ++c)
+                pk[c] = pack_bf16x2(p[2 * c] * (__uint_as_float(sv[2 * c]) - delta),
+                                    p[2 * c + 1] * (__uint_as_float(sv[2 * c + 1]) - delta));
+            tmem_st_x32(tmem_dp + lane_addr + g * 64, pk);   // dS over the first 32 columns of this group's own half
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(&ds_full[g]);
+            mbar_arrive(ds_full);
         }
         if (ok) ok = mbar_wait_warp(acc_done, 0, abort_flag, args.status, 0x92);
         if (ok) {

@@ -226,35 +226,33 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     }
     const uint64_t q_row = static_cast<uint64_t>(h) * 192, do_row = static_cast<uint64_t>(h) * 128;
-    CUtensorMap tq64, tdo64, tkv128, tpe128, tq128, tdo128, tkv64, tpe64;
-    if (!make_tmap_bf16(&tq64, q, q_row, S, q_row * 2, 64) || !make_tmap_bf16(&tdo64, dout, do_row, S, do_row * 2, 64) ||
-        !make_tmap_bf16(&tkv128, kv, N, S, static_cast<uint64_t>(N) * 2, 128) ||
-        !make_tmap_bf16(&tpe128, k_pe, kDr, S, kDr * 2, 128) || !make_tmap_bf16(&tq128, q, q_row, S, q_row * 2, 128) ||
-        !make_tmap_bf16(&tdo128, dout, do_row, S, do_row * 2, 128) ||
-        !make_tmap_bf16(&tkv64, kv, N, S, static_cast<uint64_t>(N) * 2, 64) ||
-        !make_tmap_bf16(&tpe64, k_pe, kDr, S, kDr * 2, 64))
+    CUtensorMap tq, tkv, tpe, tq64, tdo64;   // boxes of 64 columns x 128 rows (x 64 rows for the dkv query tiles)
+    if (!make_tmap_bf16(&tq, q, q_row, S, q_row * 2, 128) || !make_tmap_bf16(&tq64, q, q_row, S, q_row * 2, 64) ||
+        !make_tmap_bf16(&tdo64, dout, do_row, S, do_row * 2, 64) ||
+        !make_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, 128) ||
+        !make_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, 128))
         return LAGA_ERR_CUDA;
     dim3 grid((S + 127) / 128, h, 1);
     AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
                      reinterpret_cast<__nv_bfloat16*>(dkv), dk_rope, status};
-    AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad, reinterpret_cast<__nv_bfloat16*>(dq),
-                    status};
+    AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad,
+                    reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status};
     if (causal) {
         auto k1 = attn_bwd_dkv_sm100_kernel<true>;
         auto k2 = attn_bwd_dq_sm100_kernel<true>;
         if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
             return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv, tpe, a); }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b); }
     } else {
         auto k1 = attn_bwd_dkv_sm100_kernel<false>;
         auto k2 = attn_bwd_dq_sm100_kernel<false>;
         if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
             return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv128, tpe128, a); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv, tpe, a); }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq128, tdo128, tkv64, tpe64, b); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b); }
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     {
