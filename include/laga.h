@@ -85,8 +85,8 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
  *   dk_pe   bf16 [S, d_rope]             written: summed over this shard's heads
  *   dw_kv_b fp32 [d_c, h*(d_nope+d_v)]   overwritten, or accumulated into with LAGA_FLAG_ACCUM_DW
  * K_nope/V are recomputed from c_kv (the forward keeps only out and lse).  All accumulation is fp32.
- * dw_kv_b is reduced over the sequence with floating-point atomics: its low-order bits may differ
- * from run to run.
+ * dw_kv_b (over the sequence) and dk_pe (over the heads) are reduced with floating-point atomics:
+ * their low-order bits may differ from run to run.
  */
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
              const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
@@ -152,7 +152,7 @@ int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, 
 #define LAGA_KERNEL_BWD_DELTA 2     /* delta = rowsum(dO * O) and transposed statistics        */
 #define LAGA_KERNEL_ATTN_BWD_DKV 3  /* backward attention: dK, dV                              */
 #define LAGA_KERNEL_ATTN_BWD_DQ 4   /* backward attention: dQ                                  */
-#define LAGA_KERNEL_DKPE_REDUCE 5   /* dk_pe = sum over heads of the rope-column key gradient  */
+#define LAGA_KERNEL_DKPE_REDUCE 5   /* dk_pe: bf16 rounding of the head-summed rope-column sums */
 #define LAGA_KERNEL_DCKV_GEMM 6     /* dc_kv = dKV . W^T                                       */
 #define LAGA_KERNEL_DW_GEMM 7       /* dW = c_kv^T . dKV                                       */
 #define LAGA_KERNEL_COUNT 8

@@ -73,16 +73,18 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __r
     }
 }
 
-// dk_pe[t, r] = sum over heads of the per-head rope-column key gradients (Section 5.3: the rope band
-// is shared by every head, so its gradient is the sum over the head shard).
+// dk_pe[t, r] is the sum over heads of the rope-column key gradients (Section 5.3: the rope band is
+// shared by every head, so its gradient is the sum over the head shard).  The dK/dV kernel adds each
+// head's columns into an fp32 accumulator with atomics; this kernel rounds the sums to bf16.
 __global__ void __launch_bounds__(256)
-bwd_dkpe_reduce_kernel(const float* __restrict__ dk_rope, int S, int h, __nv_bfloat16* __restrict__ dk_pe) {
-    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const size_t n = static_cast<size_t>(S) * 64;
-    if (idx >= n) return;
-    float acc = 0.f;
-    for (int i = 0; i < h; ++i) acc += dk_rope[static_cast<size_t>(i) * n + idx];
-    dk_pe[idx] = __float2bfloat16_rn(acc);
+bwd_dkpe_convert_kernel(const float* __restrict__ dkpe_acc, int S, __nv_bfloat16* __restrict__ dk_pe) {
+    const size_t idx = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
+    if (idx >= static_cast<size_t>(S) * 64) return;
+    const float4 v = *reinterpret_cast<const float4*>(dkpe_acc + idx);
+    uint2 o;
+    o.x = pack_bf16x2(v.x, v.y);
+    o.y = pack_bf16x2(v.z, v.w);
+    *reinterpret_cast<uint2*>(dk_pe + idx) = o;
 }
 
 constexpr int kBwdThreads = 320;
@@ -97,7 +99,7 @@ struct AttnBwdDkvArgs {
     const float* stat_l2;      // [h][S_pad]
     const float* stat_delta;   // [h][S_pad]
     __nv_bfloat16* dkv;        // [S, h*256]: per head dK_nope (128) then dV (128)
-    float* dk_rope;            // [h][S][64]
+    float* dkpe_acc;           // [S][64] fp32, zeroed by the host; every head's CTA adds into it
     unsigned int* status;
 };
 
@@ -329,7 +331,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             tc_fence_after_sync();
             const bool valid = t_idx < args.S;
             __nv_bfloat16* dkv_row = args.dkv + static_cast<size_t>(t_idx) * args.h * 256 + head * 256;
-            float* dkr_row = args.dk_rope + (static_cast<size_t>(head) * args.S + t_idx) * 64;
+            float* dkr_row = args.dkpe_acc + static_cast<size_t>(t_idx) * 64;
             // 10 chunks of 32 columns: dK nope (0..3), dK rope (4..5), dV (6..9; dV follows dK in TMEM).
             // Group 0 drains chunks 0..4, group 1 chunks 5..9.
 #pragma unroll 1
@@ -344,7 +346,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     for (int v = 0; v < 8; ++v) {
                         float4 w = make_float4(__uint_as_float(r[v * 4]) * args.scale, __uint_as_float(r[v * 4 + 1]) * args.scale,
                                                __uint_as_float(r[v * 4 + 2]) * args.scale, __uint_as_float(r[v * 4 + 3]) * args.scale);
-                        reinterpret_cast<float4*>(dkr_row + (c - 4) * 32)[v] = w;
+                        atomicAdd(reinterpret_cast<float4*>(dkr_row + (c - 4) * 32) + v, w);
                     }
                 } else {
                     const float mul = c < 4 ? args.scale : 1.0f;

@@ -192,7 +192,7 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
 
 // ---- Section 5.2: backward of step 5 ------------------------------------------------------------
 struct BwdWorkspace {
-    size_t kv, dkv, stat_l2, stat_delta, dk_rope, total;
+    size_t kv, dkv, stat_l2, stat_delta, dkpe_acc, total;
     int S_pad;
 };
 
@@ -205,14 +205,14 @@ BwdWorkspace bwd_workspace_layout(int S, int h) {
     w.dkv = w.kv + kv_bytes;
     w.stat_l2 = w.dkv + kv_bytes;
     w.stat_delta = w.stat_l2 + stat_bytes;
-    w.dk_rope = w.stat_delta + stat_bytes;
-    w.total = w.dk_rope + align_up(static_cast<size_t>(h) * S * kDr * sizeof(float), 1024);
+    w.dkpe_acc = w.stat_delta + stat_bytes;
+    w.total = w.dkpe_acc + align_up(static_cast<size_t>(S) * kDr * sizeof(float), 1024);
     return w;
 }
 
 int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void* out, const float* lse,
                     const void* dout, int S, int h, float softmax_scale, int causal, void* dq, void* dkv,
-                    void* dk_pe, float* stat_l2, float* stat_delta, float* dk_rope, int S_pad, unsigned* status,
+                    void* dk_pe, float* stat_l2, float* stat_delta, float* dkpe_acc, int S_pad, unsigned* status,
                     cudaStream_t stream) {
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
@@ -225,6 +225,8 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
                                                      stat_l2, stat_delta);
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     }
+    if (cudaMemsetAsync(dkpe_acc, 0, static_cast<size_t>(S) * kDr * sizeof(float), stream) != cudaSuccess)
+        return LAGA_ERR_CUDA;
     const uint64_t q_row = static_cast<uint64_t>(h) * 192, do_row = static_cast<uint64_t>(h) * 128;
     CUtensorMap tq, tkv, tpe, tq64, tdo64;   // boxes of 64 columns x 128 rows (x 64 rows for the dkv query tiles)
     if (!make_tmap_bf16(&tq, q, q_row, S, q_row * 2, 128) || !make_tmap_bf16(&tq64, q, q_row, S, q_row * 2, 64) ||
@@ -234,7 +236,7 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         return LAGA_ERR_CUDA;
     dim3 grid((S + 127) / 128, h, 1);
     AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
-                     reinterpret_cast<__nv_bfloat16*>(dkv), dk_rope, status};
+                     reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, status};
     AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad,
                     reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status};
     if (causal) {
@@ -256,10 +258,10 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     {
-        const size_t n = static_cast<size_t>(S) * kDr;
+        const size_t n = static_cast<size_t>(S) * kDr / 4;
         ScopedKernelEvents ev(LAGA_KERNEL_DKPE_REDUCE, stream);
-        bwd_dkpe_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
-            dk_rope, S, h, reinterpret_cast<__nv_bfloat16*>(dk_pe));
+        bwd_dkpe_convert_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
+            dkpe_acc, S, reinterpret_cast<__nv_bfloat16*>(dk_pe));
     }
     return launch_status();
 }
@@ -377,7 +379,7 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
     if ((rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
     if ((rc = launch_attn_bwd(q, kv, k_pe, out, lse, dout, S, h, softmax_scale, causal, dq, dkv, dk_pe,
                               reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
-                              reinterpret_cast<float*>(base + w.dk_rope), w.S_pad, status, st)) != LAGA_OK)
+                              reinterpret_cast<float*>(base + w.dkpe_acc), w.S_pad, status, st)) != LAGA_OK)
         return rc;
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
     return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, status, st);

@@ -64,7 +64,7 @@ def test_workspace_sizes(laga):
     assert laga.fwd_workspace_bytes(S, h) == 1024 + kv_bytes
     bwd = laga.bwd_workspace_bytes(S, h)
     assert bwd >= 1024 + 2 * kv_bytes              # recomputed KV and dKV, both bf16
-    assert bwd <= 1024 + 2 * kv_bytes + S * h * (64 * 4 + 2 * 4) + 8192
+    assert bwd <= 1024 + 2 * kv_bytes + S * h * 2 * 4 + S * 64 * 4 + 8192
     assert laga.fwd_workspace_bytes(300, 3) % 1024 == 0 and laga.bwd_workspace_bytes(300, 3) % 1024 == 0
     # unsupported geometry or empty problem: 0
     assert laga.fwd_workspace_bytes(128, 2, d_c=256) == 0

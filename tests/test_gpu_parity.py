@@ -103,7 +103,8 @@ def test_forward_is_repeatable_and_accum_flag(laga):
     dq2, dc2, dk2, dw2, _ = laga.bwd(q, c_kv, k_pe, w, out1, lse1, dout, dw_kv_b=dw.clone(),
                                      flags=laga.FLAG_ACCUM_DW, workspace=ws2)
     laga.check_status(ws2)
-    assert torch.equal(dq, dq2) and torch.equal(dc, dc2) and torch.equal(dk, dk2)
+    assert torch.equal(dq, dq2) and torch.equal(dc, dc2)
+    assert (dk.float() - dk2.float()).abs().max() <= 2.0 ** -7 * dk.float().abs().max()   # head sum uses atomics
     assert (dw2 - 2 * dw).abs().max() <= 1e-3 * dw.abs().max()   # accumulated on top, up to atomic order
 
 
