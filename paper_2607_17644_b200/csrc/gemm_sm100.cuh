@@ -5,9 +5,11 @@
 //     dc_kv [S, d_c] = dKV  [S, N]   . W^T                 A K-major,  B K-major,  bf16 out
 //     dW    [d_c, N] = c_kv^T . dKV                        A MN-major, B MN-major, fp32 atomic out (split-K)
 //
-// One CTA computes one 128 x BN output tile over a K range.  Warp 0 issues TMA loads, warp 1 issues
-// the MMAs, warps 2..5 drain the accumulator from TMEM (each warp owns the 32 TMEM lanes its
-// warp-id-mod-4 selects).  Operand tiles are 64 K-elements deep, 128-byte swizzled, STAGES deep.
+// Persistent: one CTA per SM walks the 128 x BN output tiles (n fastest, so neighbouring CTAs share
+// the A tile through L2).  Warp 0 issues TMA loads, warp 1 issues the MMAs, warps 2..5 drain the
+// accumulator from TMEM (each warp owns the 32 TMEM lanes its warp-id-mod-4 selects).  There are two
+// accumulators of BN columns, so the epilogue of one tile runs under the main loop of the next.
+// Operand tiles are 64 K-elements deep, 128-byte swizzled, STAGES deep.
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -16,6 +18,7 @@ namespace laga {
 struct GemmArgs {
     int M, N, K;          // problem size; M may be ragged, N % BN == 0, K tail is zero-filled by TMA
     int k_tiles_per_split;
+    int n_splits;         // split-K factor (1 unless EPI_ATOMIC_F32)
     void* C;              // bf16 [M, ldc] (EPI_BF16) or fp32 [M, ldc] (EPI_ATOMIC_F32)
     int ldc;
     unsigned int* status;
@@ -37,25 +40,26 @@ __global__ void __launch_bounds__(192, 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const GemmArgs args) {
     using L = GemmSmem<BN, STAGES>;
+    static_assert(2 * BN <= 512, "two accumulators must fit in TMEM");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::kBarrierOffset);
     uint64_t* empty_bar = full_bar + STAGES;
-    uint64_t* acc_bar = empty_bar + STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
+    uint64_t* acc_full = empty_bar + STAGES;   // [2]
+    uint64_t* acc_empty = acc_full + 2;        // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * 128;
+    const int tiles_n = args.N / BN;
+    const int tiles_m = (args.M + 127) / 128;
+    const int total_tiles = tiles_n * tiles_m * args.n_splits;
     const int total_k_tiles = (args.K + 63) / 64;
-    const int kt_begin = blockIdx.z * args.k_tiles_per_split;
-    const int kt_end = min(total_k_tiles, kt_begin + args.k_tiles_per_split);
-    const int n_kt = max(0, kt_end - kt_begin);
-    constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;
+    constexpr uint32_t kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        mbar_init(acc_bar, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_a);
@@ -67,13 +71,24 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (n_kt > 0) {
-        if (warp == 0) {
-            if (elect_one()) {
-                for (int i = 0; i < n_kt; ++i) {
-                    const int s = i % STAGES;
-                    const uint32_t ph = (i / STAGES) & 1;
-                    if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_flag, args.status, 0x100)) break;
+    auto k_range = [&](int split, int& kt_begin, int& n_kt) {
+        kt_begin = split * args.k_tiles_per_split;
+        const int kt_end = min(total_k_tiles, kt_begin + args.k_tiles_per_split);
+        n_kt = max(0, kt_end - kt_begin);
+    };
+
+    if (warp == 0) {
+        if (elect_one()) {
+            uint32_t kc = 0;   // running k-iteration count: stage = kc % STAGES, phase = (kc / STAGES) & 1
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int n0 = (t % tiles_n) * BN, m0 = ((t / tiles_n) % tiles_m) * 128;
+                int kt_begin, n_kt;
+                k_range(t / (tiles_n * tiles_m), kt_begin, n_kt);
+                for (int i = 0; i < n_kt; ++i, ++kc) {
+                    const int s = kc % STAGES;
+                    ok = mbar_wait(&empty_bar[s], ((kc / STAGES) & 1) ^ 1, abort_flag, args.status, 0x100);
+                    if (!ok) break;
                     uint8_t* sa = smem + s * L::kStageBytes;
                     uint8_t* sb = sa + L::kABytes;
                     mbar_arrive_expect_tx(&full_bar[s], L::kStageBytes);
@@ -92,14 +107,23 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
             }
-        } else if (warp == 1) {
-            if (elect_one()) {
-                constexpr uint32_t idesc = make_idesc_bf16(128, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
-                bool ok = true;
-                for (int i = 0; i < n_kt && ok; ++i) {
-                    const int s = i % STAGES;
-                    const uint32_t ph = (i / STAGES) & 1;
-                    ok = mbar_wait(&full_bar[s], ph, abort_flag, args.status, 0x200);
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            constexpr uint32_t idesc = make_idesc_bf16(128, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+            uint32_t kc = 0, it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+                int kt_begin, n_kt;
+                k_range(t / (tiles_n * tiles_m), kt_begin, n_kt);
+                const uint32_t buf = it & 1;
+                ok = mbar_wait(&acc_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, args.status, 0x201);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t tmem_acc = tmem_base + buf * BN;
+                for (int i = 0; i < n_kt; ++i, ++kc) {
+                    const int s = kc % STAGES;
+                    ok = mbar_wait(&full_bar[s], (kc / STAGES) & 1, abort_flag, args.status, 0x200);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint32_t sa = smem_u32(smem + s * L::kStageBytes);
@@ -108,23 +132,34 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     for (int k = 0; k < 4; ++k) {
                         const uint64_t da = A_MN ? desc_mn_major(sa + k * 2048, 8192) : desc_k_major(sa + k * 32);
                         const uint64_t db = B_MN ? desc_mn_major(sb + k * 2048, 8192) : desc_k_major(sb + k * 32);
-                        mma_ss(tmem_base, da, db, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                        mma_ss(tmem_acc, da, db, idesc, (i > 0 || k > 0) ? 1u : 0u);
                     }
                     mma_commit(&empty_bar[s]);
                 }
-                mma_commit(acc_bar);
+                if (ok) mma_commit(&acc_full[buf]);
             }
-        } else {
-            // Epilogue: TMEM lane = output row within the tile, TMEM column = output column.
-            const int quarter = warp & 3;
+        }
+    } else {
+        // Epilogue: TMEM lane = output row within the tile, TMEM column = output column.
+        const int quarter = warp & 3;
+        const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+            const int n0 = (t % tiles_n) * BN, m0 = ((t / tiles_n) % tiles_m) * 128;
+            int kt_begin, n_kt;
+            k_range(t / (tiles_n * tiles_m), kt_begin, n_kt);
+            const uint32_t buf = it & 1;
             const int row = m0 + quarter * 32 + lane;
-            if (mbar_wait_warp(acc_bar, 0, abort_flag, args.status, 0x300)) {
-                tc_fence_after_sync();
+            ok = mbar_wait_warp(&acc_full[buf], (it >> 1) & 1, abort_flag, args.status, 0x300);
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (n_kt > 0) {
 #pragma unroll 1
                 for (int c = 0; c < BN / 32; ++c) {
                     uint32_t r[32];
                     __syncwarp();
-                    tmem_ld_x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + c * 32, r);
+                    tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 32, r);
                     tmem_ld_wait();
                     if (row < args.M) {
                         if (EPI == EPI_BF16) {
@@ -141,14 +176,19 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                 dst4[v] = o;
                             }
                         } else {
-                            float* dst = reinterpret_cast<float*>(args.C) + static_cast<size_t>(row) * args.ldc +
-                                         n0 + c * 32;
+                            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.C) +
+                                                                    static_cast<size_t>(row) * args.ldc + n0 + c * 32);
 #pragma unroll
-                            for (int v = 0; v < 32; ++v) atomicAdd(dst + v, __uint_as_float(r[v]));
+                            for (int v = 0; v < 8; ++v)
+                                atomicAdd(dst + v, make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                                                               __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3])));
                         }
                     }
                 }
             }
+            __syncwarp();
+            tc_fence_before_sync();
+            mbar_arrive(&acc_empty[buf]);
         }
     }
     tc_fence_before_sync();

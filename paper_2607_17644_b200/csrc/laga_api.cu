@@ -73,6 +73,25 @@ int check_device() {
     return cached_major == 10 ? LAGA_OK : LAGA_ERR_UNSUPPORTED;
 }
 
+// Number of SMs of the current device (cached per device); 148 if the query fails.
+int sm_count() {
+    static int cached_dev = -1, cached_sms = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cached_dev != dev) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) cached_sms = sms;
+        cached_dev = dev;
+    }
+    return cached_sms;
+}
+
+// Persistent kernels launch one CTA per SM (fewer if there are fewer tiles).
+unsigned persistent_grid(int total_tiles) {
+    const int sms = sm_count();
+    return static_cast<unsigned>(total_tiles < sms ? (total_tiles < 1 ? 1 : total_tiles) : sms);
+}
+
 template <typename Kernel>
 int set_smem(Kernel kernel, int bytes) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
@@ -116,8 +135,8 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
     if (!make_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
     if (!make_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
     if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-    GemmArgs a{S, N, kDc, kDc / 64, kv, N, status};
-    dim3 grid(N / BN, (S + 127) / 128, 1);
+    GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status};
+    dim3 grid(persistent_grid((N / BN) * ((S + 127) / 128)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
@@ -133,8 +152,8 @@ int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, unsig
     if (!make_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
     if (!make_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN)) return LAGA_ERR_CUDA;
     if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-    GemmArgs a{S, kDc, N, (N + 63) / 64, dc_kv, kDc, status};
-    dim3 grid(kDc / BN, (S + 127) / 128, 1);
+    GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status};
+    dim3 grid(persistent_grid((kDc / BN) * ((S + 127) / 128)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
@@ -153,15 +172,23 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool a
     if (!accumulate &&
         cudaMemsetAsync(dw, 0, sizeof(float) * static_cast<size_t>(kDc) * N, stream) != cudaSuccess)
         return LAGA_ERR_CUDA;
+    // Split the sequence so that tiles x splits fills whole waves of the persistent grid: the smallest
+    // split count (fewest atomics) whose last wave is at least 90 % full, else the best found.
     const int tiles = (kDc / 128) * (N / BN);
     const int k_tiles = (S + 63) / 64;
-    int splits = (2 * 148 + tiles - 1) / tiles;
-    if (splits > k_tiles) splits = k_tiles;
-    if (splits < 1) splits = 1;
+    const int sms = sm_count();
+    int splits = 1;
+    double best = 0.0;
+    for (int s = 1; s <= 16 && s <= k_tiles; ++s) {
+        const int total = tiles * s;
+        const double eff = static_cast<double>(total) / (static_cast<double>((total + sms - 1) / sms) * sms);
+        if (eff > best + 1e-9) { best = eff; splits = s; }
+        if (eff >= 0.9) { splits = s; break; }
+    }
     const int per_split = (k_tiles + splits - 1) / splits;
     splits = (k_tiles + per_split - 1) / per_split;
-    GemmArgs a{kDc, N, S, per_split, dw, N, status};
-    dim3 grid(N / BN, kDc / 128, splits);
+    GemmArgs a{kDc, N, S, per_split, splits, dw, N, status};
+    dim3 grid(persistent_grid(tiles * splits), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
