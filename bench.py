@@ -35,7 +35,12 @@ from paper_2607_17644_b200.inputs import CONFIGS, CONFIG_SEEDS, LagaShape, make_
 METRIC = "laga_attention_block_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 WORKLOAD = "c2"
-KERNELS_PER_STEP = 9   # fwd: up_project, attn_fwd; bwd: up_project, delta, dkv, dq, dkpe_reduce, dckv, dw
+KERNELS_PER_STEP = 9   # fwd: up_project, attn_fwd; bwd: up_project, delta, dkv, dq, dkpe_convert, dckv, dw
+# DRAM bytes (read + write) per launch of attn_bwd_dkv, from the ncu capture summarised in
+# profiles/ncu_full_c3_sp8_kernels.txt (S=8192, h=16: 155.5 MB read + 42.8 MB written), expressed per
+# (token, head).  The kernel's traffic is its inputs and outputs once each (K/V, Q and dO tiles are
+# re-read from L2, not DRAM), so it grows in proportion to S*h and is scaled that way to the workload.
+DKV_DRAM_BYTES_PER_TOKEN_HEAD = (155.488256e6 + 42.770688e6) / (8192 * 16)
 
 
 def flops(sh: LagaShape):
@@ -270,7 +275,9 @@ def run_cuda(args):
                      "peak": peaks["bf16_tflops_sustained"], "unit": UNIT,
                      "frac": fl["attn_bwd_dkv"] / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                      "peak_source": peaks["source"] + " sustained cuBLAS bf16 (kernel timed inside a long step)",
-                     "kernel_ms": dom_ms, "flops_per_launch": fl["attn_bwd_dkv"], "traffic": None},
+                     "kernel_ms": dom_ms, "flops_per_launch": fl["attn_bwd_dkv"],
+                     "traffic": DKV_DRAM_BYTES_PER_TOKEN_HEAD * sh.S * sh.h,
+                     "traffic_note": "bytes per launch, ncu dram read+write at S=8192,h=16 scaled by S*h"},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(sample_tokens=args.cpu_sample_tokens)
