@@ -147,10 +147,10 @@ def barrier(world):
     torch.cuda.synchronize()
 
 
-def max_over_ranks(value: float, world: int) -> float:
+def max_over_ranks(value: float, world: int, device: str = "cuda") -> float:
     if world > 1:
         import torch.distributed as dist
-        t = torch.tensor([value], dtype=torch.float64, device="cuda")
+        t = torch.tensor([value], dtype=torch.float64, device=device)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
     return value

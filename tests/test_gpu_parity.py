@@ -168,3 +168,36 @@ def test_benchmark_configs_sampled(laga, oracle, name):
     b = float((f64(c_kv) * f64(g["dc_kv"])).sum())
     scale = float(f64(w).norm() * f64(g["dw"]).norm())
     assert abs(a - b) <= 1e-3 * scale, (a, b, scale)
+
+
+@pytest.mark.parametrize("sp", [4, 1])
+def test_sp_degree_shards(laga, oracle, sp):
+    """Benchmark configuration 3: one rank's shard at several SP degrees (h_local = 128 / SP, S = 8192),
+    all cut from the same 128-head draw.  The GPU runs the whole shard; the oracle checks sampled rows
+    of three heads (a head's O, LSE, dQ and dW columns depend on that head alone), and the h_local=16
+    shard must reproduce the first 16 heads of the wider shard bit for bit (paper Prop. 1)."""
+    h = 128 // sp
+    sh = LagaShape(S=8192, h=h)
+    tensors = make_inputs(sh, CONFIG_SEEDS["c3_sp1"], h_generate=128)
+    q, c_kv, k_pe, w, dout = tensors
+    g = run_gpu(laga, tensors, True)
+    rows = _sample_rows(sh.S, 12, 3)
+    heads = [0, h // 2, h - 1]
+    for i in heads:
+        cols = slice(i * 256, (i + 1) * 256)
+        r = oracle.bwd_rows(q[:, i:i + 1].contiguous(), c_kv, k_pe, w[:, cols].contiguous(),
+                            dout[:, i:i + 1].contiguous(), sh.d_v, sh.softmax_scale, rows, kv_round_bf16=True)
+        check_tensor(f"out[rows, head {i}]", g["out"][rows, i:i + 1], r["out"])
+        assert max_abs(g["lse"][rows, i:i + 1], r["lse"]) <= TOL_LSE
+        check_tensor(f"dq[rows, head {i}]", g["dq"][rows, i:i + 1], r["dq"])
+    # shared-tensor gradients on late keys (cheap for the oracle) over all heads of the shard
+    keys = [sh.S - 1, sh.S - 70, sh.S - 130]
+    k = oracle.bwd_keys(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, keys, kv_round_bf16=True)
+    check_tensor("dk_pe[keys]", g["dk_pe"][keys], k["dk_pe"])
+    check_tensor("dc_kv[keys]", g["dc_kv"][keys], k["dc_kv"])
+    # the SP=8 shard is a prefix of this one
+    t16 = make_inputs(LagaShape(S=8192, h=16), CONFIG_SEEDS["c3_sp8"], h_generate=128)
+    assert torch.equal(t16[0], q[:, :16]) and torch.equal(t16[3], w[:, :16 * 256])
+    g16 = run_gpu(laga, t16, True)
+    assert torch.equal(g16["out"], g["out"][:, :16]) and torch.equal(g16["lse"], g["lse"][:, :16])
+    assert torch.equal(g16["dq"], g["dq"][:, :16])
