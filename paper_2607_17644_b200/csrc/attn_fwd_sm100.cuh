@@ -4,9 +4,12 @@
 // band k_pe[S, 64] is a separate TMA box, so the 192-wide key is never assembled in memory.
 //
 // One CTA owns 128 query rows of one head and walks the key tiles (128 keys each).
-//   warp 0      TMA producer: Q once, then K and V tiles, two stages each
+//   warp 0      TMA producer: K and V tiles, two stages each
 //   warp 1      MMA issuer:   S = Q K^T (12 tcgen05.mma of K=16) into one of two TMEM tiles;
-//                             O += P V  (8 tcgen05.mma, A operand read from TMEM) into a TMEM accumulator
+//                             O += P V  (8 tcgen05.mma) into a TMEM accumulator.  Both read their A operand
+//                             (Q, P) from TMEM: a 128x128 MMA with both operands in shared memory reads
+//                             8 KB per 64 clocks, all of the SM's shared-memory bandwidth, and the TMA
+//                             writes of the next K/V tile would have to share it.
 //   warps 2..5  softmax: one thread per query row; online max / sum in registers; P is written back as
 //               packed bf16 over the first 64 columns of the S tile it came from and consumed from
 //               there by the second contraction; lazy rescale of O
@@ -20,6 +23,7 @@ namespace laga {
 struct AttnFwdArgs {
     int S, h;
     float scale_log2;       // softmax_scale * log2(e)
+    const __nv_bfloat16* q; // [S, h, 192]
     __nv_bfloat16* out;     // [S, h, 128]
     float* lse;             // [S, h]
     unsigned int* status;
@@ -27,8 +31,7 @@ struct AttnFwdArgs {
 
 struct AttnFwdSmem {
     static constexpr int kSlab = 128 * 128;             // 128 rows x 128 bytes
-    static constexpr int kQ = 0;                        // 3 slabs
-    static constexpr int kK = kQ + 3 * kSlab;           // 2 stages x 3 slabs (nope lo, nope hi, rope)
+    static constexpr int kK = 0;                        // 2 stages x 3 slabs (nope lo, nope hi, rope)
     static constexpr int kV = kK + 2 * 3 * kSlab;       // 2 stages x 2 slabs
     static constexpr int kBar = kV + 2 * 2 * kSlab;
     static constexpr int kTotalBytes = kBar + 256 + 1024;
@@ -40,15 +43,21 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 template <bool kCausal>
 __global__ void __launch_bounds__(192, 1)
-attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
-                      const __grid_constant__ CUtensorMap tmap_kpe, const AttnFwdArgs args) {
+attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
+                      const AttnFwdArgs args) {
     using L = AttnFwdSmem;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
-    uint64_t* q_full = bars + 0;
+    uint64_t* q_ready = bars + 0;    // the softmax threads have put the Q tile into TMEM
     uint64_t* k_full = bars + 1;     // [2]
     uint64_t* k_empty = bars + 3;    // [2]
     uint64_t* v_full = bars + 5;     // [2]
@@ -67,7 +76,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     const int n_kv = kCausal ? q_tile + 1 : n_q_tiles;
 
     if (threadIdx.x == 0) {
-        mbar_init(q_full, 1);
+        mbar_init(q_ready, 128);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
             mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
@@ -76,20 +85,18 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         mbar_init(p_full, 128); mbar_init(pv_done, 1);
         abort_flag->value = 0;
         mbar_fence_init();
-        tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
+        tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
     }
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_o = tmem_base + 256;
+    const uint32_t tmem_o = tmem_base + 256;     // [0,256) two S tiles | [256,384) O | [384,480) Q as packed bf16
+    const uint32_t tmem_q = tmem_base + 384;
 
     if (warp == 0) {
         if (elect_one()) {
-            mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
-            for (int c = 0; c < 3; ++c)
-                tma_load_2d(smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
             for (int j = 0; j < n_kv; ++j) {
                 const int s = j & 1;
                 const uint32_t ph_free = ((j >> 1) & 1) ^ 1;
@@ -110,7 +117,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         if (elect_one()) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);
-            const uint32_t sq = smem_u32(smem + L::kQ);
             auto issue_qk = [&](int j) -> bool {
                 const int s = j & 1;
                 if (!mbar_wait(&k_full[s], (j >> 1) & 1, abort_flag, args.status, 0x23)) return false;
@@ -119,14 +125,14 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 #pragma unroll
                 for (int kk = 0; kk < 12; ++kk) {
                     const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
-                    mma_ss(tmem_base + s * 128, desc_k_major(sq + off), desc_k_major(sk + off), idesc_qk,
-                           kk > 0 ? 1u : 0u);
+                    mma_ts(tmem_base + s * 128, tmem_q + kk * 8, desc_k_major(sk + off), idesc_qk, kk > 0 ? 1u : 0u);
                 }
                 mma_commit(&k_empty[s]);
                 mma_commit(&s_full[s]);
                 return true;
             };
-            bool ok = mbar_wait(q_full, 0, abort_flag, args.status, 0x22);
+            bool ok = mbar_wait(q_ready, 0, abort_flag, args.status, 0x22);
+            tc_fence_after_sync();
             if (ok) ok = issue_qk(0);
             if (ok && n_kv > 1) ok = issue_qk(1);
             for (int j = 0; j < n_kv && ok; ++j) {
@@ -150,6 +156,24 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         const int row = quarter * 32 + lane;          // row inside the tile == TMEM lane
         const int sq_idx = q0 + row;                  // global query index
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+        {   // this thread's query row (192 bf16 = 96 packed words) goes to TMEM once, as the A operand of S
+            const bool q_valid = sq_idx < args.S;
+            const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(sq_idx) * args.h + head) * 192);
+#pragma unroll 1
+            for (int c = 0; c < 3; ++c) {
+                uint32_t w[32];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const uint4 x = q_valid ? src[c * 8 + v] : make_uint4(0u, 0u, 0u, 0u);
+                    w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
+                }
+                __syncwarp();
+                tmem_st_x32(tmem_q + lane_addr + c * 32, w);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(q_ready);
+        }
         float m_run = -INFINITY, l_run = 0.f;         // running max (scaled, log2 domain) and sum
         bool ok = true;
         for (int j = 0; j < n_kv; ++j) {
@@ -171,13 +195,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 }
             }
             // eight independent chains: a single warp per scheduler cannot hide a 128-deep dependency
+            // (three-input max: two elements per instruction)
             float mxs[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) mxs[e] = __uint_as_float(sv[e]);
+            for (int e = 0; e < 8; ++e) mxs[e] = fmaxf(__uint_as_float(sv[e]), __uint_as_float(sv[8 + e]));
 #pragma unroll
-            for (int c = 8; c < 128; ++c) mxs[c & 7] = fmaxf(mxs[c & 7], __uint_as_float(sv[c]));
-            const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
-                                   fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+            for (int c = 16; c < 128; c += 16)
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    mxs[e] = fmax3(mxs[e], __uint_as_float(sv[c + e]), __uint_as_float(sv[c + 8 + e]));
+            const float mx = fmaxf(fmax3(mxs[0], mxs[1], mxs[2]), fmax3(fmax3(mxs[3], mxs[4], mxs[5]), mxs[6], mxs[7]));
             const float m_new = fmaxf(m_run, mx * args.scale_log2);
             // Lazy rescale: keep the old reference max unless it fell behind by more than 2^8.
             const bool move = (m_new - m_run) > 8.0f;
