@@ -141,6 +141,16 @@ int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, 
                              void* out, float* lse, void* stream);
 
 /*
+ * Self-test of the failure-detection path.  Every device-side wait in this library is bounded: a
+ * wait that outlives its budget records where it gave up in the status word and the kernel unwinds
+ * instead of hanging.  This call launches a one-CTA kernel whose waits can never be satisfied, with a
+ * budget of `budget_us` microseconds (1 .. 1000000); afterwards laga_query_status(status_word, ...)
+ * returns LAGA_ERR_DEVICE_TIMEOUT with detail 0x54007e57, and the context stays usable.  Nothing
+ * faults, traps or spins past the budget.  The paper has no counterpart.
+ */
+int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stream);
+
+/*
  * Measurement aid.  Registers n_pairs CUDA events pairs (cudaEvent_t passed as void*, created by the
  * caller with timing enabled) that the library records on the launch stream immediately before and
  * after every launch of one kernel, cycling through the pairs launch after launch; n_pairs = 0 stops

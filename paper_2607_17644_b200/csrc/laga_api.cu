@@ -292,6 +292,22 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
     return launch_status();
 }
 
+// Self-test of the bounded-wait machinery every kernel here relies on: two warps wait on an mbarrier
+// that nothing will ever arrive on.  After `budget_ns` the first waiter records the site in the status
+// word and raises the abort flag, the other waiter sees the flag, and the CTA exits normally.
+__global__ void selftest_bounded_wait_kernel(unsigned* status, unsigned long long budget_ns) {
+    __shared__ uint64_t never_signalled;
+    __shared__ AbortFlag abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&never_signalled, 1);
+        abort_flag.value = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait_warp(&never_signalled, 0, &abort_flag, status, 0x7e57u, budget_ns);
+    if (ok && threadIdx.x == 0) atomicExch(status, 0xdeadu);   // cannot happen: nothing arrives
+}
+
 int zero_status(void* status_word, cudaStream_t stream) {
     return cudaMemsetAsync(status_word, 0, sizeof(unsigned), stream) == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA;
 }
@@ -461,6 +477,17 @@ int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, 
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
     if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
     return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st);
+}
+
+int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stream) {
+    if (!status_word || budget_us < 1 || budget_us > 1000000) return LAGA_ERR_INVALID_ARG;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = zero_status(status_word, st)) != LAGA_OK) return rc;
+    selftest_bounded_wait_kernel<<<1, 64, 0, st>>>(static_cast<unsigned*>(status_word),
+                                                   static_cast<unsigned long long>(budget_us) * 1000ull);
+    return launch_status();
 }
 
 int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs) {

@@ -76,7 +76,8 @@ struct AbortFlag {
 // Bounded wait.  Returns true when the phase completed; false after the budget ran out or another
 // role already aborted (the status word then names the first site that gave up).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, AbortFlag* abort_flag,
-                                          unsigned int* status, uint32_t site) {
+                                          unsigned int* status, uint32_t site,
+                                          unsigned long long budget_ns = kWaitBudgetNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     uint32_t polls = 0;
@@ -84,7 +85,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, AbortF
         if (mbar_try_wait(bar, parity)) return true;
         if ((++polls & 0xffu) == 0u) {
             if (abort_flag->value != 0u) return false;
-            if (global_timer_ns() - t0 > kWaitBudgetNs) {
+            if (global_timer_ns() - t0 > budget_ns) {
                 abort_flag->value = 1u;
                 if (status) atomicCAS(status, kStatusOk, kStatusTimeout | site);
                 return false;
@@ -96,8 +97,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, AbortF
 // Warp-uniform variant for code that goes on to execute warp-collective (.sync.aligned)
 // instructions: every lane gets the same answer.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, AbortFlag* abort_flag,
-                                               unsigned int* status, uint32_t site) {
-    const bool ok = mbar_wait(bar, parity, abort_flag, status, site);
+                                               unsigned int* status, uint32_t site,
+                                               unsigned long long budget_ns = kWaitBudgetNs) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, site, budget_ns);
     return __all_sync(0xffffffffu, ok);
 }
 

@@ -35,6 +35,7 @@ SIGNATURES = {
     "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
     "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
     "laga_profile_kernel": (_ci, [_ci, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _ci]),
+    "laga_selftest_bounded_wait": (_ci, [_vp, _cu, _vp]),
     "laga_fwd_builtin_scratch": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp]),
 }
 BUILTIN_SCRATCH_MAX_TOKEN_HEADS = 32768   # S * h limit of laga_fwd_builtin_scratch (16 MiB of bf16 KV)
@@ -237,6 +238,14 @@ def profile_kernel(kernel: str, start_events=(), stop_events=()):
     starts = (_vp * max(n, 1))(*[e.cuda_event for e in start_events])
     stops = (_vp * max(n, 1))(*[e.cuda_event for e in stop_events])
     _check(lib().laga_profile_kernel(KERNELS[kernel], starts, stops, n), "laga_profile_kernel")
+
+
+def selftest_bounded_wait(budget_us: int = 1000, stream=None):
+    """laga_selftest_bounded_wait: run the kernel whose waits cannot complete; returns the status word
+    tensor to pass to query_status (expected: ERR_DEVICE_TIMEOUT, detail 0x54007e57)."""
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().laga_selftest_bounded_wait(_ptr(word), int(budget_us), _stream(stream)), "laga_selftest_bounded_wait")
+    return word
 
 
 def query_status(workspace_or_word, stream=None) -> tuple[int, int]:

@@ -201,3 +201,16 @@ def test_sp_degree_shards(laga, oracle, sp):
     g16 = run_gpu(laga, t16, True)
     assert torch.equal(g16["out"], g["out"][:, :16]) and torch.equal(g16["lse"], g["lse"][:, :16])
     assert torch.equal(g16["dq"], g["dq"][:, :16])
+
+
+def test_bounded_wait_reports_a_timeout_and_leaves_the_context_usable(laga):
+    """Failure detection without a fault: a kernel whose mbarrier is never signalled gives up after
+    its budget, the host reads LAGA_ERR_DEVICE_TIMEOUT with the site id, and the next call works."""
+    word = laga.selftest_bounded_wait(budget_us=2000)
+    rc, detail = laga.query_status(word)
+    assert rc == laga.ERR_DEVICE_TIMEOUT and detail == 0x54007E57
+    sh = LagaShape(S=256, h=1)
+    q, c_kv, k_pe, w, _ = (t.cuda() if t is not None else None for t in make_inputs(sh, 5, with_dout=False))
+    out, lse, ws = laga.fwd(q, c_kv, k_pe, w)
+    laga.check_status(ws)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
