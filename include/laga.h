@@ -47,6 +47,7 @@ extern "C" {
 #define LAGA_ERR_DEVICE_TIMEOUT (-5)      /* only from laga_query_status: a bounded device wait ran out */
 
 #define LAGA_FLAG_ACCUM_DW 1u             /* laga_bwd: add into dw_kv_b instead of overwriting it   */
+#define LAGA_FLAG_DETERMINISTIC 2u        /* laga_bwd: bitwise-repeatable dk_pe and dw_kv_b (see there) */
 
 /* Library version (major*10000 + minor*100 + patch). */
 int laga_version(void);
@@ -86,7 +87,10 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
  *   dw_kv_b fp32 [d_c, h*(d_nope+d_v)]   overwritten, or accumulated into with LAGA_FLAG_ACCUM_DW
  * K_nope/V are recomputed from c_kv (the forward keeps only out and lse).  All accumulation is fp32.
  * dw_kv_b (over the sequence) and dk_pe (over the heads) are reduced with floating-point atomics:
- * their low-order bits may differ from run to run.
+ * their low-order bits may differ from run to run.  LAGA_FLAG_DETERMINISTIC removes that: dw_kv_b is
+ * then computed without splitting the sequence (one addition per element; fewer CTAs, so the dW GEMM
+ * is slower) and dk_pe is summed over per-head buffers in head order (S*h*d_rope*4 more workspace
+ * bytes: pass the same flags to laga_bwd_workspace_bytes).  dq and dc_kv are repeatable either way.
  */
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
              const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,

@@ -87,6 +87,17 @@ bwd_dkpe_convert_kernel(const float* __restrict__ dkpe_acc, int S, __nv_bfloat16
     *reinterpret_cast<uint2*>(dk_pe + idx) = o;
 }
 
+// Deterministic alternative to the atomics: sum the per-head buffers in head order.
+__global__ void __launch_bounds__(256)
+bwd_dkpe_reduce_kernel(const float* __restrict__ dk_rope, int S, int h, __nv_bfloat16* __restrict__ dk_pe) {
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const size_t n = static_cast<size_t>(S) * 64;
+    if (idx >= n) return;
+    float acc = 0.f;
+    for (int i = 0; i < h; ++i) acc += dk_rope[static_cast<size_t>(i) * n + idx];
+    dk_pe[idx] = __float2bfloat16_rn(acc);
+}
+
 constexpr int kBwdThreads = 320;
 constexpr int kBwdStages = 3;
 
@@ -100,6 +111,8 @@ struct AttnBwdDkvArgs {
     const float* stat_delta;   // [h][S_pad]
     __nv_bfloat16* dkv;        // [S, h*256]: per head dK_nope (128) then dV (128)
     float* dkpe_acc;           // [S][64] fp32, zeroed by the host; every head's CTA adds into it
+    float* dk_rope_per_head;   // deterministic mode: [h][S][64] fp32 written per head (then summed in a fixed
+                               // order by bwd_dkpe_reduce_kernel); nullptr selects the atomic path
     unsigned int* status;
 };
 
@@ -346,7 +359,11 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     for (int v = 0; v < 8; ++v) {
                         float4 w = make_float4(__uint_as_float(r[v * 4]) * args.scale, __uint_as_float(r[v * 4 + 1]) * args.scale,
                                                __uint_as_float(r[v * 4 + 2]) * args.scale, __uint_as_float(r[v * 4 + 3]) * args.scale);
-                        atomicAdd(reinterpret_cast<float4*>(dkr_row + (c - 4) * 32) + v, w);
+                        if (args.dk_rope_per_head != nullptr)
+                            reinterpret_cast<float4*>(args.dk_rope_per_head +
+                                                      (static_cast<size_t>(head) * args.S + t_idx) * 64 + (c - 4) * 32)[v] = w;
+                        else
+                            atomicAdd(reinterpret_cast<float4*>(dkr_row + (c - 4) * 32) + v, w);
                     }
                 } else {
                     const float mul = c < 4 ? args.scale : 1.0f;

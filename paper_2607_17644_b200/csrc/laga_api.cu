@@ -160,8 +160,8 @@ int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, unsig
 
 // dW[d_c, N] (+)= c_kv^T . dKV   (both operands read with the token index as K: MN-major), split over
 // the sequence with fp32 atomic accumulation.
-int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool accumulate, unsigned* status,
-              cudaStream_t stream) {
+int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool accumulate, bool deterministic,
+              unsigned* status, cudaStream_t stream) {
     constexpr int BN = 256, STAGES = 4;
     auto kernel = gemm_sm100_kernel<BN, STAGES, true, true, EPI_ATOMIC_F32>;
     using L = GemmSmem<BN, STAGES>;
@@ -179,7 +179,7 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool a
     const int sms = sm_count();
     int splits = 1;
     double best = 0.0;
-    for (int s = 1; s <= 16 && s <= k_tiles; ++s) {
+    for (int s = 1; s <= 16 && s <= k_tiles && !deterministic; ++s) {   // one split: one add per element
         const int total = tiles * s;
         const double eff = static_cast<double>(total) / (static_cast<double>((total + sms - 1) / sms) * sms);
         if (eff > best + 1e-9) { best = eff; splits = s; }
@@ -218,11 +218,11 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
 
 // ---- Section 5.2: backward of step 5 ------------------------------------------------------------
 struct BwdWorkspace {
-    size_t kv, dkv, stat_l2, stat_delta, dkpe_acc, total;
+    size_t kv, dkv, stat_l2, stat_delta, dkpe_acc, dk_rope_per_head, total;
     int S_pad;
 };
 
-BwdWorkspace bwd_workspace_layout(int S, int h) {
+BwdWorkspace bwd_workspace_layout(int S, int h, bool deterministic) {
     BwdWorkspace w;
     const size_t kv_bytes = align_up(static_cast<size_t>(S) * h * (kDn + kDv) * 2, 1024);
     w.S_pad = (S + 127) / 128 * 128;
@@ -232,13 +232,16 @@ BwdWorkspace bwd_workspace_layout(int S, int h) {
     w.stat_l2 = w.dkv + kv_bytes;
     w.stat_delta = w.stat_l2 + stat_bytes;
     w.dkpe_acc = w.stat_delta + stat_bytes;
-    w.total = w.dkpe_acc + align_up(static_cast<size_t>(S) * kDr * sizeof(float), 1024);
+    w.dk_rope_per_head = w.dkpe_acc + align_up(static_cast<size_t>(S) * kDr * sizeof(float), 1024);
+    w.total = w.dk_rope_per_head +
+              (deterministic ? align_up(static_cast<size_t>(h) * S * kDr * sizeof(float), 1024) : 0);
     return w;
 }
 
 int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void* out, const float* lse,
                     const void* dout, int S, int h, float softmax_scale, int causal, void* dq, void* dkv,
-                    void* dk_pe, float* stat_l2, float* stat_delta, float* dkpe_acc, int S_pad, unsigned* status,
+                    void* dk_pe, float* stat_l2, float* stat_delta, float* dkpe_acc, float* dk_rope_per_head, int S_pad,
+                    unsigned* status,
                     cudaStream_t stream) {
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
@@ -262,7 +265,7 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         return LAGA_ERR_CUDA;
     dim3 grid((S + 127) / 128, h, 1);
     AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
-                     reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, status};
+                     reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, dk_rope_per_head, status};
     AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad,
                     reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status};
     if (causal) {
@@ -284,10 +287,16 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     {
-        const size_t n = static_cast<size_t>(S) * kDr / 4;
         ScopedKernelEvents ev(LAGA_KERNEL_DKPE_REDUCE, stream);
-        bwd_dkpe_convert_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
-            dkpe_acc, S, reinterpret_cast<__nv_bfloat16*>(dk_pe));
+        if (dk_rope_per_head != nullptr) {
+            const size_t n = static_cast<size_t>(S) * kDr;
+            bwd_dkpe_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
+                dk_rope_per_head, S, h, reinterpret_cast<__nv_bfloat16*>(dk_pe));
+        } else {
+            const size_t n = static_cast<size_t>(S) * kDr / 4;
+            bwd_dkpe_convert_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
+                dkpe_acc, S, reinterpret_cast<__nv_bfloat16*>(dk_pe));
+        }
     }
     return launch_status();
 }
@@ -336,9 +345,8 @@ size_t laga_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, i
 }
 
 size_t laga_bwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v, unsigned flags) {
-    (void)flags;
     if (S < 1 || h < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
-    return bwd_workspace_layout(S, h).total;
+    return bwd_workspace_layout(S, h, (flags & LAGA_FLAG_DETERMINISTIC) != 0).total;
 }
 
 int laga_up_project(const void* c_kv, const void* w_kv_b, int S, int h, int d_c, int d_nope, int d_v, void* kv,
@@ -359,7 +367,7 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
         return LAGA_ERR_INVALID_ARG;
     if (!aligned16(dkv) || !aligned16(c_kv) || !aligned16(w_kv_b) || !aligned16(dc_kv) || !aligned16(dw_kv_b))
         return LAGA_ERR_INVALID_ARG;
-    if (flags & ~LAGA_FLAG_ACCUM_DW) return LAGA_ERR_INVALID_ARG;
+    if (flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC)) return LAGA_ERR_INVALID_ARG;
     if (!geometry_supported(d_c, d_nope, kDr, d_v)) return LAGA_ERR_UNSUPPORTED;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
@@ -368,7 +376,8 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
     const int N = h * (kDn + kDv);
     if ((rc = zero_status(status_word, st)) != LAGA_OK) return rc;
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
-    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, status, st);
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0,
+                     (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st);
 }
 
 int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
@@ -404,9 +413,10 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
         !aligned16(lse) || !aligned16(dout) || !aligned16(dq) || !aligned16(dc_kv) || !aligned16(dk_pe) ||
         !aligned16(dw_kv_b) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return LAGA_ERR_INVALID_ARG;
-    if ((flags & ~LAGA_FLAG_ACCUM_DW) || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
+    if ((flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC)) || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
     if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
-    const BwdWorkspace w = bwd_workspace_layout(S, h);
+    const bool deterministic = (flags & LAGA_FLAG_DETERMINISTIC) != 0;
+    const BwdWorkspace w = bwd_workspace_layout(S, h, deterministic);
     if (workspace_bytes < w.total) return LAGA_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
@@ -421,10 +431,12 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
     if ((rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
     if ((rc = launch_attn_bwd(q, kv, k_pe, out, lse, dout, S, h, softmax_scale, causal, dq, dkv, dk_pe,
                               reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
-                              reinterpret_cast<float*>(base + w.dkpe_acc), w.S_pad, status, st)) != LAGA_OK)
+                              reinterpret_cast<float*>(base + w.dkpe_acc),
+                              deterministic ? reinterpret_cast<float*>(base + w.dk_rope_per_head) : nullptr, w.S_pad, status,
+                              st)) != LAGA_OK)
         return rc;
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
-    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, status, st);
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, deterministic, status, st);
 }
 
 // ---- forward without caller-provided scratch ----------------------------------------------------

@@ -18,6 +18,7 @@ ERR_WORKSPACE_TOO_SMALL = -3
 ERR_CUDA = -4
 ERR_DEVICE_TIMEOUT = -5
 FLAG_ACCUM_DW = 1
+FLAG_DETERMINISTIC = 2
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblaga.so")
 _lib = None

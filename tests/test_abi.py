@@ -65,6 +65,7 @@ def test_workspace_sizes(laga):
     bwd = laga.bwd_workspace_bytes(S, h)
     assert bwd >= 1024 + 2 * kv_bytes              # recomputed KV and dKV, both bf16
     assert bwd <= 1024 + 2 * kv_bytes + S * h * 2 * 4 + S * 64 * 4 + 8192
+    assert laga.bwd_workspace_bytes(S, h, flags=laga.FLAG_DETERMINISTIC) >= bwd + S * h * 64 * 4
     assert laga.fwd_workspace_bytes(300, 3) % 1024 == 0 and laga.bwd_workspace_bytes(300, 3) % 1024 == 0
     # unsupported geometry or empty problem: 0
     assert laga.fwd_workspace_bytes(128, 2, d_c=256) == 0
@@ -102,7 +103,7 @@ def test_argument_validation_happens_before_any_device_work(laga):
                             a["d_rope"], a["d_v"], 0.07, 1, dq, good, good, good, good, ws_bytes, flags, None)
 
     assert bwd(dq=None) == laga.ERR_INVALID_ARG
-    assert bwd(flags=2) == laga.ERR_INVALID_ARG
+    assert bwd(flags=4) == laga.ERR_INVALID_ARG
     assert bwd(d_v=64) == laga.ERR_UNSUPPORTED
     assert bwd(ws_bytes=4096) == laga.ERR_WORKSPACE_TOO_SMALL
     assert lib.laga_up_project(None, good, 128, 2, 512, 128, 128, good, good, None) == laga.ERR_INVALID_ARG

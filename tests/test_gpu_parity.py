@@ -214,3 +214,25 @@ def test_bounded_wait_reports_a_timeout_and_leaves_the_context_usable(laga):
     out, lse, ws = laga.fwd(q, c_kv, k_pe, w)
     laga.check_status(ws)
     assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+
+
+def test_deterministic_flag_gives_bitwise_repeatable_gradients(laga, oracle):
+    sh = LagaShape(S=1100, h=5)
+    tensors = make_inputs(sh, 77)
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in tensors)
+    out, lse, ws = laga.fwd(q, c_kv, k_pe, w)
+    runs = []
+    for _ in range(3):
+        dq, dc, dk, dw, ws2 = laga.bwd(q, c_kv, k_pe, w, out, lse, dout, flags=laga.FLAG_DETERMINISTIC)
+        laga.check_status(ws2)
+        runs.append([t.clone() for t in (dq, dc, dk, dw)])
+    for other in runs[1:]:
+        for a, b in zip(runs[0], other):
+            assert torch.equal(a, b)
+    r = oracle.bwd(*tensors, sh.d_v, sh.softmax_scale, kv_round_bf16=True)
+    check_tensor("dk_pe", runs[0][2], r["dk_pe"])
+    check_dw(runs[0][3], r["dw"])
+    # the default (atomic) path agrees with it to rounding
+    dq2, dc2, dk2, dw2, _ = laga.bwd(q, c_kv, k_pe, w, out, lse, dout)
+    assert torch.equal(dq2, runs[0][0]) and torch.equal(dc2, runs[0][1])
+    assert (dw2 - runs[0][3]).abs().max() <= 1e-4 * runs[0][3].abs().max()
