@@ -64,6 +64,38 @@ def activation_memory(sh: LagaShape, ws_fwd: int, ws_bwd: int, allocated_in_step
             "workspace_bytes": {"fwd": ws_fwd, "bwd": ws_bwd}, "allocated_inside_step": allocated_in_step}
 
 
+def compare_eager(sh: LagaShape, inputs, cuda_results, laga_ms: float, laga_peak_bytes: dict, reps: int = 2):
+    """Time the explicit (B1) and absorbed (B2) forms of the same block written in eager PyTorch ops
+    with the full S x S score matrix, as the paper's memory study ran them (Section 6, memory table),
+    and record what each keeps alive beyond its inputs.  Library kernels, comparison only."""
+    from paper_2607_17644_b200 import eager_forms
+    q, c_kv, k_pe, w, dout = inputs
+    res = {"how": "eager PyTorch bf16 (cuBLAS + ATen) with autograd, full S x S scores per head; peak_bytes = "
+                  "torch.cuda.max_memory_allocated above the inputs, over one forward+backward",
+           "laga_cuda": {"ms_per_step": laga_ms, "peak_bytes": laga_peak_bytes["laga_bytes"]}}
+    names = ("out", "dq", "dc_kv", "dk_pe", "dw_kv_b")
+    for name, form in (("explicit", eager_forms.explicit_form), ("absorbed", eager_forms.absorbed_form)):
+        torch.cuda.synchronize()
+        torch.cuda.empty_cache()
+        got = eager_forms.run_form(form, q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale)   # warm-up + check
+        err = {n: float((g.float() - r.float()).abs().max()) for n, g, r in zip(names, got, cuda_results)}
+        del got
+        torch.cuda.synchronize()
+        torch.cuda.empty_cache()
+        base = torch.cuda.memory_allocated()
+        torch.cuda.reset_peak_memory_stats()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            eager_forms.run_form(form, q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale)
+        e1.record()
+        torch.cuda.synchronize()
+        res[name] = {"ms_per_step": e0.elapsed_time(e1) / reps, "peak_bytes": torch.cuda.max_memory_allocated() - base,
+                     "max_abs_diff_vs_laga_cuda": err}
+    res["absorbed_minus_explicit_bytes"] = res["absorbed"]["peak_bytes"] - res["explicit"]["peak_bytes"]
+    return res
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -338,6 +370,10 @@ def run_cuda(args):
                      "traffic": DKV_DRAM_BYTES_PER_TOKEN_HEAD * sh.S * sh.h,
                      "traffic_note": "bytes per launch, ncu dram read+write at S=8192,h=16 scaled by S*h"},
     }
+    if args.compare_eager and world == 1:
+        del in_dev, out_dev, host_outs
+        line["eager_forms"] = compare_eager(sh, (q, c_kv, k_pe, w, dout), (out, dq, dc_kv, dk_pe, dw),
+                                            laga_ms=ms_per_step, laga_peak_bytes=line["activation_memory"])
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(sample_tokens=args.cpu_sample_tokens)
     if rank == 0:
@@ -414,6 +450,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--workload", choices=sorted(CONFIGS), default=WORKLOAD,
                     help="benchmark configuration (default c2, the headline; others are for profiling)")
+    ap.add_argument("--compare-eager", action="store_true",
+                    help="also time the explicit and absorbed forms in eager PyTorch (N=1; tens of GB at c2)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=16384,
                     help="tokens of head 0 the cpu_baseline leg runs (16384 = the whole head: ~10 s on 16 cores)")
     ap.add_argument("--ref-sample-tokens", type=int, default=2048,
