@@ -3,18 +3,27 @@
 // S x S scores.  K_nope and V are read from the bf16 up-projection KV[S, h*256]; the shared rope
 // band k_pe[S, 64] is a separate TMA box, so the 192-wide key is never assembled in memory.
 //
-// One CTA owns 128 query rows of one head and walks the key tiles (128 keys each).
-//   warp 0      TMA producer: K and V tiles, two stages each
-//   warp 1      MMA issuer:   S = Q K^T (12 tcgen05.mma of K=16) into one of two TMEM tiles;
-//                             O += P V  (8 tcgen05.mma) into a TMEM accumulator.  Both read their A operand
-//                             (Q, P) from TMEM: a 128x128 MMA with both operands in shared memory reads
-//                             8 KB per 64 clocks, all of the SM's shared-memory bandwidth, and the TMA
-//                             writes of the next K/V tile would have to share it.
-//   warps 2..5  softmax: one thread per query row; online max / sum in registers; P is written back as
-//               packed bf16 over the first 64 columns of the S tile it came from and consumed from
-//               there by the second contraction; lazy rescale of O
-// The score tile for key tile j+2 reuses the TMEM columns of tile j; it is issued after P_j V_j by the
-// same thread, and the tensor pipe executes a thread's MMAs in order, so no extra barrier guards it.
+// One CTA owns 128 query rows of one head and walks the key tiles (96 keys each).
+//   warps 0..3  softmax warpgroup 0: even key tiles      one thread per query row in each group; the
+//   warps 4..7  softmax warpgroup 1: odd key tiles       exponentials of one group's tile run beside
+//                                                        the row maximum / load / store phases of the other's
+//   warp 8      TMA producer: K tiles, three stages
+//   warp 9      MMA issuer:   S = Q K^T (12 tcgen05.mma of K=16, N=96) into one of three TMEM tiles;
+//                             O += P V (6 tcgen05.mma of N=128).  Both read their A operand (Q, P) from TMEM:
+//                             an MMA with both operands in shared memory is bound by shared-memory
+//                             bandwidth (128 B/clk).
+//   warp 10     TMA producer: V tiles, three stages
+// Why 96 keys: the Q tile (96 columns of packed bf16), the O accumulator (128) and THREE score tiles
+// (3 x 96) fill the 512 TMEM columns exactly.  With three score tiles the tensor pipe computes S_{j+3}
+// while the two groups work on tiles j+1 and j+2, so neither side waits for the other; with 128-key
+// tiles only two fit and the chain S -> softmax -> P V -> next S on the same columns sets the pace.
+// The two groups share one running reference maximum per row (a word of shared memory handed from
+// tile to tile through the max_done barriers: only the short row-maximum phase is serial, the
+// exponentials are not) and therefore one O accumulator; each keeps its own partial row sum, brought
+// to the common reference at the end.  P is written back as packed bf16 over the first 48 columns of
+// the S tile it came from.  The score tile for key tile j+3 reuses the TMEM columns of tile j; it is
+// issued after P_j V_j by the same thread, and the tensor pipe executes a thread's MMAs in order, so
+// no extra barrier guards it.
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -29,12 +38,18 @@ struct AttnFwdArgs {
     unsigned int* status;
 };
 
+constexpr int kFwdThreads = 352;
+constexpr int kFwdKeys = 96;     // keys per tile
+constexpr int kFwdStages = 3;
+
 struct AttnFwdSmem {
-    static constexpr int kSlab = 128 * 128;             // 128 rows x 128 bytes
-    static constexpr int kK = 0;                        // 2 stages x 3 slabs (nope lo, nope hi, rope)
-    static constexpr int kV = kK + 2 * 3 * kSlab;       // 2 stages x 2 slabs
-    static constexpr int kBar = kV + 2 * 2 * kSlab;
-    static constexpr int kTotalBytes = kBar + 256 + 1024;
+    static constexpr int kSlab = kFwdKeys * 128;                 // 96 rows x 128 bytes
+    static constexpr int kK = 0;                                 // stages x 3 slabs (nope lo, nope hi, rope)
+    static constexpr int kV = kK + kFwdStages * 3 * kSlab;       // stages x 2 slabs
+    static constexpr int kMref = kV + kFwdStages * 2 * kSlab;    // 128 floats: the rows' reference maxima
+    static constexpr int kLsum = kMref + 512;                    // 2 x 128 floats: the groups' row sums
+    static constexpr int kBar = kLsum + 1024;
+    static constexpr int kTotalBytes = kBar + 512 + 1024;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -50,113 +65,147 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 }
 
 template <bool kCausal>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
                       const AttnFwdArgs args) {
     using L = AttnFwdSmem;
+    constexpr int BK = kFwdKeys;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
-    uint64_t* q_ready = bars + 0;    // the softmax threads have put the Q tile into TMEM
-    uint64_t* k_full = bars + 1;     // [2]
-    uint64_t* k_empty = bars + 3;    // [2]
-    uint64_t* v_full = bars + 5;     // [2]
-    uint64_t* v_empty = bars + 7;    // [2]
-    uint64_t* s_full = bars + 9;     // [2]
-    uint64_t* p_full = bars + 11;
-    uint64_t* pv_done = bars + 12;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+    uint64_t* q_ready = bars + 0;    // warpgroup 0 has put the Q tile into TMEM
+    uint64_t* k_full = bars + 1;     // [3]
+    uint64_t* k_empty = bars + 4;    // [3]
+    uint64_t* v_full = bars + 7;     // [3]
+    uint64_t* v_empty = bars + 10;   // [3]
+    uint64_t* s_full = bars + 13;    // [3]  S tile j is in TMEM buffer j % 3
+    uint64_t* p_full = bars + 16;    // [2]  group g has written P of its tile
+    uint64_t* pv_done = bars + 18;   // [2]  P_j V_j has completed (index j & 1)
+    uint64_t* max_done = bars + 20;  // [2]  group g has published the reference maxima of its tile
+    uint64_t* all_done = bars + 22;  // every MMA has completed
+    uint64_t* l_ready = bars + 23;   // both groups have stored their row sums
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
+    float* mref = reinterpret_cast<float*>(smem + L::kMref);
+    float* lsum = reinterpret_cast<float*>(smem + L::kLsum);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_q_tiles = (args.S + 127) / 128;
     const int q_tile = n_q_tiles - 1 - static_cast<int>(blockIdx.x);   // longest rows first
     const int head = blockIdx.y;
     const int q0 = q_tile * 128;
-    const int n_kv = kCausal ? q_tile + 1 : n_q_tiles;
+    const int n_keys = kCausal ? min(q0 + 128, args.S) : args.S;       // keys any row of this tile attends to
+    const int n_kv = (n_keys + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         mbar_init(q_ready, 128);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
-            mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
-            mbar_init(&s_full[s], 1);
+        for (int s = 0; s < 3; ++s) {
+            mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); mbar_init(&s_full[s], 1);
         }
-        mbar_init(p_full, 128); mbar_init(pv_done, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&p_full[s], 128); mbar_init(&pv_done[s], 1); mbar_init(&max_done[s], 128);
+        }
+        mbar_init(all_done, 1);
+        mbar_init(l_ready, 256);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
     }
-    if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+    if (warp == 9) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_o = tmem_base + 256;     // [0,256) two S tiles | [256,384) O | [384,480) Q as packed bf16
-    const uint32_t tmem_q = tmem_base + 384;
+    const uint32_t tmem_o = tmem_base + 3 * BK;       // [0,288) three S tiles | [288,416) O | [416,512) Q as packed bf16
+    const uint32_t tmem_q = tmem_o + 128;
 
-    if (warp == 0) {
+    if (warp == 8) {
+        // K and V have producers of their own: the score MMAs run up to three tiles ahead of the P V MMAs,
+        // and a single thread waiting for a V stage would hold back the K tile the tensor pipe needs next.
         if (elect_one()) {
             for (int j = 0; j < n_kv; ++j) {
-                const int s = j & 1;
-                const uint32_t ph_free = ((j >> 1) & 1) ^ 1;
-                if (!mbar_wait(&k_empty[s], ph_free, abort_flag, args.status, 0x10)) break;
+                const int s = j % kFwdStages;
+                if (!mbar_wait(&k_empty[s], ((j / kFwdStages) & 1) ^ 1, abort_flag, args.status, 0x10)) break;
                 uint8_t* dk = smem + L::kK + s * 3 * L::kSlab;
                 mbar_arrive_expect_tx(&k_full[s], 3 * L::kSlab);
-                tma_load_2d(dk, &tmap_kv, &k_full[s], head * 256, j * 128);
-                tma_load_2d(dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * 128);
-                tma_load_2d(dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * 128);
-                if (!mbar_wait(&v_empty[s], ph_free, abort_flag, args.status, 0x11)) break;
+                tma_load_2d(dk, &tmap_kv, &k_full[s], head * 256, j * BK);
+                tma_load_2d(dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * BK);
+                tma_load_2d(dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * BK);
+            }
+        }
+    } else if (warp == 10) {
+        if (elect_one()) {
+            for (int j = 0; j < n_kv; ++j) {
+                const int s = j % kFwdStages;
+                if (!mbar_wait(&v_empty[s], ((j / kFwdStages) & 1) ^ 1, abort_flag, args.status, 0x11)) break;
                 uint8_t* dv = smem + L::kV + s * 2 * L::kSlab;
                 mbar_arrive_expect_tx(&v_full[s], 2 * L::kSlab);
-                tma_load_2d(dv, &tmap_kv, &v_full[s], head * 256 + 128, j * 128);
-                tma_load_2d(dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * 128);
+                tma_load_2d(dv, &tmap_kv, &v_full[s], head * 256 + 128, j * BK);
+                tma_load_2d(dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * BK);
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 9) {
         if (elect_one()) {
-            constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
+            // tcgen05.mma issue is close to synchronous with the tensor pipe (about one MMA of queue), so
+            // whatever else this thread does is time the pipe idles: an mbarrier wait costs some 90 clocks
+            // even when the barrier is already complete.  Each barrier is therefore probed BEFORE the
+            // preceding batch of MMAs is issued and the answer read after it: the probe's latency passes
+            // while the MMAs block, and the bounded wait runs only when the probe came back false.
+            constexpr uint32_t idesc_qk = make_idesc_bf16(128, BK, 0, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);
-            auto issue_qk = [&](int j) -> bool {
-                const int s = j & 1;
-                if (!mbar_wait(&k_full[s], (j >> 1) & 1, abort_flag, args.status, 0x23)) return false;
-                tc_fence_after_sync();
+            auto qk_mmas = [&](int j) {
+                const int s = j % kFwdStages;
                 const uint32_t sk = smem_u32(smem + L::kK + s * 3 * L::kSlab);
 #pragma unroll
-                for (int kk = 0; kk < 12; ++kk) {
-                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
-                    mma_ts(tmem_base + s * 128, tmem_q + kk * 8, desc_k_major(sk + off), idesc_qk, kk > 0 ? 1u : 0u);
-                }
+                for (int kk = 0; kk < 12; ++kk)
+                    mma_ts(tmem_base + s * BK, tmem_q + kk * 8, desc_k_major(sk + (kk >> 2) * L::kSlab + (kk & 3) * 32),
+                           idesc_qk, kk > 0 ? 1u : 0u);
                 mma_commit(&k_empty[s]);
                 mma_commit(&s_full[s]);
-                return true;
             };
             bool ok = mbar_wait(q_ready, 0, abort_flag, args.status, 0x22);
-            tc_fence_after_sync();
-            if (ok) ok = issue_qk(0);
-            if (ok && n_kv > 1) ok = issue_qk(1);
+            for (int j = 0; j < 3 && j < n_kv && ok; ++j) {
+                ok = mbar_wait(&k_full[j], 0, abort_flag, args.status, 0x23);
+                tc_fence_after_sync();
+                if (ok) qk_mmas(j);
+            }
+            bool v_ok = false, p_ok = false;      // probes of v_full / p_full for tile j
             for (int j = 0; j < n_kv && ok; ++j) {
-                const int s = j & 1;
-                ok = mbar_wait(&v_full[s], (j >> 1) & 1, abort_flag, args.status, 0x20) &&
-                     mbar_wait(p_full, j & 1, abort_flag, args.status, 0x21);
+                const int s = j % kFwdStages, g = j & 1;
+                const uint32_t ph = (j / kFwdStages) & 1;
+                if (!v_ok) ok = mbar_wait(&v_full[s], ph, abort_flag, args.status, 0x20);
+                if (ok && !p_ok) ok = mbar_wait(&p_full[g], (j >> 1) & 1, abort_flag, args.status, 0x21);
                 if (!ok) break;
                 tc_fence_after_sync();
+                const bool more = j + 3 < n_kv;
+                const bool k_ok = more && mbar_try_wait(&k_full[s], ph ^ 1);   // K_{j+3} lands in the stage K_j left
                 const uint32_t sv = smem_u32(smem + L::kV + s * 2 * L::kSlab);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)   // A = P_j: packed bf16, 8 TMEM columns per 16 keys
-                    mma_ts(tmem_o, tmem_base + s * 128 + kk * 8, desc_mn_major(sv + kk * 2048, L::kSlab), idesc_pv,
+                for (int kk = 0; kk < BK / 16; ++kk)   // A = P_j: packed bf16, 8 TMEM columns per 16 keys
+                    mma_ts(tmem_o, tmem_base + s * BK + kk * 8, desc_mn_major(sv + kk * 2048, L::kSlab), idesc_pv,
                            (j > 0 || kk > 0) ? 1u : 0u);
                 mma_commit(&v_empty[s]);
-                mma_commit(pv_done);
-                if (j + 2 < n_kv) ok = issue_qk(j + 2);
+                mma_commit(&pv_done[g]);
+                v_ok = p_ok = false;
+                if (more) {
+                    if (!k_ok) ok = mbar_wait(&k_full[s], ph ^ 1, abort_flag, args.status, 0x23);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const int s1 = (j + 1) % kFwdStages;
+                    v_ok = mbar_try_wait(&v_full[s1], ((j + 1) / kFwdStages) & 1);
+                    p_ok = mbar_try_wait(&p_full[g ^ 1], ((j + 1) >> 1) & 1);
+                    qk_mmas(j + 3);
+                }
             }
+            if (ok) mma_commit(all_done);
         }
     } else {
+        const int g = warp >> 2;                      // softmax warpgroup: key tiles j with (j & 1) == g
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;          // row inside the tile == TMEM lane
         const int sq_idx = q0 + row;                  // global query index
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-        {   // this thread's query row (192 bf16 = 96 packed words) goes to TMEM once, as the A operand of S
+        if (g == 0) {   // this thread's query row (192 bf16 = 96 packed words) goes to TMEM once, as the A operand of S
             const bool q_valid = sq_idx < args.S;
             const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(sq_idx) * args.h + head) * 192);
 #pragma unroll 1
@@ -174,57 +223,74 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             tc_fence_before_sync();
             mbar_arrive(q_ready);
         }
-        float m_run = -INFINITY, l_run = 0.f;         // running max (scaled, log2 domain) and sum
+        float m_mine = -INFINITY;                     // reference max (scaled, log2 domain) l_part refers to
+        float l_part = 0.f;                           // this group's part of the row sum
         bool ok = true;
-        for (int j = 0; j < n_kv; ++j) {
-            const int s = j & 1;
-            ok = mbar_wait_warp(&s_full[s], (j >> 1) & 1, abort_flag, args.status, 0x30);
+        for (int j = g; j < n_kv; j += 2) {
+            const int b = j % kFwdStages;
+            const uint32_t tmem_s = tmem_base + lane_addr + b * BK;
+            ok = mbar_wait_warp(&s_full[b], (j / kFwdStages) & 1, abort_flag, args.status, 0x30);
             if (!ok) break;
             tc_fence_after_sync();
-            uint32_t sv[128];
+            uint32_t sv[BK];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld_x32(tmem_base + lane_addr + s * 128 + c * 32, sv + c * 32);
+            for (int c = 0; c < BK / 32; ++c) tmem_ld_x32(tmem_s + c * 32, sv + c * 32);
             tmem_ld_wait();
 
-            const bool edge = (j == n_kv - 1);
-            if (edge) {
+            const int t_last = j * BK + BK - 1;
+            if ((kCausal && t_last > q0) || t_last >= args.S) {   // the causal edge can cross two tiles
 #pragma unroll
-                for (int c = 0; c < 128; ++c) {
-                    const int t = j * 128 + c;
+                for (int c = 0; c < BK; ++c) {
+                    const int t = j * BK + c;
                     if ((kCausal && t > sq_idx) || t >= args.S) sv[c] = __float_as_uint(-INFINITY);
                 }
             }
-            // eight independent chains: a single warp per scheduler cannot hide a 128-deep dependency
-            // (three-input max: two elements per instruction)
+            // eight independent chains (three-input max: two elements per instruction)
             float mxs[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) mxs[e] = fmaxf(__uint_as_float(sv[e]), __uint_as_float(sv[8 + e]));
 #pragma unroll
-            for (int c = 16; c < 128; c += 16)
+            for (int c = 16; c < BK; c += 16)
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
                     mxs[e] = fmax3(mxs[e], __uint_as_float(sv[c + e]), __uint_as_float(sv[c + 8 + e]));
             const float mx = fmaxf(fmax3(mxs[0], mxs[1], mxs[2]), fmax3(fmax3(mxs[3], mxs[4], mxs[5]), mxs[6], mxs[7]));
-            const float m_new = fmaxf(m_run, mx * args.scale_log2);
-            // Lazy rescale: keep the old reference max unless it fell behind by more than 2^8.
-            const bool move = (m_new - m_run) > 8.0f;
-            const float alpha = move ? fast_exp2(m_run - m_new) : 1.0f;
-            if (move) m_run = m_new;
+
+            // The reference maximum as the other group left it after tile j-1.  Tile 0 holds an unmasked key
+            // for every row, so the reference is finite from there on; a later tile may be masked out for a
+            // row altogether (mx = -inf), which leaves the reference alone and yields P = 0.
+            float m_old = -INFINITY;
+            if (j > 0) {
+                ok = mbar_wait_warp(&max_done[g ^ 1], ((j - 1) >> 1) & 1, abort_flag, args.status, 0x33);
+                if (!ok) break;
+                m_old = mref[row];
+            }
+            const float m_cand = fmaxf(m_old, mx * args.scale_log2);
+            // Lazy rescale: keep the old reference unless it fell behind by more than 2^8.
+            const bool move = (m_cand - m_old) > 8.0f;
+            const float m_new = move ? m_cand : m_old;
+            if (move) mref[row] = m_new;
+            mbar_arrive(&max_done[g]);
+            const float alpha = move ? fast_exp2(m_old - m_new) : 1.0f;               // for O (all earlier tiles)
+            const float beta = (m_mine == m_new) ? 1.0f : fast_exp2(m_mine - m_new);   // for this group's sum
+            m_mine = m_new;
+
             float sums[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            uint32_t pk[64];
+            uint32_t pk[BK / 2];
 #pragma unroll
-            for (int c = 0; c < 64; ++c) {
-                const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * c]), args.scale_log2, -m_run));
-                const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * c + 1]), args.scale_log2, -m_run));
+            for (int c = 0; c < BK / 2; ++c) {
+                const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * c]), args.scale_log2, -m_new));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * c + 1]), args.scale_log2, -m_new));
                 sums[c & 7] += p0 + p1;
                 pk[c] = pack_bf16x2(p0, p1);
             }
             const float sum = ((sums[0] + sums[1]) + (sums[2] + sums[3])) + ((sums[4] + sums[5]) + (sums[6] + sums[7]));
-            l_run = l_run * alpha + sum;
+            l_part = l_part * beta + sum;
 
             if (j > 0 && __any_sync(0xffffffffu, move)) {
-                // O must be at rest: P_{j-1} V_{j-1} finished, P_j V_j not issued before p_full below.
-                ok = mbar_wait_warp(pv_done, (j - 1) & 1, abort_flag, args.status, 0x31);
+                // O must be at rest: P_{j-1} V_{j-1} finished (the previous phase of its barrier, tile j-3,
+                // is known complete because S_j was issued after it), P_j V_j not issued before p_full below.
+                ok = mbar_wait_warp(&pv_done[g ^ 1], ((j - 1) >> 1) & 1, abort_flag, args.status, 0x31);
                 if (!ok) break;
                 tc_fence_after_sync();
 #pragma unroll 1
@@ -237,20 +303,32 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     tmem_st_x32(tmem_o + lane_addr + c * 32, o);
                 }
             }
-            tmem_st_x32(tmem_base + lane_addr + s * 128, pk);
-            tmem_st_x32(tmem_base + lane_addr + s * 128 + 32, pk + 32);
+            tmem_st_x32(tmem_s, pk);
+            tmem_st_x16(tmem_s + 32, pk + 32);
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(p_full);
+            mbar_arrive(&p_full[g]);
         }
-        if (ok) ok = mbar_wait_warp(pv_done, (n_kv - 1) & 1, abort_flag, args.status, 0x32);
+        // Bring this group's sum to the final reference (set by the owner of the last tile) and add the
+        // two groups' sums.
+        const int last = n_kv - 1;
+        if (ok && (last & 1) != g) ok = mbar_wait_warp(&max_done[g ^ 1], (last >> 1) & 1, abort_flag, args.status, 0x34);
+        float m_fin = 0.f;
+        if (ok) {
+            m_fin = mref[row];
+            lsum[g * 128 + row] = l_part * ((m_mine == m_fin) ? 1.0f : fast_exp2(m_mine - m_fin));
+            mbar_arrive(l_ready);
+            ok = mbar_wait_warp(l_ready, 0, abort_flag, args.status, 0x35);
+        }
+        if (ok) ok = mbar_wait_warp(all_done, 0, abort_flag, args.status, 0x32);
         if (ok) {
             tc_fence_after_sync();
+            const float l_run = lsum[row] + lsum[128 + row];
             const float inv_l = 1.0f / l_run;
             const bool valid = sq_idx < args.S;
             __nv_bfloat16* dst = args.out + (static_cast<size_t>(sq_idx) * args.h + head) * 128;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 2 * g; c < 2 * g + 2; ++c) {     // each group drains half of the O columns
                 uint32_t o[32];
                 __syncwarp();
                 tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
@@ -267,13 +345,13 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     }
                 }
             }
-            if (valid)
-                args.lse[static_cast<size_t>(sq_idx) * args.h + head] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+            if (valid && g == 0)
+                args.lse[static_cast<size_t>(sq_idx) * args.h + head] = (m_fin + log2f(l_run)) * 0.6931471805599453f;
         }
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    if (warp == 9) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
 }
 
 }  // namespace laga

@@ -198,20 +198,20 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
                     int causal, void* out, float* lse, unsigned* status, cudaStream_t stream) {
     using L = AttnFwdSmem;
     const int N = h * (kDn + kDv);
-    CUtensorMap tkv, tpe;
-    if (!make_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
-    if (!make_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, 128)) return LAGA_ERR_CUDA;
+    CUtensorMap tkv, tpe;   // boxes of 64 columns x one key tile of rows
+    if (!make_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, kFwdKeys)) return LAGA_ERR_CUDA;
+    if (!make_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, kFwdKeys)) return LAGA_ERR_CUDA;
     AttnFwdArgs a{S, h, softmax_scale * 1.4426950408889634f, reinterpret_cast<const __nv_bfloat16*>(q),
                   reinterpret_cast<__nv_bfloat16*>(out), lse, status};
     dim3 grid((S + 127) / 128, h, 1);
     if (causal) {
         auto kernel = attn_fwd_sm100_kernel<true>;
         if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(tkv, tpe, a); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a); }
     } else {
         auto kernel = attn_fwd_sm100_kernel<false>;
         if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(tkv, tpe, a); }
+        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a); }
     }
     return launch_status();
 }
