@@ -237,18 +237,22 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 mma_commit(&dp_full[g]);
                 return true;
             };
-            auto issue_acc = [&](int j) -> bool {    // dV += P^T dO_j, dK += dS^T Q_j (A operands from TMEM)
+            auto issue_dv = [&](int j) -> bool {     // dV += P^T dO_j (A operand from TMEM)
                 const int g = j & 1;
-                const uint32_t ph = (j >> 1) & 1;
-                if (!mbar_wait(&p_full[g], ph, abort_flag, args.status, 0x50)) return false;
-                if (!mbar_wait(&ds_full[g], ph, abort_flag, args.status, 0x51)) return false;
+                if (!mbar_wait(&p_full[g], (j >> 1) & 1, abort_flag, args.status, 0x50)) return false;
                 tc_fence_after_sync();
-                const uint32_t sq = stage_q(j);
-                const uint32_t sdo = sq + 3 * L::kSlab64;
+                const uint32_t sdo = stage_q(j) + 3 * L::kSlab64;
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
                     mma_ts(tmem_dv, tmem_pt + g * 32 + kk * 8, desc_mn_major(sdo + kk * 2048, L::kSlab64), idesc_dv,
                            (j > 0 || kk > 0) ? 1u : 0u);
+                return true;
+            };
+            auto issue_dk = [&](int j) -> bool {     // dK += dS^T Q_j (A operand from TMEM)
+                const int g = j & 1;
+                if (!mbar_wait(&ds_full[g], (j >> 1) & 1, abort_flag, args.status, 0x51)) return false;
+                tc_fence_after_sync();
+                const uint32_t sq = stage_q(j);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
                     mma_ts(tmem_dk, tmem_base + g * 64 + kk * 8, desc_mn_major(sq + kk * 2048, L::kSlab64), idesc_dk,
@@ -256,16 +260,18 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 mma_commit(&qdo_empty[j % kBwdStages]);
                 return true;
             };
-            // Issue order per tile: S^T(j), then the accumulations of tile j-1, then dP^T(j).  Each wait
-            // has about one MMA group of slack: the other warpgroup finishes dS^T(j-1) while S^T(j)
-            // runs, and this tile's warpgroup has loaded S^T(j) long before dP^T(j) is due.
+            // Issue order per tile: S^T(j), dV(j-1), dP^T(j), dK(j-1).  dV(j-1) gives this tile's warpgroup
+            // time to load S^T(j) before dP^T(j) overwrites it, and dK(j-1) comes last so that the other
+            // warpgroup has S^T(j), dV(j-1) and dP^T(j) -- some 1200 clocks -- to turn dP^T(j-1) into dS^T(j-1).
             bool ok = mbar_wait(kv_full, 0, abort_flag, args.status, 0x54);
             for (int j = 0; j < n_iter && ok; ++j) {
                 ok = issue_st(j);
-                if (ok && j > 0) ok = issue_acc(j - 1);
+                if (ok && j > 0) ok = issue_dv(j - 1);
                 if (ok) ok = issue_dp(j);
+                if (ok && j > 0) ok = issue_dk(j - 1);
             }
-            if (ok) ok = issue_acc(n_iter - 1);
+            if (ok) ok = issue_dv(n_iter - 1);
+            if (ok) ok = issue_dk(n_iter - 1);
             if (ok) mma_commit(acc_done);
         }
     } else {
