@@ -38,38 +38,36 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gmem_sr
 // delta[s,i] = sum_d dO[s,i,d] O[s,i,d].  Written head-major and padded: stat_l2[i][s] = LSE*log2(e),
 // stat_delta[i][s] = delta for s < S; for S <= s < S_pad the entries are (+inf, 0) so that query rows
 // past the end of the sequence produce P = 0.
+// Eight lanes per (row, head): each lane reads 16 channels of O and dO as two 16-byte loads apiece.
 __global__ void __launch_bounds__(256)
 bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
                  const float* __restrict__ lse, int S, int h, int S_pad, float* __restrict__ stat_l2,
                  float* __restrict__ stat_delta) {
-    const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (warp_global >= S_pad * h) return;
-    const int s = warp_global / h, i = warp_global % h;
-    if (s >= S) {
-        if (lane == 0) {
-            stat_l2[static_cast<size_t>(i) * S_pad + s] = INFINITY;
-            stat_delta[static_cast<size_t>(i) * S_pad + s] = 0.f;
-        }
-        return;
-    }
-    const size_t base = (static_cast<size_t>(s) * h + i) * 128 + lane * 4;
-    const uint2 a = *reinterpret_cast<const uint2*>(out + base);
-    const uint2 b = *reinterpret_cast<const uint2*>(dout + base);
-    const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
-    const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b);
+    const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;   // (row, head) pair
+    const int sub = threadIdx.x & 7;
+    const bool live = item < static_cast<long long>(S_pad) * h;
+    const int s = live ? static_cast<int>(item / h) : 0, i = live ? static_cast<int>(item % h) : 0;
     float acc = 0.f;
+    if (live && s < S) {
+        const size_t base = (static_cast<size_t>(s) * h + i) * 128 + sub * 16;
+        const uint4 a0 = *reinterpret_cast<const uint4*>(out + base), a1 = *reinterpret_cast<const uint4*>(out + base + 8);
+        const uint4 b0 = *reinterpret_cast<const uint4*>(dout + base), b1 = *reinterpret_cast<const uint4*>(dout + base + 8);
+        const uint32_t aw[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+        const uint32_t bw[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        const float2 x = __bfloat1622float2(a2[k]), y = __bfloat1622float2(b2[k]);
-        acc = fmaf(x.x, y.x, acc);
-        acc = fmaf(x.y, y.y, acc);
+        for (int k = 0; k < 8; ++k) {
+            const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[k]));
+            const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[k]));
+            acc = fmaf(x.x, y.x, acc);
+            acc = fmaf(x.y, y.y, acc);
+        }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    if (lane == 0) {
-        stat_l2[static_cast<size_t>(i) * S_pad + s] = lse[static_cast<size_t>(s) * h + i] * 1.4426950408889634f;
-        stat_delta[static_cast<size_t>(i) * S_pad + s] = acc;
+    for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (live && sub == 0) {
+        const bool valid = s < S;
+        stat_l2[static_cast<size_t>(i) * S_pad + s] = valid ? lse[static_cast<size_t>(s) * h + i] * 1.4426950408889634f : INFINITY;
+        stat_delta[static_cast<size_t>(i) * S_pad + s] = valid ? acc : 0.f;
     }
 }
 

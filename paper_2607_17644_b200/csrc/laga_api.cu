@@ -246,8 +246,8 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
     {   // delta and the transposed, padded softmax statistics
-        const long long warps = static_cast<long long>(S_pad) * h;
-        const unsigned blocks = static_cast<unsigned>((warps * 32 + 255) / 256);
+        const long long items = static_cast<long long>(S_pad) * h;   // eight lanes per (row, head)
+        const unsigned blocks = static_cast<unsigned>((items * 8 + 255) / 256);
         ScopedKernelEvents ev(LAGA_KERNEL_BWD_DELTA, stream);
         bwd_delta_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(out),
                                                      reinterpret_cast<const __nv_bfloat16*>(dout), lse, S, h, S_pad,
