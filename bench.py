@@ -37,10 +37,10 @@ UNIT = "TFLOP/s"
 WORKLOAD = "c2"
 KERNELS_PER_STEP = 9   # fwd: up_project, attn_fwd; bwd: up_project, delta, dkv, dq, dkpe_convert, dckv, dw
 # DRAM bytes (read + write) per launch of attn_bwd_dkv, from the ncu capture summarised in
-# profiles/ncu_full_c3_sp8_kernels.txt (S=8192, h=16: 155.5 MB read + 42.8 MB written), expressed per
+# profiles/ncu_full_c3_sp8_kernels.txt (S=8192, h=16: 155.5 MB read + 43.3 MB written), expressed per
 # (token, head).  The kernel's traffic is its inputs and outputs once each (K/V, Q and dO tiles are
 # re-read from L2, not DRAM), so it grows in proportion to S*h and is scaled that way to the workload.
-DKV_DRAM_BYTES_PER_TOKEN_HEAD = (155.488256e6 + 42.770688e6) / (8192 * 16)
+DKV_DRAM_BYTES_PER_TOKEN_HEAD = (155.500800e6 + 43.290624e6) / (8192 * 16)
 
 
 def flops(sh: LagaShape):
