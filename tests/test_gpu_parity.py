@@ -44,6 +44,12 @@ SMALL_CASES = [
     (129, 2, True),      # one row past a tile boundary
     (1024, 4, True),     # eight key tiles
     (200, 1, False),
+    # the forward walks 96-key tiles in a three-deep ring shared by two softmax groups
+    (96, 1, True),       # exactly one forward key tile
+    (97, 2, True),       # one key past it: the second group gets a one-key tile
+    (385, 2, True),      # five forward key tiles: the ring wraps, both groups take several tiles
+    (289, 1, False),     # non-causal, four tiles with a one-key tail
+    (700, 1, True),
 ]
 
 
