@@ -48,6 +48,7 @@ extern "C" {
 
 #define LAGA_FLAG_ACCUM_DW 1u             /* laga_bwd: add into dw_kv_b instead of overwriting it   */
 #define LAGA_FLAG_DETERMINISTIC 2u        /* laga_bwd: bitwise-repeatable dk_pe and dw_kv_b (see there) */
+#define LAGA_FLAG_KV_SAVED 4u             /* laga_bwd: the workspace still holds laga_fwd's K_nope/V (see there) */
 
 /* Library version (major*10000 + minor*100 + patch). */
 int laga_version(void);
@@ -91,6 +92,11 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
  * then computed without splitting the sequence (one addition per element; fewer CTAs, so the dW GEMM
  * is slower) and dk_pe is summed over per-head buffers in head order (S*h*d_rope*4 more workspace
  * bytes: pass the same flags to laga_bwd_workspace_bytes).  dq and dc_kv are repeatable either way.
+ * LAGA_FLAG_KV_SAVED skips the recomputation of step 4: it promises that laga_fwd ran on the same
+ * c_kv and w_kv_b with this very workspace pointer (sized by laga_bwd_workspace_bytes) and that nothing
+ * has written to the workspace since -- the forward leaves K_nope/V where the backward looks for them.
+ * This is the explicit form's way of saving K/V for the backward; the price is that the workspace cannot
+ * be shared with another layer between the two calls.  The library cannot check the promise.
  */
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
              const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,

@@ -413,7 +413,8 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
         !aligned16(lse) || !aligned16(dout) || !aligned16(dq) || !aligned16(dc_kv) || !aligned16(dk_pe) ||
         !aligned16(dw_kv_b) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return LAGA_ERR_INVALID_ARG;
-    if ((flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC)) || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
+    if ((flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC | LAGA_FLAG_KV_SAVED)) || !(softmax_scale > 0.f))
+        return LAGA_ERR_INVALID_ARG;
     if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
     const bool deterministic = (flags & LAGA_FLAG_DETERMINISTIC) != 0;
     const BwdWorkspace w = bwd_workspace_layout(S, h, deterministic);
@@ -427,8 +428,9 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
     void* dkv = base + w.dkv;
     const int N = h * (kDn + kDv);
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
-    // K_nope / V are recomputed from the latent: the forward keeps only out and lse.
-    if ((rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
+    // K_nope / V are recomputed from the latent (the forward keeps only out and lse) unless the caller
+    // vouches that the forward's copy is still in this workspace: both layouts put it right after the status.
+    if (!(flags & LAGA_FLAG_KV_SAVED) && (rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
     if ((rc = launch_attn_bwd(q, kv, k_pe, out, lse, dout, S, h, softmax_scale, causal, dq, dkv, dk_pe,
                               reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
                               reinterpret_cast<float*>(base + w.dkpe_acc),

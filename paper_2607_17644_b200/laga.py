@@ -19,6 +19,7 @@ ERR_CUDA = -4
 ERR_DEVICE_TIMEOUT = -5
 FLAG_ACCUM_DW = 1
 FLAG_DETERMINISTIC = 2
+FLAG_KV_SAVED = 4
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblaga.so")
 _lib = None

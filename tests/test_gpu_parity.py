@@ -242,3 +242,23 @@ def test_deterministic_flag_gives_bitwise_repeatable_gradients(laga, oracle):
     dq2, dc2, dk2, dw2, _ = laga.bwd(q, c_kv, k_pe, w, out, lse, dout)
     assert torch.equal(dq2, runs[0][0]) and torch.equal(dc2, runs[0][1])
     assert (dw2 - runs[0][3]).abs().max() <= 1e-4 * runs[0][3].abs().max()
+
+
+def test_kv_saved_flag_reuses_the_forwards_up_projection(laga):
+    """With LAGA_FLAG_KV_SAVED the backward reads K_nope/V where the forward left them in the shared
+    workspace; with the deterministic flag on both sides the two backwards must agree bit for bit."""
+    sh = LagaShape(S=900, h=3)
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in make_inputs(sh, 78))
+    det = laga.FLAG_DETERMINISTIC
+    ws = laga.alloc_workspace(laga.bwd_workspace_bytes(sh.S, sh.h, flags=det))
+    out, lse, _ = laga.fwd(q, c_kv, k_pe, w, workspace=ws)                 # leaves KV in ws
+    saved = laga.bwd(q, c_kv, k_pe, w, out, lse, dout, workspace=ws, flags=det | laga.FLAG_KV_SAVED)[:4]
+    laga.check_status(ws)
+    saved = [t.clone() for t in saved]
+    ws.zero_()                                                            # nothing of the forward survives
+    recomputed = laga.bwd(q, c_kv, k_pe, w, out, lse, dout, workspace=ws, flags=det)[:4]
+    laga.check_status(ws)
+    for a, b in zip(saved, recomputed):
+        assert torch.equal(a, b)
+    with pytest.raises(laga.LagaError):
+        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, flags=8)               # unknown flag bit
