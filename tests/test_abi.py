@@ -103,7 +103,7 @@ def test_argument_validation_happens_before_any_device_work(laga):
                             a["d_rope"], a["d_v"], 0.07, 1, dq, good, good, good, good, ws_bytes, flags, None)
 
     assert bwd(dq=None) == laga.ERR_INVALID_ARG
-    assert bwd(flags=4) == laga.ERR_INVALID_ARG
+    assert bwd(flags=8) == laga.ERR_INVALID_ARG     # 1, 2 and 4 are defined
     assert bwd(d_v=64) == laga.ERR_UNSUPPORTED
     assert bwd(ws_bytes=4096) == laga.ERR_WORKSPACE_TOO_SMALL
     assert lib.laga_up_project(None, good, 128, 2, 512, 128, 128, good, good, None) == laga.ERR_INVALID_ARG
