@@ -228,6 +228,11 @@ def run_cuda(args):
     for e in k_starts + k_stops:
         e.record()
     laga.profile_kernel(dom, k_starts, k_stops)
+    d_starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]     # the one HBM-bound kernel of weight: delta
+    d_stops = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    for e in d_starts + d_stops:
+        e.record()
+    laga.profile_kernel("bwd_delta", d_starts, d_stops)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -240,6 +245,10 @@ def run_cuda(args):
     barrier(world)
     clocks = sampler.stop()
     laga.profile_kernel(dom)
+    laga.profile_kernel("bwd_delta")
+    delta_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(d_starts, d_stops))
+    s_pad = (sh.S + 127) // 128 * 128
+    delta_bytes = 2 * sh.S * sh.h * sh.d_v * 2 + sh.S * sh.h * 4 + 2 * s_pad * sh.h * 4   # O, dO, LSE in; two statistics out
     total_ms = max_over_ranks(ev0.elapsed_time(ev1), world)
     ms_per_step = total_ms / K
     dom_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(k_starts, k_stops))
@@ -374,6 +383,10 @@ def run_cuda(args):
         del in_dev, out_dev, host_outs
         line["eager_forms"] = compare_eager(sh, (q, c_kv, k_pe, w, dout), (out, dq, dc_kv, dk_pe, dw),
                                             laga_ms=ms_per_step, laga_peak_bytes=line["activation_memory"])
+    line["hbm_kernels"] = {"bwd_delta": {"kernel_ms": delta_ms, "bytes_per_launch": delta_bytes,
+                                         "achieved": delta_bytes / (delta_ms * 1e-3) / 1e9, "unit": "GB/s",
+                                         "peak": peaks["hbm_gbs"], "frac": delta_bytes / (delta_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                         "share_of_step": delta_ms / ms_per_step}}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(sample_tokens=args.cpu_sample_tokens)
     if rank == 0:
