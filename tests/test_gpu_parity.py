@@ -289,3 +289,27 @@ def test_long_ragged_sequence_sampled(laga, oracle):
     scale = float(f64(w).norm() * f64(g["dw"]).norm())
     assert abs(a - b) <= 1e-3 * scale, (a, b, scale)
     assert all(bool(torch.isfinite(t.float()).all()) for t in g.values())
+
+
+def test_random_small_shapes(laga, oracle):
+    """Thirty seeded random (S, h, causal) combinations with S <= 900: whatever tile-boundary case the
+    hand-picked sizes above miss (the forward tiles keys by 96, the dq kernel by 128, the dkv kernel tiles
+    queries by 64 and keys by 128).  Same element-wise bars as the fixed cases."""
+    rng = torch.Generator().manual_seed(20260717)
+    for case in range(30):
+        S = int(torch.randint(2, 901, (1,), generator=rng))
+        h = int(torch.randint(1, 5, (1,), generator=rng))
+        causal = bool(torch.randint(0, 4, (1,), generator=rng) > 0)      # three in four causal
+        sh = LagaShape(S=S, h=h)
+        tensors = make_inputs(sh, 5000 + case)
+        g = run_gpu(laga, tensors, causal)
+        q, c_kv, k_pe, w, dout = tensors
+        r = oracle.bwd(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, causal=causal, kv_round_bf16=True,
+                       return_fwd=True)
+        tag = f"[S={S} h={h} causal={causal}] "
+        check_tensor(tag + "out", g["out"], r["out"])
+        assert max_abs(g["lse"], r["lse"]) <= TOL_LSE, tag + "lse"
+        check_tensor(tag + "dq", g["dq"], r["dq"])
+        check_tensor(tag + "dk_pe", g["dk_pe"], r["dk_pe"])
+        check_tensor(tag + "dc_kv", g["dc_kv"], r["dc_kv"])
+        check_dw(g["dw"], r["dw"])
