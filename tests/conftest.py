@@ -17,3 +17,11 @@ def oracle():
     import oracle as _oracle
     _oracle.build()
     return _oracle
+
+
+def free_port() -> int:
+    """A TCP port that is free right now on 127.0.0.1 (for torch.distributed rendezvous in tests)."""
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]

@@ -59,7 +59,8 @@ def test_max_over_ranks_with_two_gloo_ranks():
     import torch.multiprocessing as mp
     ctx = mp.get_context("spawn")
     results = ctx.Manager().dict()
-    port = 29611
+    from conftest import free_port
+    port = free_port()
     procs = [ctx.Process(target=_rank_main, args=(r, 2, port, results)) for r in range(2)]
     for p in procs:
         p.start()

@@ -22,7 +22,8 @@ def test_sp_block_world_size_one_equals_direct_calls(laga):
     from paper_2607_17644_b200 import sp
     sh = LagaShape(S=640, h=4)
     q, c_kv, k_pe, w, dout = (t.cuda() for t in make_inputs(sh, 97))
-    dist.init_process_group(backend="nccl", init_method="tcp://127.0.0.1:29651", rank=0, world_size=1)
+    from conftest import free_port
+    dist.init_process_group(backend="nccl", init_method=f"tcp://127.0.0.1:{free_port()}", rank=0, world_size=1)
     try:
         compute = sp.CudaCompute()
         out_local, ctx = sp.sp_forward(q, c_kv, k_pe, w, sh.h, compute)
