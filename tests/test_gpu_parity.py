@@ -8,7 +8,8 @@ import pytest
 import torch
 
 from paper_2607_17644_b200.inputs import CONFIGS, CONFIG_SEEDS, LagaShape, make_inputs
-from parity import (TOL_LSE, TOL_LSE_UNROUNDED, check_dw, check_row_bands, check_tensor, f64, max_abs)
+from parity import (TOL_LSE, TOL_LSE_UNROUNDED, check_dw, check_row_bands, check_tensor, f64, max_abs, rel_l2,
+                    scaled_max_abs)
 
 pytestmark = pytest.mark.gpu
 
@@ -22,13 +23,24 @@ def laga():
     return _laga
 
 
+def nan_like(shape, dtype):
+    return torch.full(shape, float("nan"), dtype=dtype, device="cuda")
+
+
 def run_gpu(laga, tensors, causal, backward=True):
+    """Every output starts as NaN: a tile the kernels fail to write cannot pass on stale memory."""
     q, c_kv, k_pe, w, dout = (t.cuda() if t is not None else None for t in tensors)
-    out, lse, ws = laga.fwd(q, c_kv, k_pe, w, causal=causal)
+    S, h = q.shape[0], q.shape[1]
+    out, lse, ws = laga.fwd(q, c_kv, k_pe, w, causal=causal, out=nan_like((S, h, 128), torch.bfloat16),
+                            lse=nan_like((S, h), torch.float32))
     laga.check_status(ws, where="laga_fwd")
     res = {"out": out, "lse": lse}
     if backward:
-        dq, dc_kv, dk_pe, dw, ws2 = laga.bwd(q, c_kv, k_pe, w, out, lse, dout, causal=causal)
+        dq, dc_kv, dk_pe, dw, ws2 = laga.bwd(q, c_kv, k_pe, w, out, lse, dout, causal=causal,
+                                             dq=nan_like(tuple(q.shape), torch.bfloat16),
+                                             dc_kv=nan_like(tuple(c_kv.shape), torch.bfloat16),
+                                             dk_pe=nan_like(tuple(k_pe.shape), torch.bfloat16),
+                                             dw_kv_b=nan_like(tuple(w.shape), torch.float32))
         laga.check_status(ws2, where="laga_bwd")
         res.update(dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw=dw)
     return {k: v.cpu() for k, v in res.items()}
@@ -174,6 +186,60 @@ def test_benchmark_configs_sampled(laga, oracle, name):
     b = float((f64(c_kv) * f64(g["dc_kv"])).sum())
     scale = float(f64(w).norm() * f64(g["dw"]).norm())
     assert abs(a - b) <= 1e-3 * scale, (a, b, scale)
+
+
+def test_headline_config_every_element(laga, oracle):
+    """The headline configuration (c2: S=16384, h_local=16, causal, forward+backward) at full size, in the
+    launch configuration bench.py times, against the COMPLETE oracle result in both of its K/V rounding
+    modes: every element of out, lse, dq, dc_kv, dk_pe and dw.  The oracle runs head by head (a head's out,
+    lse, dq and dW columns depend on that head alone; dc_kv and dk_pe are sums over the heads), which
+    bounds its memory; about a minute per mode on 16 host cores.  Raw and scaled errors are printed, and
+    written as JSON to the file LAGA_PARITY_REPORT names when that variable is set."""
+    import json
+    import os
+    sh = CONFIGS["c2"]
+    tensors = make_inputs(sh, CONFIG_SEEDS["c2"])
+    q, c_kv, k_pe, w, dout = tensors
+    g = run_gpu(laga, tensors, True)
+    report = {}
+    for rounded in (True, False):
+        ref = {"out": torch.empty(sh.S, sh.h, sh.d_v, dtype=torch.float64),
+               "lse": torch.empty(sh.S, sh.h, dtype=torch.float64),
+               "dq": torch.empty(sh.S, sh.h, sh.d_qk, dtype=torch.float64),
+               "dw": torch.empty(sh.d_c, sh.n_cols, dtype=torch.float64),
+               "dc_kv": torch.zeros(sh.S, sh.d_c, dtype=torch.float64),
+               "dk_pe": torch.zeros(sh.S, sh.d_rope, dtype=torch.float64)}
+        for i in range(sh.h):
+            cols = slice(i * 256, (i + 1) * 256)
+            r = oracle.bwd(q[:, i:i + 1].contiguous(), c_kv, k_pe, w[:, cols].contiguous(),
+                           dout[:, i:i + 1].contiguous(), sh.d_v, sh.softmax_scale, causal=True,
+                           kv_round_bf16=rounded, return_fwd=True)
+            ref["out"][:, i:i + 1], ref["lse"][:, i:i + 1], ref["dq"][:, i:i + 1] = r["out"], r["lse"], r["dq"]
+            ref["dw"][:, cols] = r["dw"]
+            ref["dc_kv"] += r["dc_kv"]
+            ref["dk_pe"] += r["dk_pe"]
+        mode = "kv_round_bf16" if rounded else "unrounded"
+        stats = {}
+        for name in ("out", "dq", "dc_kv", "dk_pe", "dw"):
+            stats[name] = {"max_abs": max_abs(g[name], ref[name]), "rel_l2": rel_l2(g[name], ref[name]),
+                           "scaled_max_abs": scaled_max_abs(g[name], ref[name]),
+                           "ref_rms": float(ref[name].pow(2).mean().sqrt()), "ref_max": float(ref[name].abs().max())}
+        stats["lse"] = {"max_abs": max_abs(g["lse"], ref["lse"])}
+        report[mode] = stats
+        print(f"[c2 full parity, oracle {mode}] " + json.dumps(stats))
+        check_tensor("out", g["out"], ref["out"])
+        assert stats["out"]["max_abs"] <= 2e-2 and stats["dq"]["max_abs"] <= 2e-2     # the plain bound binds here
+        assert stats["lse"]["max_abs"] <= (TOL_LSE if rounded else TOL_LSE_UNROUNDED)
+        check_tensor("dq", g["dq"], ref["dq"])
+        check_tensor("dc_kv", g["dc_kv"], ref["dc_kv"])
+        check_tensor("dk_pe", g["dk_pe"], ref["dk_pe"])
+        check_dw(g["dw"], ref["dw"])
+        for name in ("out", "dq", "dc_kv", "dk_pe"):          # query-row bands, and key-position bands
+            check_row_bands(name, g[name], ref[name])
+    path = os.environ.get("LAGA_PARITY_REPORT")
+    if path:
+        with open(path, "w") as f:
+            json.dump(report, f, indent=1)
 
 
 @pytest.mark.parametrize("sp", [4, 1])
