@@ -36,11 +36,12 @@ METRIC = "laga_attention_block_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 WORKLOAD = "c2"
 KERNELS_PER_STEP = 9   # fwd: up_project, attn_fwd; bwd: up_project, delta, dkv, dq, dkpe_convert, dckv, dw
-# DRAM bytes (read + write) per launch of attn_bwd_dkv, from the ncu capture summarised in
-# profiles/ncu_full_c3_sp8_kernels.txt (S=8192, h=16: 155.5 MB read + 43.3 MB written), expressed per
-# (token, head).  The kernel's traffic is its inputs and outputs once each (K/V, Q and dO tiles are
-# re-read from L2, not DRAM), so it grows in proportion to S*h and is scaled that way to the workload.
-DKV_DRAM_BYTES_PER_TOKEN_HEAD = (155.500800e6 + 43.290624e6) / (8192 * 16)
+# DRAM bytes (read + write) of ONE launch of attn_bwd_dkv at the headline workload (c2), from the ncu
+# capture summarised in profiles/ncu_dram_c2_attn_bwd_dkv.txt.  For other workloads the figure is scaled
+# by S*h (the kernel reads its inputs and writes its outputs once; tiles are re-read from L2, not DRAM)
+# and flagged as scaled.
+DKV_DRAM_BYTES_C2 = None          # filled in from the capture; None until one exists
+DKV_DRAM_C2_TOKEN_HEADS = 16384 * 16
 
 
 def flops(sh: LagaShape):
@@ -49,7 +50,10 @@ def flops(sh: LagaShape):
     f_attn_fwd = 2 * sh.h * pairs * (sh.d_qk + sh.d_v)
     f_up = 2 * sh.S * sh.d_c * sh.n_cols
     f_attn_bwd = 2 * sh.h * pairs * (3 * sh.d_qk + 2 * sh.d_v)
-    return {"fwd": f_attn_fwd + f_up, "bwd": f_attn_bwd + 2 * f_up, "attn_bwd_dkv": 2 * sh.h * pairs * (2 * sh.d_qk + 2 * sh.d_v)}
+    return {"fwd": f_attn_fwd + f_up, "bwd": f_attn_bwd + 2 * f_up, "attn_fwd": f_attn_fwd, "attn_bwd": f_attn_bwd,
+            # executed by each backward kernel (S and dP are recomputed in both): dkv = S^T, dP^T, dV, dK; dq = S, dP, dQ
+            "attn_bwd_dkv": 2 * sh.h * pairs * (2 * sh.d_qk + 2 * sh.d_v),
+            "attn_bwd_dq": 2 * sh.h * pairs * (2 * sh.d_qk + sh.d_v)}
 
 
 def activation_memory(sh: LagaShape, ws_fwd: int, ws_bwd: int, allocated_in_step: int):
@@ -66,7 +70,7 @@ def activation_memory(sh: LagaShape, ws_fwd: int, ws_bwd: int, allocated_in_step
 
 def compare_eager(sh: LagaShape, inputs, cuda_results, laga_ms: float, laga_peak_bytes: dict, reps: int = 2):
     """Time the explicit (B1) and absorbed (B2) forms of the same block written in eager PyTorch ops
-    with the full S x S score matrix, as the paper's memory study ran them (Section 6, memory table),
+    with the full S x S score matrix, as the paper's memory study ran them (Section 4, activation-memory table),
     and record what each keeps alive beyond its inputs.  Library kernels, comparison only."""
     from paper_2607_17644_b200 import eager_forms
     q, c_kv, k_pe, w, dout = inputs
@@ -107,7 +111,10 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while a region runs.  The period
+    is 20 ms; the timed region of the default run lasts about 0.1 s, so this is a coarse record (and
+    nvidia-smi's clock reading lags the power controller): the clock the kernels really ran at is taken
+    inside the kernels themselves (laga_query_kernel_clocks) and reported beside it."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
@@ -120,7 +127,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -139,7 +146,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, sm_max, reasons = [], [], set()
+        sm, sm_max, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
@@ -148,25 +155,40 @@ class ClockSampler:
             try:
                 sm.append(float(parts[0]))
                 sm_max.append(float(parts[1]))
+                power.append(float(parts[2]))
             except ValueError:
                 continue
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(sm_max) if sm_max else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "power_w_max": max(power) if power else None, "reasons": sorted(reasons)}
 
 
-def dist_setup(n_gpus: int):
+def self_launch(n_gpus: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script under torch.distributed.run
+    on one node (127.0.0.1, a free port) and hand back its exit code.  Rank 0 of that job prints the line."""
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.run(cmd).returncode
+
+
+def dist_setup(n_gpus: int, backend: str = "nccl"):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if backend == "nccl":
+        torch.cuda.set_device(local_rank if world > 1 else 0)
     if world > 1:
         import torch.distributed as dist
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
-    else:
-        torch.cuda.set_device(0)
+        if backend == "nccl":
+            dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group(backend=backend)
     if world != n_gpus and rank == 0:
         print(f"[bench] note: --gpus {n_gpus} but WORLD_SIZE={world}; using WORLD_SIZE", file=sys.stderr)
     return world, rank, local_rank
@@ -186,6 +208,22 @@ def max_over_ranks(value: float, world: int, device: str = "cuda") -> float:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
     return value
+
+
+def run_dry(args):
+    """The launch and reduction plumbing of the N-rank run with no GPU work (gloo): every rank contributes a
+    made-up step time and rank 0 prints the line's skeleton.  Used by the CPU test of the launcher."""
+    world, rank, _ = dist_setup(args.gpus, backend="gloo")
+    fake_ms = 10.0 + 5.0 * rank
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    total_ms = max_over_ranks(fake_ms, world, device="cpu")
+    if rank == 0:
+        print(json.dumps({"impl": "dry-run", "n_gpus": world, "ms_per_step": total_ms, "scaling": "weak"}), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
 
 
 def run_cuda(args):
@@ -215,24 +253,28 @@ def run_cuda(args):
     def fwd_only():
         laga.fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_f)
 
+    def step_kv_saved():   # variant: the backward reuses the forward's K_nope/V from a workspace both calls share
+        laga.fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_b)
+        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw_kv_b=dw, workspace=ws_b,
+                 flags=laga.FLAG_KV_SAVED)
+
     for _ in range(max(args.warmup, 3)):
         step()
     laga.check_status(ws_f, where="warm-up laga_fwd")
     laga.check_status(ws_b, where="warm-up laga_bwd")
 
-    # ---- timed region: exactly K steps, device-timed, events around the dominant kernel -------------
+    # ---- timed region: exactly K steps, device-timed, events around the attention kernels and delta ----
     K = args.steps
     dom = "attn_bwd_dkv"
-    k_starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
-    k_stops = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
-    for e in k_starts + k_stops:
-        e.record()
-    laga.profile_kernel(dom, k_starts, k_stops)
-    d_starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]     # the one HBM-bound kernel of weight: delta
-    d_stops = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
-    for e in d_starts + d_stops:
-        e.record()
-    laga.profile_kernel("bwd_delta", d_starts, d_stops)
+    timed = ("attn_bwd_dkv", "attn_bwd_dq", "attn_fwd", "bwd_delta")
+    kernel_events = {}
+    for name in timed:
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+        for e in starts + stops:
+            e.record()
+        laga.profile_kernel(name, starts, stops)
+        kernel_events[name] = (starts, stops)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -244,14 +286,18 @@ def run_cuda(args):
     ev1.record()
     barrier(world)
     clocks = sampler.stop()
-    laga.profile_kernel(dom)
-    laga.profile_kernel("bwd_delta")
-    delta_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(d_starts, d_stops))
+    for name in timed:
+        laga.profile_kernel(name)
+    kernel_ms = {name: statistics.mean(a.elapsed_time(b) for a, b in zip(*kernel_events[name])) for name in timed}
+    # the SM clock the attention kernels of the LAST timed step ran at, measured inside the kernels
+    in_kernel = {**laga.query_kernel_clocks(ws_f), **laga.query_kernel_clocks(ws_b)}
+    clocks["in_kernel_sm_mhz"] = {k: round(v[0], 1) for k, v in in_kernel.items()}
+    delta_ms = kernel_ms["bwd_delta"]
     s_pad = (sh.S + 127) // 128 * 128
-    delta_bytes = 2 * sh.S * sh.h * sh.d_v * 2 + sh.S * sh.h * 4 + 2 * s_pad * sh.h * 4   # O, dO, LSE in; two statistics out
+    delta_bytes = 2 * sh.S * sh.h * sh.d_v * 2 + sh.S * sh.h * 4 + 2 * s_pad * sh.h * 4 + sh.S * sh.d_rope * 4   # O, dO, LSE in; two statistics out; rope-gradient accumulator cleared
     total_ms = max_over_ranks(ev0.elapsed_time(ev1), world)
     ms_per_step = total_ms / K
-    dom_ms = statistics.mean(a.elapsed_time(b) for a, b in zip(k_starts, k_stops))
+    dom_ms = kernel_ms[dom]
     laga.check_status(ws_f, where="timed laga_fwd")
     laga.check_status(ws_b, where="timed laga_bwd")
 
@@ -265,6 +311,19 @@ def run_cuda(args):
     barrier(world)
     fwd_ms = max_over_ranks(f0.elapsed_time(f1), world) / K
     peak_act = torch.cuda.max_memory_allocated() - base_mem   # nothing is allocated inside a step
+
+    # ---- variant: LAGA_FLAG_KV_SAVED (reported, not the headline) ------------------------------------
+    for _ in range(2):
+        step_kv_saved()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    s0.record()
+    for _ in range(K):
+        step_kv_saved()
+    s1.record()
+    barrier(world)
+    kv_saved_ms = max_over_ranks(s0.elapsed_time(s1), world) / K
+    laga.check_status(ws_b, where="kv-saved step")
 
     # ---- end to end: pinned host buffers in, results out, every step ------------------------------
     host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (out, lse, dq, dc_kv, dk_pe, dw)]
@@ -349,6 +408,16 @@ def run_cuda(args):
     peaks = measured_peaks()
     total_flops = fl["fwd"] + fl["bwd"]
     value = world * total_flops / (ms_per_step * 1e-3) / 1e12
+    dom_tflops = fl[dom] / (dom_ms * 1e-3) / 1e12
+    bwd_attn_ms = kernel_ms["attn_bwd_dkv"] + kernel_ms["attn_bwd_dq"]
+    token_heads = sh.S * sh.h
+    if DKV_DRAM_BYTES_C2 is None:
+        traffic, traffic_note = None, "no ncu capture of this kernel yet"
+    elif token_heads == DKV_DRAM_C2_TOKEN_HEADS:
+        traffic, traffic_note = DKV_DRAM_BYTES_C2, "ncu dram read+write of one launch at this workload (profiles/ncu_dram_c2_attn_bwd_dkv.txt)"
+    else:
+        traffic = DKV_DRAM_BYTES_C2 * token_heads / DKV_DRAM_C2_TOKEN_HEADS
+        traffic_note = "ncu dram read+write of one launch at S=16384,h=16, scaled by S*h"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -371,13 +440,29 @@ def run_cuda(args):
                 "serial_ms_per_step": e2e_serial_ms,
                 "serial_value": world * total_flops / (e2e_serial_ms * 1e-3) / 1e12},
         "gpu_launches": KERNELS_PER_STEP * K,
-        "roofline": {"bound": "tensor", "kernel": dom, "achieved": fl["attn_bwd_dkv"] / (dom_ms * 1e-3) / 1e12,
-                     "peak": peaks["bf16_tflops_sustained"], "unit": UNIT,
-                     "frac": fl["attn_bwd_dkv"] / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                     "peak_source": peaks["source"] + " sustained cuBLAS bf16 (kernel timed inside a long step)",
-                     "kernel_ms": dom_ms, "flops_per_launch": fl["attn_bwd_dkv"],
-                     "traffic": DKV_DRAM_BYTES_PER_TOKEN_HEAD * sh.S * sh.h,
-                     "traffic_note": "bytes per launch, ncu dram read+write at S=8192,h=16 scaled by S*h"},
+        # Dominant kernel.  `achieved` = FLOPs this kernel executes per launch (S^T, dP^T, dV, dK: 1280 per causal
+        # pair and head) / its mean CUDA-event time over the K timed launches.  `peak` is the measured cuBLAS bf16
+        # BURST figure; the same kernel against the sustained figure, the clock it ran at (stamped inside the
+        # kernel) and the whole backward attention on algorithmic FLOPs are given beside it.
+        "roofline": {"bound": "tensor", "kernel": dom, "achieved": dom_tflops, "peak": peaks["bf16_tflops"], "unit": UNIT,
+                     "frac": dom_tflops / peaks["bf16_tflops"],
+                     "frac_of_sustained_peak": dom_tflops / peaks["bf16_tflops_sustained"],
+                     "peak_source": peaks["source"] + " cuBLAS bf16, burst (sustained: "
+                                    f"{peaks['bf16_tflops_sustained']})",
+                     "kernel_ms": dom_ms, "flops_per_launch": fl[dom],
+                     "sm_mhz_in_kernel": clocks["in_kernel_sm_mhz"].get(dom),
+                     "kernel_ms_x_sm_mhz": dom_ms * clocks["in_kernel_sm_mhz"].get(dom, 0.0),
+                     "traffic": traffic, "traffic_note": traffic_note,
+                     "other_kernels": {
+                         "attn_bwd_dq": {"kernel_ms": kernel_ms["attn_bwd_dq"], "executed_tflops": fl["attn_bwd_dq"] / (kernel_ms["attn_bwd_dq"] * 1e-3) / 1e12},
+                         "attn_fwd": {"kernel_ms": kernel_ms["attn_fwd"], "executed_tflops": fl["attn_fwd"] / (kernel_ms["attn_fwd"] * 1e-3) / 1e12}},
+                     "backward_attention": {"ms": bwd_attn_ms, "algorithmic_flops": fl["attn_bwd"],
+                                            "algorithmic_tflops": fl["attn_bwd"] / (bwd_attn_ms * 1e-3) / 1e12,
+                                            "frac_of_burst_peak": fl["attn_bwd"] / (bwd_attn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                            "note": "dkv + dq kernels; S and dP are recomputed in both (2304 executed vs 1664 algorithmic FLOP per pair)"}},
+        "variants": {"kv_saved": {"ms_per_step": kv_saved_ms, "value": world * total_flops / (kv_saved_ms * 1e-3) / 1e12,
+                                  "note": "LAGA_FLAG_KV_SAVED: the backward reads the forward's K_nope/V from a shared "
+                                          "workspace instead of recomputing step 4 (one launch less); not the headline"}},
     }
     if args.compare_eager and world == 1:
         del in_dev, out_dev, host_outs
@@ -388,7 +473,11 @@ def run_cuda(args):
                                          "peak": peaks["hbm_gbs"], "frac": delta_bytes / (delta_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                          "share_of_step": delta_ms / ms_per_step}}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(sample_tokens=args.cpu_sample_tokens)
+        step()                                                    # the results the parity figures are taken from
+        torch.cuda.synchronize()
+        gpu_results = {"out": out, "lse": lse, "dq": dq, "dw": dw}
+        line["cpu_baseline"], line["parity"] = cpu_baseline(args.cpu_sample_tokens, args.workload, gpu_results,
+                                                            lambda t: head0_shard_gradients(laga, sh, t, dev))
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -396,28 +485,73 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
-def oracle_sample(sample_tokens: int):
-    """The bounded sample both CPU legs run: head 0 of the c2 shard restricted to its first
+def head0_shard_gradients(laga, sh, tensors, dev):
+    """dc_kv and dk_pe are sums over the shard's heads, so head 0's share is not visible in the full run:
+    run the CUDA path once more on the one-head shard the oracle sample is (outside any timed region)."""
+    q, c_kv, k_pe, w, dout = (t.to(dev) for t in tensors)
+    out, lse, ws = laga.fwd(q, c_kv, k_pe, w)
+    _, dc_kv, dk_pe, _, ws2 = laga.bwd(q, c_kv, k_pe, w, out, lse, dout)
+    laga.check_status(ws, where="parity laga_fwd")
+    laga.check_status(ws2, where="parity laga_bwd")
+    return {"dc_kv": dc_kv, "dk_pe": dk_pe}
+
+
+def oracle_sample(sample_tokens: int, workload: str = WORKLOAD):
+    """The bounded sample both CPU legs run: head 0 of the workload's shard restricted to its first
     `sample_tokens` tokens (a causal prefix is a self-contained sub-problem of the same workload)."""
-    sh = CONFIGS[WORKLOAD]
-    q, c_kv, k_pe, w, dout = make_inputs(sh, CONFIG_SEEDS[WORKLOAD])
-    n = sample_tokens
+    sh = CONFIGS[workload]
+    q, c_kv, k_pe, w, dout = make_inputs(sh, CONFIG_SEEDS[workload])
+    n = min(sample_tokens, sh.S)
     sub = LagaShape(S=n, h=1)
     tensors = (q[:n, :1].contiguous(), c_kv[:n].contiguous(), k_pe[:n].contiguous(), w[:, :256].contiguous(),
                dout[:n, :1].contiguous())
     return sub, tensors
 
 
-def cpu_baseline(sample_tokens: int):
+def error_metrics(g, r):
+    g, r = g.detach().to("cpu", torch.float64), r.to(torch.float64)
+    diff = (g - r).abs()
+    rms = float(r.pow(2).mean().sqrt())
+    return {"max_abs": float(diff.max()), "rel_l2": float((g - r).norm() / r.norm().clamp_min(1e-300)),
+            "scaled_max_abs": float(diff.max()) / max(1.0, rms), "ref_rms": rms, "ref_max": float(r.abs().max())}
+
+
+def cpu_baseline(sample_tokens: int, workload: str = WORKLOAD, gpu_results=None, one_head_gradients=None):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload.  When the GPU
+    results of the same workload are passed in, the oracle's numbers double as the parity record: raw
+    max-abs, relative L2 and max-abs scaled by the reference's rms for every tensor, against the plain oracle
+    (the timed call) and against the oracle that rounds K_nope/V to bf16 (a second, untimed call).  out, lse
+    and dq are the head-0 rows of the timed configuration's own results; dc_kv and dk_pe (sums over heads)
+    come from one more run of the CUDA path on the one-head sample."""
     import oracle
-    sub, (q, c_kv, k_pe, w, dout) = oracle_sample(sample_tokens)
+    sub, tensors = oracle_sample(sample_tokens, workload)
+    q, c_kv, k_pe, w, dout = tensors
     fl = flops(sub)
     t0 = time.perf_counter()
-    oracle.bwd(q, c_kv, k_pe, w, dout, sub.d_v, sub.softmax_scale, causal=True)   # computes forward and backward
+    ref = oracle.bwd(q, c_kv, k_pe, w, dout, sub.d_v, sub.softmax_scale, causal=True, return_fwd=True)   # forward and backward
     dt = time.perf_counter() - t0
-    return {"value": (fl["fwd"] + fl["bwd"]) / dt / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "seconds": dt, "sample": f"head 0, first {sample_tokens} tokens of the c2 shard (causal prefix), "
+    base = {"value": (fl["fwd"] + fl["bwd"]) / dt / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "seconds": dt, "sample": f"head 0, first {sub.S} tokens of the {workload} shard (causal prefix), "
                                       "forward+backward in fp64, one pass"}
+    if gpu_results is None:
+        return base, None
+    n, full = sub.S, sub.S == CONFIGS[workload].S
+    shard = one_head_gradients(tensors)
+    # (dW sums over every token: the full run's head-0 columns match only a full-length sample)
+    got = {"out": gpu_results["out"][:n, :1], "dq": gpu_results["dq"][:n, :1], "dc_kv": shard["dc_kv"],
+           "dk_pe": shard["dk_pe"]}
+    if full:
+        got["dw"] = gpu_results["dw"][:, :256]
+    refs = {"unrounded": ref,
+            "kv_round_bf16": oracle.bwd(q, c_kv, k_pe, w, dout, sub.d_v, sub.softmax_scale, causal=True,
+                                        kv_round_bf16=True, return_fwd=True)}
+    parity = {"sample": base["sample"], "tolerances": {"max_abs": 2e-2, "rel_l2": 5e-3, "lse_vs_kv_round_bf16": 1e-3,
+                                                       "note": "dw, and the early-key rows of dc_kv / dk_pe, are bound on "
+                                                               "the scaled max-abs (their entries reach 5..35)"}}
+    for mode, r in refs.items():
+        parity[mode] = {name: error_metrics(t, r[name]) for name, t in got.items()}
+        parity[mode]["lse"] = {"max_abs": float((gpu_results["lse"][:n, :1].detach().to("cpu", torch.float64) - r["lse"]).abs().max())}
+    return base, parity
 
 
 def run_reference(args):
@@ -460,7 +594,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
-    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing and parity leg")
     ap.add_argument("--workload", choices=sorted(CONFIGS), default=WORKLOAD,
                     help="benchmark configuration (default c2, the headline; others are for profiling)")
     ap.add_argument("--compare-eager", action="store_true",
@@ -469,8 +603,15 @@ def main():
                     help="tokens of head 0 the cpu_baseline leg runs (16384 = the whole head: ~10 s on 16 cores)")
     ap.add_argument("--ref-sample-tokens", type=int, default=2048,
                     help="tokens of head 0 per step in --impl reference (2048: well under a second per step)")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="exercise the N-rank launch and the max-over-ranks reduction on the CPU (gloo), no GPU work")
     args = ap.parse_args()
-    if args.impl == "reference":
+    # `python bench.py --gpus N` outside a launcher: start the N ranks ourselves (one per GPU)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "cuda":
+        raise SystemExit(self_launch(args.gpus))
+    if args.dry_run:
+        run_dry(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         if not torch.cuda.is_available():

@@ -23,12 +23,18 @@
  *     stream) and return without synchronising, except laga_query_status.
  *   - Return value: LAGA_OK (0) or a negative LAGA_ERR_* code.  Argument errors are detected before
  *     anything is enqueued.  Nothing throws, aborts or traps.
+ *   - Work runs on the CURRENT device (cudaSetDevice): every data pointer must be device memory of that
+ *     device (or managed memory); a pointer that belongs to another device, or to the host, returns
+ *     LAGA_ERR_INVALID_ARG before anything is enqueued.
+ *   - The entry points may be called from several host threads at once (the library's per-device and
+ *     tensor-map caches are locked); what the callers must keep apart is the memory: two calls that may
+ *     overlap on the GPU must not share a workspace or an output.
  *   - This build is tuned for the DeepSeek-V3 head geometry: d_c = 512, d_nope = 128, d_rope = 64,
  *     d_v = 128.  Other values return LAGA_ERR_UNSUPPORTED.  S >= 1 and h >= 1 are arbitrary (S need
  *     not be a multiple of any tile).  Batch is a caller loop.
  *   - `workspace` is caller-provided scratch of at least laga_*_workspace_bytes(...) bytes, 1024-byte
- *     aligned.  Its first word is the launch status word read by laga_query_status.  Two calls that
- *     may overlap on the GPU must not share a workspace.
+ *     aligned.  Its first 1024 bytes are the launch status slot (the status word laga_query_status reads,
+ *     the work counters of the persistent kernels, their clock probes); every call clears what it needs.
  */
 #ifndef LAGA_H_
 #define LAGA_H_
@@ -45,6 +51,8 @@ extern "C" {
 #define LAGA_ERR_WORKSPACE_TOO_SMALL (-3)
 #define LAGA_ERR_CUDA (-4)                /* a CUDA runtime/driver call or a launch failed          */
 #define LAGA_ERR_DEVICE_TIMEOUT (-5)      /* only from laga_query_status: a bounded device wait ran out */
+#define LAGA_ERR_DEVICE_CHECK (-6)        /* only from laga_query_status: a device-side self-check failed
+                                             (the kernel recorded where, skipped the access and returned)   */
 
 #define LAGA_FLAG_ACCUM_DW 1u             /* laga_bwd: add into dw_kv_b instead of overwriting it   */
 #define LAGA_FLAG_DETERMINISTIC 2u        /* laga_bwd: bitwise-repeatable dk_pe and dw_kv_b (see there) */
@@ -135,7 +143,10 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
  *     Every GPU on which the library is loaded carries these 16 MiB (+1 KiB) until the process exits.
  *   - The call allocates and frees nothing (no cudaMalloc/cudaFree, no allocating library routine).
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- *     that device current) and caches it; make that first call outside any stream capture.
+ *     that device current) and caches it; make that first call outside any stream capture.  Under CUDA's
+ *     lazy module loading the first library call on a device also loads the library's device code, which
+ *     is when the array itself comes into being (an implicit device allocation and synchronisation made
+ *     by the CUDA runtime, once): keep that first call in the initialisation phase of the program.
  *   - All calls on a device share the one array, and it keeps the previous call's contents.  The
  *     call itself clears the status word and overwrites the KV rows it uses, so back-to-back calls
  *     on ONE stream are safe; calls that can overlap on the GPU (different streams, no ordering
@@ -165,7 +176,7 @@ int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stre
  * caller with timing enabled) that the library records on the launch stream immediately before and
  * after every launch of one kernel, cycling through the pairs launch after launch; n_pairs = 0 stops
  * it.  The caller reads the times (cudaEventElapsedTime) after synchronising, and keeps the events
- * alive while registered.  Not thread-safe; intended for benchmarks.  The paper has no counterpart.
+ * alive while registered.  Intended for benchmarks.  The paper has no counterpart.
  */
 #define LAGA_KERNEL_UP_PROJECT 0    /* step 4 GEMM (also the recomputation in laga_bwd)        */
 #define LAGA_KERNEL_ATTN_FWD 1      /* step 5 forward attention                               */
@@ -179,8 +190,21 @@ int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stre
 int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs);
 
 /*
+ * Measurement aid.  The three attention kernels stamp the SM cycle counter and the nanosecond timer when
+ * their first CTA starts and when it ends (they are persistent: that CTA lives as long as the kernel) into
+ * the workspace's status slot.  This call synchronises `stream`, reads the stamps the last call on
+ * `workspace` left and fills two arrays of LAGA_KERNEL_COUNT doubles: the SM clock in MHz the kernel
+ * actually ran at (cycles / time) and its duration in milliseconds; entries of kernels without stamps
+ * (the GEMMs and the small kernels, or an attention kernel that has not run on this workspace) are 0.
+ * Under a power cap this is the clock the tensor pipe really saw, which a coarse host-side sampler
+ * cannot resolve for millisecond kernels.  The paper has no counterpart.
+ */
+int laga_query_kernel_clocks(const void* workspace, void* stream, double* sm_mhz, double* kernel_ms);
+
+/*
  * Synchronises `stream`, reads the status word at the start of `workspace` (or a `status_word`
- * given to a step entry point) and returns LAGA_OK, LAGA_ERR_DEVICE_TIMEOUT or LAGA_ERR_CUDA.
+ * given to a step entry point) and returns LAGA_OK, LAGA_ERR_DEVICE_TIMEOUT, LAGA_ERR_DEVICE_CHECK or
+ * LAGA_ERR_CUDA.
  * If `detail` is not NULL it receives the raw device word (which wait gave up).
  */
 int laga_query_status(const void* workspace, void* stream, unsigned* detail);

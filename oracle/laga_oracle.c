@@ -172,13 +172,6 @@ int laga_oracle_fwd_rows(const uint16_t* q, const uint16_t* c_kv, const uint16_t
     return fail ? -2 : 0;
 }
 
-int laga_oracle_fwd(const uint16_t* q, const uint16_t* c_kv, const uint16_t* k_pe,
-                    const uint16_t* w_kv_b, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
-                    double softmax_scale, int causal, int kv_round_bf16, double* out, double* lse) {
-    return laga_oracle_fwd_rows(q, c_kv, k_pe, w_kv_b, S, h, d_c, d_nope, d_rope, d_v, softmax_scale,
-                                causal, kv_round_bf16, NULL, 0, out, lse, NULL, NULL);
-}
-
 /* Backward restricted to a list of query rows: dq [n_rows][h][d_n+d_r] (a row of dQ depends on that
  * query row only), plus the forward values out [n_rows][h][d_v] and lse [n_rows][h] it used. */
 int laga_oracle_bwd_rows(const uint16_t* q, const uint16_t* c_kv, const uint16_t* k_pe,

@@ -24,6 +24,7 @@
 #pragma once
 #include "attn_fwd_sm100.cuh"
 #include "sm100_ptx.cuh"
+#include "work_sched.cuh"
 
 namespace laga {
 
@@ -42,7 +43,12 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gmem_sr
 __global__ void __launch_bounds__(256)
 bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
                  const float* __restrict__ lse, int S, int h, int S_pad, float* __restrict__ stat_l2,
-                 float* __restrict__ stat_delta) {
+                 float* __restrict__ stat_delta, float4* __restrict__ zero_begin, size_t zero_count) {
+    // Also clears the fp32 buffer the dK/dV kernel accumulates the rope-column key gradients into
+    // (zero_count float4 elements): one launch less than a separate memset.
+    for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < zero_count;
+         z += static_cast<size_t>(gridDim.x) * blockDim.x)
+        zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
     const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;   // (row, head) pair
     const int sub = threadIdx.x & 7;
     const bool live = item < static_cast<long long>(S_pad) * h;
@@ -97,7 +103,6 @@ bwd_dkpe_reduce_kernel(const float* __restrict__ dk_rope, int S, int h, __nv_bfl
 }
 
 constexpr int kBwdThreads = 320;
-constexpr int kBwdStages = 3;
 
 // ================================================================================================
 // dK / dV kernel
@@ -108,243 +113,324 @@ struct AttnBwdDkvArgs {
     const float* stat_l2;      // [h][S_pad]
     const float* stat_delta;   // [h][S_pad]
     __nv_bfloat16* dkv;        // [S, h*256]: per head dK_nope (128) then dV (128)
-    float* dkpe_acc;           // [S][64] fp32, zeroed by the host; every head's CTA adds into it
+    float* dkpe_acc;           // [S][64] fp32, zero when the kernel starts; every head's CTA adds into it
     float* dk_rope_per_head;   // deterministic mode: [h][S][64] fp32 written per head (then summed in a fixed
                                // order by bwd_dkpe_reduce_kernel); nullptr selects the atomic path
     unsigned int* status;
+    WorkSchedule sched;        // items = (128-key tile, head); rank 0 = key tile 0 (every query attends to it)
+    ClockProbe* clock_probe;   // may be nullptr
 };
 
 struct AttnBwdDkvSmem {
-    static constexpr int kSlab128 = 128 * 128;                 // 128 rows x 128 B
-    static constexpr int kSlab64 = 64 * 128;                   // 64 rows x 128 B
-    static constexpr int kStage = 5 * kSlab64;                 // Q (3 slabs) + dO (2 slabs), 64 rows each
-    static constexpr int kK = 0;                               // 3 slabs of 128 rows
-    static constexpr int kV = kK + 3 * kSlab128;               // 2 slabs of 128 rows
-    static constexpr int kQdO = kV + 2 * kSlab128;             // kBwdStages stages
-    static constexpr int kStat = kQdO + kBwdStages * kStage;   // per stage: 64 l2 + 64 delta floats
-    static constexpr int kBar = kStat + kBwdStages * 512;
-    static constexpr int kTotalBytes = kBar + 256 + 1024;
+    static constexpr int kSlab = 128 * 128;                    // 128 rows x 128 B
+    static constexpr int kQStages = 2;
+    static constexpr int kK = 0;                               // 3 slabs: K_nope (2), rope band (1)
+    static constexpr int kV = kK + 3 * kSlab;                  // 2 slabs
+    static constexpr int kQ = kV + 2 * kSlab;                  // kQStages x 3 slabs
+    static constexpr int kDo = kQ + kQStages * 3 * kSlab;      // 1 stage x 2 slabs
+    static constexpr int kStat = kDo + 2 * kSlab;              // per Q stage: 128 l2 + 128 delta floats
+    static constexpr int kBar = kStat + kQStages * 1024;
+    static constexpr int kTotalBytes = kBar + 512;
 };
+static_assert(AttnBwdDkvSmem::kTotalBytes <= 232448, "dkv kernel exceeds the 227 KB of shared memory per CTA");
 
+// Persistent: one CTA per SM takes (key tile, head) items from the work counter.  Per item the 128-key
+// K/V tile is stationary and the 128-row query tiles that attend to it stream through.  Every MMA is
+// 128 wide or wider: a 64-wide tcgen05.mma re-reads its 4 KB A tile for half the work and costs 48
+// clocks against 32, and this kernel is bound by the shared-memory port as much as by the tensor pipe.
+// TMEM: X (128 columns, fp32) holds S^T and then dP^T of the tile; Y (64 columns, packed bf16) holds
+// P^T and then dS^T, the A operands of the two accumulating MMAs; dK (192) and dV (128) fill the rest.
+//     ... dV(j-1) | S^T(j) | dK(j-1) | dP^T(j) | dV(j) | S^T(j+1) | ...
+// S^T(j) is issued as soon as the consumers have read dP^T(j-1) out of X, so the exponentials of tile j
+// run under dK(j-1) and dP^T(j); dS^T(j-1) is computed under dV(j-1) and S^T(j).  The two consumer
+// warpgroups split each tile's query columns (64 each).
 template <bool kCausal>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_do,
                           const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
                           const AttnBwdDkvArgs args) {
     using L = AttnBwdDkvSmem;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
     uint64_t* kv_full = bars + 0;
-    uint64_t* qdo_full = bars + 1;    // [3]
-    uint64_t* qdo_empty = bars + 4;   // [3]
-    uint64_t* st_full = bars + 7;     // [2]  S^T of the group's tile is in TMEM
-    uint64_t* st_read = bars + 9;     // [2]  the group has loaded it: the columns may take dP^T
-    uint64_t* p_full = bars + 11;     // [2]  P^T (bf16) is in TMEM
-    uint64_t* dp_full = bars + 13;    // [2]  dP^T is in TMEM
-    uint64_t* ds_full = bars + 15;    // [2]  dS^T (bf16) is in TMEM
-    uint64_t* acc_done = bars + 17;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
+    uint64_t* kv_empty = bars + 1;    // the item's last S^T / dP^T have read K and V
+    uint64_t* q_full = bars + 2;      // [2]  Q tile and its statistics
+    uint64_t* q_empty = bars + 4;     // [2]
+    uint64_t* do_full = bars + 6;
+    uint64_t* do_empty = bars + 7;
+    uint64_t* st_full = bars + 8;     // S^T of the tile is in X
+    uint64_t* st_read = bars + 9;     // both groups have loaded it: X may take dP^T
+    uint64_t* dp_full = bars + 10;    // dP^T is in X
+    uint64_t* dp_read = bars + 11;    // both groups have loaded it: X may take the next S^T
+    uint64_t* p_full = bars + 12;     // P^T (bf16) is in Y
+    uint64_t* dv_done = bars + 13;    // dV += P^T dO has read Y: it may take dS^T
+    uint64_t* ds_full = bars + 14;    // dS^T (bf16) is in Y
+    uint64_t* dk_done = bars + 15;    // dK += dS^T Q has read Y: it may take the next P^T
+    uint64_t* acc_full = bars + 16;   // the item's dK / dV are complete
+    uint64_t* acc_empty = bars + 17;  // both groups have drained them
+    ItemRing ring{bars + 18, bars + 20, reinterpret_cast<volatile int*>(bars + 22)};
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 23);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int k_tile = blockIdx.x, head = blockIdx.y;
-    const int t0 = k_tile * 128;
-    const int n_q64 = (args.S + 63) / 64;
-    const int j_begin = kCausal ? (t0 / 64) : 0;
-    const int n_iter = n_q64 - j_begin;              // >= 1 because t0 < S
+    const int n_q128 = (args.S + 127) / 128;
 
     if (threadIdx.x == 0) {
-        mbar_init(kv_full, 1);
-        for (int s = 0; s < kBwdStages; ++s) { mbar_init(&qdo_full[s], 1); mbar_init(&qdo_empty[s], 1); }
-        for (int g = 0; g < 2; ++g) {
-            mbar_init(&st_full[g], 1); mbar_init(&st_read[g], 128); mbar_init(&p_full[g], 128);
-            mbar_init(&dp_full[g], 1); mbar_init(&ds_full[g], 128);
-        }
-        mbar_init(acc_done, 1);
+        mbar_init(kv_full, 1); mbar_init(kv_empty, 1);
+        for (int s = 0; s < L::kQStages; ++s) { mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); }
+        mbar_init(do_full, 1); mbar_init(do_empty, 1);
+        mbar_init(st_full, 1); mbar_init(st_read, 256); mbar_init(dp_full, 1); mbar_init(dp_read, 256);
+        mbar_init(p_full, 256); mbar_init(dv_done, 1); mbar_init(ds_full, 256); mbar_init(dk_done, 1);
+        mbar_init(acc_full, 1); mbar_init(acc_empty, 256);
+        for (int s = 0; s < 2; ++s) { mbar_init(&ring.full[s], 1); mbar_init(&ring.empty[s], 9); }
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_do);
         tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
+        if ((smem_u32(smem) & 1023u) != 0u) {   // the swizzled operand slabs need a 1024-byte aligned base
+            abort_flag->value = 1;
+            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD0u);
+        }
     }
+    clock_probe_begin(args.clock_probe);
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    // columns: [0,64) group 0 scratch (S^T, then dP^T, then dS^T bf16) | [64,128) group 1 scratch |
-    //          [128,160) P^T group 0 | [160,192) P^T group 1 | [192,384) dK | [384,512) dV
-    const uint32_t tmem_pt = tmem_base + 128;
+    // columns: [0,128) X | [128,192) Y | [192,384) dK | [384,512) dV
+    const uint32_t tmem_y = tmem_base + 128;
     const uint32_t tmem_dk = tmem_base + 192;
     const uint32_t tmem_dv = tmem_base + 384;
+    auto item_geometry = [&](int item, int& t0, int& head, int& j_begin, int& n_iter) {
+        int k_tile;
+        decode_item(args.sched, item, k_tile, head);
+        t0 = k_tile * 128;
+        j_begin = kCausal ? k_tile : 0;
+        n_iter = n_q128 - j_begin;             // >= 1 because t0 < S
+    };
 
-    if (warp == 0) {
+    if (abort_flag->value != 0u) {
+        // misaligned shared memory: nothing was started, fall through to the common exit
+    } else if (warp == 0) {
         if (elect_one()) {
-            mbar_arrive_expect_tx(kv_full, 5 * L::kSlab128);
-            tma_load_2d(smem + L::kK, &tmap_kv, kv_full, head * 256, t0);
-            tma_load_2d(smem + L::kK + L::kSlab128, &tmap_kv, kv_full, head * 256 + 64, t0);
-            tma_load_2d(smem + L::kK + 2 * L::kSlab128, &tmap_kpe, kv_full, 0, t0);
-            tma_load_2d(smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, t0);
-            tma_load_2d(smem + L::kV + L::kSlab128, &tmap_kv, kv_full, head * 256 + 192, t0);
-            for (int j = 0; j < n_iter; ++j) {
-                const int st = j % kBwdStages;
-                if (!mbar_wait(&qdo_empty[st], ((j / kBwdStages) & 1) ^ 1, abort_flag, args.status, 0x40)) break;
-                const int q0 = (j_begin + j) * 64;
-                mbar_arrive_expect_tx(&qdo_full[st], L::kStage + 512);
-                uint8_t* sq = smem + L::kQdO + st * L::kStage;
-                uint8_t* sdo = sq + 3 * L::kSlab64;
-                for (int c = 0; c < 3; ++c)
-                    tma_load_2d(sq + c * L::kSlab64, &tmap_q, &qdo_full[st], head * 192 + c * 64, q0);
-                for (int c = 0; c < 2; ++c)
-                    tma_load_2d(sdo + c * L::kSlab64, &tmap_do, &qdo_full[st], head * 128 + c * 64, q0);
-                float* stat = reinterpret_cast<float*>(smem + L::kStat + st * 512);
-                bulk_load_1d(stat, args.stat_l2 + static_cast<size_t>(head) * args.S_pad + q0, 256, &qdo_full[st]);
-                bulk_load_1d(stat + 64, args.stat_delta + static_cast<size_t>(head) * args.S_pad + q0, 256,
-                             &qdo_full[st]);
+            uint32_t T = 0;                      // running tile count of this CTA: ring positions and phases
+            bool ok = true;
+            for (uint32_t n = 0; ok; ++n) {
+                const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
+                if (!ok || item < 0) break;
+                int t0, head, j_begin, n_iter;
+                item_geometry(item, t0, head, j_begin, n_iter);
+                ok = mbar_wait(kv_empty, (n & 1u) ^ 1u, abort_flag, args.status, 0x41);
+                if (!ok) break;
+                mbar_arrive_expect_tx(kv_full, 5 * L::kSlab);
+                tma_load_2d(smem + L::kK, &tmap_kv, kv_full, head * 256, t0);
+                tma_load_2d(smem + L::kK + L::kSlab, &tmap_kv, kv_full, head * 256 + 64, t0);
+                tma_load_2d(smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, t0);
+                tma_load_2d(smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, t0);
+                tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, kv_full, head * 256 + 192, t0);
+                for (int j = 0; j < n_iter; ++j, ++T) {
+                    const uint32_t sq = T % L::kQStages;
+                    const int q0 = (j_begin + j) * 128;
+                    ok = mbar_wait(&q_empty[sq], ((T / L::kQStages) & 1u) ^ 1u, abort_flag, args.status, 0x40);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&q_full[sq], 3 * L::kSlab + 1024);
+                    uint8_t* dst_q = smem + L::kQ + sq * 3 * L::kSlab;
+                    for (int c = 0; c < 3; ++c)
+                        tma_load_2d(dst_q + c * L::kSlab, &tmap_q, &q_full[sq], head * 192 + c * 64, q0);
+                    float* stat = reinterpret_cast<float*>(smem + L::kStat + sq * 1024);
+                    bulk_load_1d(stat, args.stat_l2 + static_cast<size_t>(head) * args.S_pad + q0, 512, &q_full[sq]);
+                    bulk_load_1d(stat + 128, args.stat_delta + static_cast<size_t>(head) * args.S_pad + q0, 512, &q_full[sq]);
+                    ok = mbar_wait(do_empty, (T & 1u) ^ 1u, abort_flag, args.status, 0x42);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(do_full, 2 * L::kSlab);
+                    for (int c = 0; c < 2; ++c)
+                        tma_load_2d(smem + L::kDo + c * L::kSlab, &tmap_do, do_full, head * 128 + c * 64, q0);
+                }
             }
         }
     } else if (warp == 1) {
         if (elect_one()) {
-            constexpr uint32_t idesc_st = make_idesc_bf16(128, 64, 0, 0);    // S^T, dP^T: both K-major
+            constexpr uint32_t idesc_st = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: both K-major
             constexpr uint32_t idesc_dv = make_idesc_bf16(128, 128, 0, 1);   // dV: A = P^T (TMEM), B = dO MN-major
             constexpr uint32_t idesc_dk = make_idesc_bf16(128, 192, 0, 1);   // dK: A = dS^T (TMEM), B = Q MN-major
-            const uint32_t sk = smem_u32(smem + L::kK), sv = smem_u32(smem + L::kV);
-            auto stage_q = [&](int j) { return smem_u32(smem + L::kQdO + (j % kBwdStages) * L::kStage); };
-            auto issue_st = [&](int j) -> bool {     // S^T(j) = K Q_j^T into the group's scratch columns
-                const int g = j & 1;
-                if (!mbar_wait(&qdo_full[j % kBwdStages], (j / kBwdStages) & 1, abort_flag, args.status, 0x52))
-                    return false;
+            const uint32_t sk = smem_u32(smem + L::kK), sv = smem_u32(smem + L::kV), sdo = smem_u32(smem + L::kDo);
+            auto stage_q = [&](uint32_t T) { return smem_u32(smem + L::kQ + (T % L::kQStages) * 3 * L::kSlab); };
+            auto issue_st = [&](uint32_t T, bool first_of_cta) -> bool {   // S^T(T) = K Q^T into X
+                if (!mbar_wait(&q_full[T % L::kQStages], (T / L::kQStages) & 1u, abort_flag, args.status, 0x52)) return false;
+                // X still holds dP^T of the previous tile until both groups have loaded it
+                if (!first_of_cta && !mbar_wait(dp_read, (T - 1) & 1u, abort_flag, args.status, 0x57)) return false;
                 tc_fence_after_sync();
-                const uint32_t sq = stage_q(j);
+                const uint32_t sq = stage_q(T);
 #pragma unroll
-                for (int kk = 0; kk < 12; ++kk)
-                    mma_ss(tmem_base + g * 64, desc_k_major(sk + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
-                           desc_k_major(sq + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_st, kk > 0 ? 1u : 0u);
-                mma_commit(&st_full[g]);
+                for (int kk = 0; kk < 12; ++kk) {
+                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
+                    mma_ss(tmem_base, desc_k_major(sk + off), desc_k_major(sq + off), idesc_st, kk > 0 ? 1u : 0u);
+                }
+                mma_commit(st_full);
                 return true;
             };
-            auto issue_dp = [&](int j) -> bool {     // dP^T(j) = V dO_j^T over the same columns once S^T was read
-                const int g = j & 1;
-                if (!mbar_wait(&st_read[g], (j >> 1) & 1, abort_flag, args.status, 0x53)) return false;
+            auto issue_dp = [&](uint32_t T) -> bool {     // dP^T(T) = V dO^T over X once S^T(T) was read
+                if (!mbar_wait(st_read, T & 1u, abort_flag, args.status, 0x53)) return false;
+                if (!mbar_wait(do_full, T & 1u, abort_flag, args.status, 0x55)) return false;
                 tc_fence_after_sync();
-                const uint32_t sdo = stage_q(j) + 3 * L::kSlab64;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    mma_ss(tmem_base + g * 64, desc_k_major(sv + (kk >> 2) * L::kSlab128 + (kk & 3) * 32),
-                           desc_k_major(sdo + (kk >> 2) * L::kSlab64 + (kk & 3) * 32), idesc_st, kk > 0 ? 1u : 0u);
-                mma_commit(&dp_full[g]);
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
+                    mma_ss(tmem_base, desc_k_major(sv + off), desc_k_major(sdo + off), idesc_st, kk > 0 ? 1u : 0u);
+                }
+                mma_commit(dp_full);
                 return true;
             };
-            auto issue_dv = [&](int j) -> bool {     // dV += P^T dO_j (A operand from TMEM)
-                const int g = j & 1;
-                if (!mbar_wait(&p_full[g], (j >> 1) & 1, abort_flag, args.status, 0x50)) return false;
-                tc_fence_after_sync();
-                const uint32_t sdo = stage_q(j) + 3 * L::kSlab64;
+            uint32_t T0 = 0;
+            bool ok = true;
+            for (uint32_t n = 0; ok; ++n) {
+                const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
+                if (!ok || item < 0) break;
+                int t0, head, j_begin, n_iter;
+                item_geometry(item, t0, head, j_begin, n_iter);
+                ok = mbar_wait(kv_full, n & 1u, abort_flag, args.status, 0x54);
+                if (ok) ok = issue_st(T0, T0 == 0);
+                if (ok) ok = issue_dp(T0);
+                if (ok && n_iter == 1) mma_commit(kv_empty);
+                for (int j = 0; j < n_iter && ok; ++j) {
+                    const uint32_t T = T0 + j;
+                    // dV += P^T(j) dO(j)   (A from Y: group 0's 64 queries, then group 1's)
+                    ok = mbar_wait(p_full, T & 1u, abort_flag, args.status, 0x50);
+                    // the first accumulation of an item overwrites dV and dK: the previous item's must be drained
+                    if (ok && j == 0 && n > 0) ok = mbar_wait(acc_empty, (n - 1) & 1u, abort_flag, args.status, 0x56);
+                    if (!ok) break;
+                    tc_fence_after_sync();
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ts(tmem_dv, tmem_pt + g * 32 + kk * 8, desc_mn_major(sdo + kk * 2048, L::kSlab64), idesc_dv,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-                return true;
-            };
-            auto issue_dk = [&](int j) -> bool {     // dK += dS^T Q_j (A operand from TMEM)
-                const int g = j & 1;
-                if (!mbar_wait(&ds_full[g], (j >> 1) & 1, abort_flag, args.status, 0x51)) return false;
-                tc_fence_after_sync();
-                const uint32_t sq = stage_q(j);
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ts(tmem_dv, tmem_y + kk * 8, desc_mn_major(sdo + kk * 2048, L::kSlab), idesc_dv,
+                               (j > 0 || kk > 0) ? 1u : 0u);
+                    mma_commit(do_empty);
+                    mma_commit(dv_done);
+                    if (j + 1 < n_iter) {
+                        ok = issue_st(T + 1, false);
+                        if (!ok) break;
+                    }
+                    // dK += dS^T(j) Q(j)
+                    ok = mbar_wait(ds_full, T & 1u, abort_flag, args.status, 0x51);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t sq = stage_q(T);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ts(tmem_dk, tmem_base + g * 64 + kk * 8, desc_mn_major(sq + kk * 2048, L::kSlab64), idesc_dk,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-                mma_commit(&qdo_empty[j % kBwdStages]);
-                return true;
-            };
-            // Issue order per tile: S^T(j), dV(j-1), dP^T(j), dK(j-1).  dV(j-1) gives this tile's warpgroup
-            // time to load S^T(j) before dP^T(j) overwrites it, and dK(j-1) comes last so that the other
-            // warpgroup has S^T(j), dV(j-1) and dP^T(j) -- some 1200 clocks -- to turn dP^T(j-1) into dS^T(j-1).
-            bool ok = mbar_wait(kv_full, 0, abort_flag, args.status, 0x54);
-            for (int j = 0; j < n_iter && ok; ++j) {
-                ok = issue_st(j);
-                if (ok && j > 0) ok = issue_dv(j - 1);
-                if (ok) ok = issue_dp(j);
-                if (ok && j > 0) ok = issue_dk(j - 1);
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ts(tmem_dk, tmem_y + kk * 8, desc_mn_major(sq + kk * 2048, L::kSlab), idesc_dk,
+                               (j > 0 || kk > 0) ? 1u : 0u);
+                    mma_commit(&q_empty[T % L::kQStages]);
+                    mma_commit(dk_done);
+                    if (j + 1 < n_iter) {
+                        ok = issue_dp(T + 1);
+                        if (ok && j + 2 == n_iter) mma_commit(kv_empty);   // that was the item's last read of K and V
+                    }
+                }
+                if (ok) mma_commit(acc_full);
+                T0 += static_cast<uint32_t>(n_iter);
             }
-            if (ok) ok = issue_dv(n_iter - 1);
-            if (ok) ok = issue_dk(n_iter - 1);
-            if (ok) mma_commit(acc_done);
         }
     } else {
-        const int g = (warp - 2) >> 2;               // consumer warpgroup 0 or 1
+        const int g = (warp - 2) >> 2;               // consumer warpgroup: query columns [64g, 64g+64) of every tile
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;         // key row inside the tile == TMEM lane
-        const int t_idx = t0 + row;
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-        const uint32_t tmem_scr = tmem_base + g * 64 + lane_addr;
+        const uint32_t tmem_x = tmem_base + lane_addr + g * 64;
+        const uint32_t tmem_yg = tmem_y + lane_addr + g * 32;
+        uint32_t T0 = 0;
         bool ok = true;
-        for (int j = g; j < n_iter; j += 2) {
-            const uint32_t ph = (j >> 1) & 1;
-            const int st = j % kBwdStages;
-            const int q0 = (j_begin + j) * 64;
-            ok = mbar_wait_warp(&st_full[g], ph, abort_flag, args.status, 0x60);
-            if (!ok) break;
-            tc_fence_after_sync();
-            uint32_t sv[64];
-            tmem_ld_x32(tmem_scr, sv);
-            tmem_ld_x32(tmem_scr + 32, sv + 32);
-            tmem_ld_wait();
-            tc_fence_before_sync();
-            mbar_arrive(&st_read[g]);
-            // The statistics arrived with Q/dO on qdo_full[st]; waiting on it here makes those
-            // bulk-copy writes visible to this thread as well.
-            ok = mbar_wait_warp(&qdo_full[st], (j / kBwdStages) & 1, abort_flag, args.status, 0x61);
-            if (!ok) break;
-            const float* stat = reinterpret_cast<const float*>(smem + L::kStat + st * 512);
-            const bool diag = kCausal && (q0 < t0 + 128);
-            float p[64];
-#pragma unroll
-            for (int c4 = 0; c4 < 16; ++c4) {
-                const float4 l2 = *reinterpret_cast<const float4*>(stat + c4 * 4);
-                const float l2v[4] = {l2.x, l2.y, l2.z, l2.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = c4 * 4 + e;
-                    float v = fast_exp2(fmaf(__uint_as_float(sv[c]), args.scale_log2, -l2v[e]));
-                    if (diag && t_idx > q0 + c) v = 0.f;
-                    p[c] = v;
-                }
+        for (uint32_t n = 0; ok; ++n) {
+            int item = 0;
+            {
+                ok = mbar_wait_warp(&ring.full[n & 1u], (n >> 1) & 1u, abort_flag, args.status, 0xA1);
+                if (!ok) break;
+                item = ring.item[n & 1u];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ring.empty[n & 1u]);
             }
-            uint32_t pk[32];
+            if (item < 0) break;
+            int t0, head, j_begin, n_iter;
+            item_geometry(item, t0, head, j_begin, n_iter);
+            const int t_idx = t0 + row;
+            for (int j = 0; j < n_iter; ++j) {
+                const uint32_t T = T0 + j;
+                const uint32_t ph = T & 1u;
+                const uint32_t sq = T % L::kQStages;
+                const int q0 = (j_begin + j) * 128 + g * 64;     // first query of this group's columns
+                ok = mbar_wait_warp(st_full, ph, abort_flag, args.status, 0x60);
+                if (!ok) break;
+                tc_fence_after_sync();
+                uint32_t sv[64];
+                tmem_ld_x32(tmem_x, sv);
+                tmem_ld_x32(tmem_x + 32, sv + 32);
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                mbar_arrive(st_read);
+                // The statistics arrived with the Q tile; waiting on its barrier here makes those bulk-copy
+                // writes visible to this thread as well (the wait returns at once: S^T needed the same tile).
+                ok = mbar_wait_warp(&q_full[sq], (T / L::kQStages) & 1u, abort_flag, args.status, 0x61);
+                if (!ok) break;
+                const float* stat = reinterpret_cast<const float*>(smem + L::kStat + sq * 1024) + g * 64;
+                const bool diag = kCausal && (q0 < t0 + 128);
+                float p[64];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
-            tmem_st_x32(tmem_pt + g * 32 + lane_addr, pk);
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(&p_full[g]);
+                for (int c4 = 0; c4 < 16; ++c4) {
+                    const float4 l2 = *reinterpret_cast<const float4*>(stat + c4 * 4);
+                    const float l2v[4] = {l2.x, l2.y, l2.z, l2.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int c = c4 * 4 + e;
+                        float v = fast_exp2(fmaf(__uint_as_float(sv[c]), args.scale_log2, -l2v[e]));
+                        if (diag && t_idx > q0 + c) v = 0.f;
+                        p[c] = v;
+                    }
+                }
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(p[2 * c], p[2 * c + 1]);
+                // Y still holds dS^T of the previous tile until dK has consumed it
+                if (T > 0) {
+                    ok = mbar_wait_warp(dk_done, (T - 1) & 1u, abort_flag, args.status, 0x62);
+                    if (!ok) break;
+                }
+                tmem_st_x32(tmem_yg, pk);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(p_full);
 
-            ok = mbar_wait_warp(&dp_full[g], ph, abort_flag, args.status, 0x63);
-            if (!ok) break;
-            tc_fence_after_sync();
-            tmem_ld_x32(tmem_scr, sv);
-            tmem_ld_x32(tmem_scr + 32, sv + 32);
-            tmem_ld_wait();
+                ok = mbar_wait_warp(dp_full, ph, abort_flag, args.status, 0x63);
+                if (!ok) break;
+                tc_fence_after_sync();
+                tmem_ld_x32(tmem_x, sv);
+                tmem_ld_x32(tmem_x + 32, sv + 32);
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                mbar_arrive(dp_read);
 #pragma unroll
-            for (int c8 = 0; c8 < 8; ++c8) {
-                const float4 d0 = *reinterpret_cast<const float4*>(stat + 64 + c8 * 8);
-                const float4 d1 = *reinterpret_cast<const float4*>(stat + 64 + c8 * 8 + 4);
-                const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    const float4 d0 = *reinterpret_cast<const float4*>(stat + 128 + c8 * 8);
+                    const float4 d1 = *reinterpret_cast<const float4*>(stat + 128 + c8 * 8 + 4);
+                    const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int c = c8 * 8 + 2 * e;
-                    pk[c8 * 4 + e] = pack_bf16x2(p[c] * (__uint_as_float(sv[c]) - dl[2 * e]),
-                                                 p[c + 1] * (__uint_as_float(sv[c + 1]) - dl[2 * e + 1]));
+                    for (int e = 0; e < 4; ++e) {
+                        const int c = c8 * 8 + 2 * e;
+                        pk[c8 * 4 + e] = pack_bf16x2(p[c] * (__uint_as_float(sv[c]) - dl[2 * e]),
+                                                     p[c + 1] * (__uint_as_float(sv[c + 1]) - dl[2 * e + 1]));
+                    }
                 }
+                // Y holds P^T of this tile until dV has consumed it
+                ok = mbar_wait_warp(dv_done, ph, abort_flag, args.status, 0x65);
+                if (!ok) break;
+                tmem_st_x32(tmem_yg, pk);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(ds_full);
             }
-            tmem_st_x32(tmem_scr, pk);               // dS^T over the first 32 of the columns dP^T occupied
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(&ds_full[g]);
-        }
-        if (ok) ok = mbar_wait_warp(acc_done, 0, abort_flag, args.status, 0x64);
-        if (ok) {
+            if (!ok) break;
+            T0 += static_cast<uint32_t>(n_iter);
+            ok = mbar_wait_warp(acc_full, n & 1u, abort_flag, args.status, 0x64);
+            if (!ok) break;
             tc_fence_after_sync();
             const bool valid = t_idx < args.S;
             __nv_bfloat16* dkv_row = args.dkv + static_cast<size_t>(t_idx) * args.h * 256 + head * 256;
@@ -383,11 +469,15 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     }
                 }
             }
+            __syncwarp();
+            tc_fence_before_sync();
+            mbar_arrive(acc_empty);
         }
     }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    clock_probe_end(args.clock_probe);
 }
 
 
@@ -403,6 +493,8 @@ struct AttnBwdDqArgs {
     const __nv_bfloat16* dout;   // [S, h, 128]
     __nv_bfloat16* dq;           // [S, h, 192]
     unsigned int* status;
+    WorkSchedule sched;          // items = (128-query tile, head); rank 0 = the last query tile (most keys)
+    ClockProbe* clock_probe;     // may be nullptr
 };
 
 constexpr int kDqKStages = 3;
@@ -413,52 +505,59 @@ struct AttnBwdDqSmem {
     static constexpr int kK = kQ + 3 * kSlab;                  // 3 stages x 3 slabs
     static constexpr int kV = kK + kDqKStages * 3 * kSlab;     // 1 stage x 2 slabs
     static constexpr int kBar = kV + 2 * kSlab;
-    static constexpr int kTotalBytes = kBar + 256 + 1024;
+    static constexpr int kTotalBytes = kBar + 512;
 };
 
-// dO of the query tile is the A operand of dP = dO V^T for every key tile.  It is kept in TMEM as
-// packed bf16 (64 columns) instead of 32 KB of shared memory, which is what leaves room for a third
-// stage of K: a K tile lives from its score MMA to its dQ MMA, a whole tile period later.
+// Persistent: one CTA per SM takes (query tile, head) items from the work counter.  dO of the query
+// tile is the A operand of dP = dO V^T for every key tile; it is kept in TMEM as packed bf16 (64
+// columns) instead of 32 KB of shared memory, which is what leaves room for a third stage of K: a K
+// tile lives from its score MMA to its dQ MMA, a whole tile period later.  Between items the
+// consumers first put the next tile's dO into TMEM and only then drain the finished dQ, so the score
+// MMAs of the next item run under the drain; the K ring simply keeps going across items.
 template <bool kCausal>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                          const __grid_constant__ CUtensorMap tmap_kpe, const AttnBwdDqArgs args) {
     using L = AttnBwdDqSmem;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
     uint64_t* q_full = bars + 0;
-    uint64_t* k_full = bars + 1;      // [3]
-    uint64_t* k_empty = bars + 4;     // [3]
-    uint64_t* v_full = bars + 7;
-    uint64_t* v_empty = bars + 8;
-    uint64_t* do_ready = bars + 9;    // dO is in TMEM
-    uint64_t* s_full = bars + 10;     // S is in TMEM
-    uint64_t* s_read = bars + 11;     // both groups have loaded it
-    uint64_t* dp_full = bars + 12;    // dP is in TMEM
-    uint64_t* ds_full = bars + 13;    // dS (bf16) is in TMEM
-    uint64_t* acc_done = bars + 14;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+    uint64_t* q_empty = bars + 1;     // the item's last score MMA has read Q
+    uint64_t* k_full = bars + 2;      // [3]
+    uint64_t* k_empty = bars + 5;     // [3]
+    uint64_t* v_full = bars + 8;
+    uint64_t* v_empty = bars + 9;
+    uint64_t* do_ready = bars + 10;   // the item's dO is in TMEM
+    uint64_t* s_full = bars + 11;     // S is in TMEM
+    uint64_t* s_read = bars + 12;     // both groups have loaded it
+    uint64_t* dp_full = bars + 13;    // dP is in TMEM
+    uint64_t* ds_full = bars + 14;    // dS (bf16) is in TMEM
+    uint64_t* acc_full = bars + 15;   // the item's dQ is complete
+    uint64_t* acc_empty = bars + 16;  // both groups have drained it
+    ItemRing ring{bars + 17, bars + 19, reinterpret_cast<volatile int*>(bars + 21)};
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_q_tiles = (args.S + 127) / 128;
-    const int q_tile = n_q_tiles - 1 - static_cast<int>(blockIdx.x);
-    const int head = blockIdx.y;
-    const int q0 = q_tile * 128;
-    const int n_iter = kCausal ? q_tile + 1 : n_q_tiles;
 
     if (threadIdx.x == 0) {
-        mbar_init(q_full, 1);
+        mbar_init(q_full, 1); mbar_init(q_empty, 1);
         for (int s = 0; s < kDqKStages; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); }
         mbar_init(v_full, 1); mbar_init(v_empty, 1);
         mbar_init(do_ready, 256);
         mbar_init(s_full, 1); mbar_init(s_read, 256); mbar_init(dp_full, 1); mbar_init(ds_full, 256);
-        mbar_init(acc_done, 1);
+        mbar_init(acc_full, 1); mbar_init(acc_empty, 256);
+        for (int s = 0; s < 2; ++s) { mbar_init(&ring.full[s], 1); mbar_init(&ring.empty[s], 9); }
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
+        if ((smem_u32(smem) & 1023u) != 0u) {
+            abort_flag->value = 1;
+            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD1u);
+        }
     }
+    clock_probe_begin(args.clock_probe);
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
@@ -469,15 +568,23 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     const uint32_t tmem_dp = tmem_base + 128;
     const uint32_t tmem_do = tmem_base + 256;
     const uint32_t tmem_dq = tmem_base + 320;
+    auto item_geometry = [&](int item, int& q0, int& head, int& n_iter) {
+        int rank;
+        decode_item(args.sched, item, rank, head);
+        const int q_tile = n_q_tiles - 1 - rank;               // longest rows first
+        q0 = q_tile * 128;
+        n_iter = kCausal ? q_tile + 1 : n_q_tiles;
+    };
 
-    if (warp == 0) {
+    if (abort_flag->value != 0u) {
+        // misaligned shared memory: nothing was started, fall through to the common exit
+    } else if (warp == 0) {
         if (elect_one()) {
-            mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
-            for (int c = 0; c < 3; ++c)
-                tma_load_2d(smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
-            auto load_k = [&](int j) -> bool {
-                const int st = j % kDqKStages;
-                if (!mbar_wait(&k_empty[st], ((j / kDqKStages) & 1) ^ 1, abort_flag, args.status, 0x70)) return false;
+            uint32_t T0 = 0;
+            bool ok = true;
+            auto load_k = [&](uint32_t T, int j, int head) -> bool {
+                const uint32_t st = T % kDqKStages;
+                if (!mbar_wait(&k_empty[st], ((T / kDqKStages) & 1u) ^ 1u, abort_flag, args.status, 0x70)) return false;
                 mbar_arrive_expect_tx(&k_full[st], 3 * L::kSlab);
                 uint8_t* sk = smem + L::kK + st * 3 * L::kSlab;
                 tma_load_2d(sk, &tmap_kv, &k_full[st], head * 256, j * 128);
@@ -485,15 +592,28 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 tma_load_2d(sk + 2 * L::kSlab, &tmap_kpe, &k_full[st], 0, j * 128);
                 return true;
             };
-            bool ok = load_k(0);
-            for (int j = 0; j < n_iter && ok; ++j) {
-                if (j + 1 < n_iter) ok = load_k(j + 1);
+            for (uint32_t n = 0; ok; ++n) {
+                const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
+                if (!ok || item < 0) break;
+                int q0, head, n_iter;
+                item_geometry(item, q0, head, n_iter);
+                ok = mbar_wait(q_empty, (n & 1u) ^ 1u, abort_flag, args.status, 0x72);
                 if (!ok) break;
-                ok = mbar_wait(v_empty, (j & 1) ^ 1, abort_flag, args.status, 0x71);
-                if (!ok) break;
-                mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
-                tma_load_2d(smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
-                tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
+                mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
+                for (int c = 0; c < 3; ++c)
+                    tma_load_2d(smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
+                ok = load_k(T0, 0, head);
+                for (int j = 0; j < n_iter && ok; ++j) {
+                    const uint32_t T = T0 + j;
+                    if (j + 1 < n_iter) ok = load_k(T + 1, j + 1, head);
+                    if (!ok) break;
+                    ok = mbar_wait(v_empty, (T & 1u) ^ 1u, abort_flag, args.status, 0x71);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
+                    tma_load_2d(smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
+                    tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
+                }
+                T0 += static_cast<uint32_t>(n_iter);
             }
         }
     } else if (warp == 1) {
@@ -502,12 +622,12 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, 192, 0, 1);   // dQ: A = dS (TMEM), B = K MN-major
             const uint32_t sq = smem_u32(smem + L::kQ);
             const uint32_t sv = smem_u32(smem + L::kV);
-            auto stage_k = [&](int j) { return smem_u32(smem + L::kK + (j % kDqKStages) * 3 * L::kSlab); };
-            auto issue_s = [&](int j) -> bool {      // S(j) = Q K_j^T
-                if (!mbar_wait(&k_full[j % kDqKStages], (j / kDqKStages) & 1, abort_flag, args.status, 0x82)) return false;
-                if (j > 0 && !mbar_wait(s_read, (j - 1) & 1, abort_flag, args.status, 0x83)) return false;
+            auto stage_k = [&](uint32_t T) { return smem_u32(smem + L::kK + (T % kDqKStages) * 3 * L::kSlab); };
+            auto issue_s = [&](uint32_t T) -> bool {      // S(T) = Q K^T
+                if (!mbar_wait(&k_full[T % kDqKStages], (T / kDqKStages) & 1u, abort_flag, args.status, 0x82)) return false;
+                if (T > 0 && !mbar_wait(s_read, (T - 1) & 1u, abort_flag, args.status, 0x83)) return false;
                 tc_fence_after_sync();
-                const uint32_t sk = stage_k(j);
+                const uint32_t sk = stage_k(T);
 #pragma unroll
                 for (int kk = 0; kk < 12; ++kk) {
                     const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
@@ -516,8 +636,8 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 mma_commit(s_full);
                 return true;
             };
-            auto issue_dp = [&](int j) -> bool {     // dP(j) = dO V_j^T; overwrites dS(j-1), whose reader was issued earlier
-                if (!mbar_wait(v_full, j & 1, abort_flag, args.status, 0x84)) return false;
+            auto issue_dp = [&](uint32_t T) -> bool {     // dP(T) = dO V^T; overwrites dS(T-1), whose reader was issued earlier
+                if (!mbar_wait(v_full, T & 1u, abort_flag, args.status, 0x84)) return false;
                 tc_fence_after_sync();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
@@ -527,100 +647,63 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 mma_commit(dp_full);
                 return true;
             };
-            bool ok = mbar_wait(q_full, 0, abort_flag, args.status, 0x81) &&
-                      mbar_wait(do_ready, 0, abort_flag, args.status, 0x85);
-            if (ok) ok = issue_s(0);
-            if (ok) ok = issue_dp(0);
-            for (int j = 0; j < n_iter && ok; ++j) {
-                if (j + 1 < n_iter) ok = issue_s(j + 1);
-                if (!ok) break;
-                ok = mbar_wait(ds_full, j & 1, abort_flag, args.status, 0x80);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t sk = stage_k(j);
+            uint32_t T0 = 0;
+            bool ok = true;
+            for (uint32_t n = 0; ok; ++n) {
+                const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
+                if (!ok || item < 0) break;
+                int q0, head, n_iter;
+                item_geometry(item, q0, head, n_iter);
+                ok = mbar_wait(q_full, n & 1u, abort_flag, args.status, 0x81);
+                if (ok) ok = issue_s(T0);
+                if (ok && n_iter == 1) mma_commit(q_empty);
+                if (ok) ok = mbar_wait(do_ready, n & 1u, abort_flag, args.status, 0x85);
+                if (ok) ok = issue_dp(T0);
+                for (int j = 0; j < n_iter && ok; ++j) {
+                    const uint32_t T = T0 + j;
+                    if (j + 1 < n_iter) {
+                        ok = issue_s(T + 1);
+                        if (ok && j + 2 == n_iter) mma_commit(q_empty);   // that was the item's last read of Q
+                    }
+                    if (!ok) break;
+                    ok = mbar_wait(ds_full, T & 1u, abort_flag, args.status, 0x80);
+                    // the first accumulation of an item overwrites dQ: the previous item's must be drained
+                    if (ok && j == 0 && n > 0) ok = mbar_wait(acc_empty, (n - 1) & 1u, abort_flag, args.status, 0x86);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t sk = stage_k(T);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    mma_ts(tmem_dq, tmem_dp + (kk >> 2) * 64 + (kk & 3) * 8, desc_mn_major(sk + kk * 2048, L::kSlab),
-                           idesc_dq, (j > 0 || kk > 0) ? 1u : 0u);
-                mma_commit(&k_empty[j % kDqKStages]);
-                if (j + 1 < n_iter) ok = issue_dp(j + 1);
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ts(tmem_dq, tmem_dp + (kk >> 2) * 64 + (kk & 3) * 8, desc_mn_major(sk + kk * 2048, L::kSlab),
+                               idesc_dq, (j > 0 || kk > 0) ? 1u : 0u);
+                    mma_commit(&k_empty[T % kDqKStages]);
+                    if (j + 1 < n_iter) ok = issue_dp(T + 1);
+                }
+                if (ok) mma_commit(acc_full);
+                T0 += static_cast<uint32_t>(n_iter);
             }
-            if (ok) mma_commit(acc_done);
         }
     } else {
         const int g = (warp - 2) >> 2;               // consumer group: key columns [64g, 64g+64) of the tile
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
-        const int s_idx = q0 + row;
-        const bool valid = s_idx < args.S;
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-        {   // this thread's dO row, channels [64g, 64g+64), as 32 packed words into TMEM
-            uint32_t w[32];
-            if (valid) {
-                const uint4* src = reinterpret_cast<const uint4*>(args.dout + (static_cast<size_t>(s_idx) * args.h + head) * 128 + g * 64);
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                    const uint4 x = src[v];
-                    w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
-                }
-            } else {
-#pragma unroll
-                for (int v = 0; v < 32; ++v) w[v] = 0u;
-            }
+        auto read_item = [&](uint32_t n, bool& ok) -> int {
+            ok = mbar_wait_warp(&ring.full[n & 1u], (n >> 1) & 1u, abort_flag, args.status, 0xA1);
+            if (!ok) return -1;
+            const int it = ring.item[n & 1u];
             __syncwarp();
-            tmem_st_x32(tmem_do + lane_addr + g * 32, w);
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(do_ready);
-        }
-        // Rows past the end of the sequence get LSE = +inf so that their P is exactly zero.
-        const float l2 = valid ? args.lse[static_cast<size_t>(s_idx) * args.h + head] * 1.4426950408889634f : INFINITY;
-        const float delta = valid ? args.stat_delta[static_cast<size_t>(head) * args.S_pad + s_idx] : 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_iter; ++j) {
-            ok = mbar_wait_warp(s_full, j & 1, abort_flag, args.status, 0x90);
-            if (!ok) break;
+            if (lane == 0) mbar_arrive(&ring.empty[n & 1u]);
+            return it;
+        };
+        // dQ of a finished item: six 32-column chunks, three per group
+        auto drain = [&](uint32_t n_done, int s_idx, int head) -> bool {
+            if (!mbar_wait_warp(acc_full, n_done & 1u, abort_flag, args.status, 0x92)) return false;
             tc_fence_after_sync();
-            uint32_t sv[64];
-            tmem_ld_x32(tmem_base + lane_addr + g * 64, sv);
-            tmem_ld_x32(tmem_base + lane_addr + g * 64 + 32, sv + 32);
-            tmem_ld_wait();
-            tc_fence_before_sync();
-            mbar_arrive(s_read);
-            const int tk0 = j * 128 + g * 64;
-            const bool edge = (kCausal && tk0 + 63 > q0) || (tk0 + 64 > args.S);
-            float p[64];
-#pragma unroll
-            for (int c = 0; c < 64; ++c) {
-                float v = fast_exp2(fmaf(__uint_as_float(sv[c]), args.scale_log2, -l2));
-                if (edge) {
-                    const int t = tk0 + c;
-                    if ((kCausal && t > s_idx) || t >= args.S) v = 0.f;
-                }
-                p[c] = v;
-            }
-            ok = mbar_wait_warp(dp_full, j & 1, abort_flag, args.status, 0x91);
-            if (!ok) break;
-            tc_fence_after_sync();
-            tmem_ld_x32(tmem_dp + lane_addr + g * 64, sv);
-            tmem_ld_x32(tmem_dp + lane_addr + g * 64 + 32, sv + 32);
-            tmem_ld_wait();
-            uint32_t pk[32];
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-                pk[c] = pack_bf16x2(p[2 * c] * (__uint_as_float(sv[2 * c]) - delta),
-                                    p[2 * c + 1] * (__uint_as_float(sv[2 * c + 1]) - delta));
-            tmem_st_x32(tmem_dp + lane_addr + g * 64, pk);   // dS over the first 32 columns of this group's own half
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(ds_full);
-        }
-        if (ok) ok = mbar_wait_warp(acc_done, 0, abort_flag, args.status, 0x92);
-        if (ok) {
-            tc_fence_after_sync();
+            const bool valid = s_idx < args.S;
             __nv_bfloat16* dst = args.dq + (static_cast<size_t>(s_idx) * args.h + head) * 192;
 #pragma unroll 1
-            for (int c = g * 3; c < g * 3 + 3; ++c) {   // six 32-column chunks, three per group
+            for (int c = g * 3; c < g * 3 + 3; ++c) {
                 uint32_t r[32];
                 __syncwarp();
                 tmem_ld_x32(tmem_dq + lane_addr + c * 32, r);
@@ -636,11 +719,95 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     reinterpret_cast<uint4*>(dst + c * 32)[v] = w;
                 }
             }
+            __syncwarp();
+            tc_fence_before_sync();
+            mbar_arrive(acc_empty);
+            return true;
+        };
+        uint32_t T0 = 0;
+        bool ok = true;
+        int item = read_item(0, ok);
+        int prev_s_idx = 0, prev_head = 0;
+        for (uint32_t n = 0; ok && item >= 0; ++n) {
+            int q0, head, n_iter;
+            item_geometry(item, q0, head, n_iter);
+            const int s_idx = q0 + row;
+            const bool valid = s_idx < args.S;
+            {   // this thread's dO row, channels [64g, 64g+64), as 32 packed words into TMEM (the previous item's
+                // last dP MMA has completed: this group waited for it before writing its last dS)
+                uint32_t w[32];
+                if (valid) {
+                    const uint4* src = reinterpret_cast<const uint4*>(args.dout + (static_cast<size_t>(s_idx) * args.h + head) * 128 + g * 64);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const uint4 x = src[v];
+                        w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int v = 0; v < 32; ++v) w[v] = 0u;
+                }
+                __syncwarp();
+                tmem_st_x32(tmem_do + lane_addr + g * 32, w);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(do_ready);
+            }
+            // Rows past the end of the sequence get LSE = +inf so that their P is exactly zero.
+            const float l2 = valid ? args.lse[static_cast<size_t>(s_idx) * args.h + head] * 1.4426950408889634f : INFINITY;
+            const float delta = valid ? args.stat_delta[static_cast<size_t>(head) * args.S_pad + s_idx] : 0.f;
+            if (n > 0) ok = drain(n - 1, prev_s_idx, prev_head);
+            for (int j = 0; j < n_iter && ok; ++j) {
+                const uint32_t T = T0 + j;
+                ok = mbar_wait_warp(s_full, T & 1u, abort_flag, args.status, 0x90);
+                if (!ok) break;
+                tc_fence_after_sync();
+                uint32_t sv[64];
+                tmem_ld_x32(tmem_base + lane_addr + g * 64, sv);
+                tmem_ld_x32(tmem_base + lane_addr + g * 64 + 32, sv + 32);
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                mbar_arrive(s_read);
+                const int tk0 = j * 128 + g * 64;
+                const bool edge = (kCausal && tk0 + 63 > q0) || (tk0 + 64 > args.S);
+                float p[64];
+#pragma unroll
+                for (int c = 0; c < 64; ++c) {
+                    float v = fast_exp2(fmaf(__uint_as_float(sv[c]), args.scale_log2, -l2));
+                    if (edge) {
+                        const int t = tk0 + c;
+                        if ((kCausal && t > s_idx) || t >= args.S) v = 0.f;
+                    }
+                    p[c] = v;
+                }
+                ok = mbar_wait_warp(dp_full, T & 1u, abort_flag, args.status, 0x91);
+                if (!ok) break;
+                tc_fence_after_sync();
+                tmem_ld_x32(tmem_dp + lane_addr + g * 64, sv);
+                tmem_ld_x32(tmem_dp + lane_addr + g * 64 + 32, sv + 32);
+                tmem_ld_wait();
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    pk[c] = pack_bf16x2(p[2 * c] * (__uint_as_float(sv[2 * c]) - delta),
+                                        p[2 * c + 1] * (__uint_as_float(sv[2 * c + 1]) - delta));
+                tmem_st_x32(tmem_dp + lane_addr + g * 64, pk);   // dS over the first 32 columns of this group's own half
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(ds_full);
+            }
+            if (!ok) break;
+            T0 += static_cast<uint32_t>(n_iter);
+            prev_s_idx = s_idx;
+            prev_head = head;
+            item = read_item(n + 1, ok);
+            if (ok && item < 0) ok = drain(n, prev_s_idx, prev_head);
         }
     }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    clock_probe_end(args.clock_probe);
 }
 
 }  // namespace laga

@@ -26,6 +26,7 @@
 // no extra barrier guards it.
 #pragma once
 #include "sm100_ptx.cuh"
+#include "work_sched.cuh"
 
 namespace laga {
 
@@ -36,6 +37,8 @@ struct AttnFwdArgs {
     __nv_bfloat16* out;     // [S, h, 128]
     float* lse;             // [S, h]
     unsigned int* status;
+    WorkSchedule sched;     // items = (128-query tile, head); rank 0 = the last query tile (most keys)
+    ClockProbe* clock_probe;   // may be nullptr
 };
 
 constexpr int kFwdThreads = 352;
@@ -47,9 +50,9 @@ struct AttnFwdSmem {
     static constexpr int kK = 0;                                 // stages x 3 slabs (nope lo, nope hi, rope)
     static constexpr int kV = kK + kFwdStages * 3 * kSlab;       // stages x 2 slabs
     static constexpr int kMref = kV + kFwdStages * 2 * kSlab;    // 128 floats: the rows' reference maxima
-    static constexpr int kLsum = kMref + 512;                    // 2 x 128 floats: the groups' row sums
-    static constexpr int kBar = kLsum + 1024;
-    static constexpr int kTotalBytes = kBar + 512 + 1024;
+    static constexpr int kLsum = kMref + 512;                    // 2 items x 2 groups x 128 floats: row sums
+    static constexpr int kBar = kLsum + 2048;
+    static constexpr int kTotalBytes = kBar + 512;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -64,38 +67,39 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return r;
 }
 
+// Persistent: one CTA per SM takes (query tile, head) items from the work counter.  The K, V and
+// score-tile rings and the alternation of the two softmax groups run on a tile count that continues
+// across items, so the producers prefetch the next item's first key tiles under the current item's
+// last ones; between items, group 0 puts the next query tile into TMEM before the finished O is
+// drained, so the next item's first score MMAs run under the drain.
 template <bool kCausal>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
                       const AttnFwdArgs args) {
     using L = AttnFwdSmem;
     constexpr int BK = kFwdKeys;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
-    uint64_t* q_ready = bars + 0;    // warpgroup 0 has put the Q tile into TMEM
+    uint64_t* q_ready = bars + 0;    // warpgroup 0 has put the item's Q tile into TMEM
     uint64_t* k_full = bars + 1;     // [3]
     uint64_t* k_empty = bars + 4;    // [3]
     uint64_t* v_full = bars + 7;     // [3]
     uint64_t* v_empty = bars + 10;   // [3]
-    uint64_t* s_full = bars + 13;    // [3]  S tile j is in TMEM buffer j % 3
+    uint64_t* s_full = bars + 13;    // [3]  S of tile T is in TMEM buffer T % 3
     uint64_t* p_full = bars + 16;    // [2]  group g has written P of its tile
-    uint64_t* pv_done = bars + 18;   // [2]  P_j V_j has completed (index j & 1)
+    uint64_t* pv_done = bars + 18;   // [2]  P V of a tile of group g has completed
     uint64_t* max_done = bars + 20;  // [2]  group g has published the reference maxima of its tile
-    uint64_t* all_done = bars + 22;  // every MMA has completed
+    uint64_t* all_done = bars + 22;  // every MMA of the item has completed
     uint64_t* l_ready = bars + 23;   // both groups have stored their row sums
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
+    uint64_t* o_empty = bars + 24;   // both groups have drained O
+    ItemRing ring{bars + 25, bars + 27, reinterpret_cast<volatile int*>(bars + 29)};
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 30);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
     float* mref = reinterpret_cast<float*>(smem + L::kMref);
     float* lsum = reinterpret_cast<float*>(smem + L::kLsum);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_q_tiles = (args.S + 127) / 128;
-    const int q_tile = n_q_tiles - 1 - static_cast<int>(blockIdx.x);   // longest rows first
-    const int head = blockIdx.y;
-    const int q0 = q_tile * 128;
-    const int n_keys = kCausal ? min(q0 + 128, args.S) : args.S;       // keys any row of this tile attends to
-    const int n_kv = (n_keys + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         mbar_init(q_ready, 128);
@@ -104,13 +108,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&p_full[s], 128); mbar_init(&pv_done[s], 1); mbar_init(&max_done[s], 128);
+            mbar_init(&ring.full[s], 1); mbar_init(&ring.empty[s], 10);
         }
         mbar_init(all_done, 1);
         mbar_init(l_ready, 256);
+        mbar_init(o_empty, 256);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
+        if ((smem_u32(smem) & 1023u) != 0u) {   // the swizzled operand slabs need a 1024-byte aligned base
+            abort_flag->value = 1;
+            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD2u);
+        }
     }
+    clock_probe_begin(args.clock_probe);
     if (warp == 9) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
@@ -118,30 +129,57 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base + 3 * BK;       // [0,288) three S tiles | [288,416) O | [416,512) Q as packed bf16
     const uint32_t tmem_q = tmem_o + 128;
+    auto item_geometry = [&](int item, int& q0, int& head, int& n_kv) {
+        int rank;
+        decode_item(args.sched, item, rank, head);
+        q0 = (n_q_tiles - 1 - rank) * 128;                              // longest rows first
+        const int n_keys = kCausal ? min(q0 + 128, args.S) : args.S;    // keys any row of this tile attends to
+        n_kv = (n_keys + BK - 1) / BK;
+    };
 
-    if (warp == 8) {
+    if (abort_flag->value != 0u) {
+        // misaligned shared memory: nothing was started, fall through to the common exit
+    } else if (warp == 8) {
         // K and V have producers of their own: the score MMAs run up to three tiles ahead of the P V MMAs,
         // and a single thread waiting for a V stage would hold back the K tile the tensor pipe needs next.
         if (elect_one()) {
-            for (int j = 0; j < n_kv; ++j) {
-                const int s = j % kFwdStages;
-                if (!mbar_wait(&k_empty[s], ((j / kFwdStages) & 1) ^ 1, abort_flag, args.status, 0x10)) break;
-                uint8_t* dk = smem + L::kK + s * 3 * L::kSlab;
-                mbar_arrive_expect_tx(&k_full[s], 3 * L::kSlab);
-                tma_load_2d(dk, &tmap_kv, &k_full[s], head * 256, j * BK);
-                tma_load_2d(dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * BK);
-                tma_load_2d(dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * BK);
+            uint32_t T = 0;
+            bool ok = true;
+            for (uint32_t n = 0; ok; ++n) {
+                const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
+                if (!ok || item < 0) break;
+                int q0, head, n_kv;
+                item_geometry(item, q0, head, n_kv);
+                for (int j = 0; j < n_kv; ++j, ++T) {
+                    const uint32_t s = T % kFwdStages;
+                    ok = mbar_wait(&k_empty[s], ((T / kFwdStages) & 1u) ^ 1u, abort_flag, args.status, 0x10);
+                    if (!ok) break;
+                    uint8_t* dk = smem + L::kK + s * 3 * L::kSlab;
+                    mbar_arrive_expect_tx(&k_full[s], 3 * L::kSlab);
+                    tma_load_2d(dk, &tmap_kv, &k_full[s], head * 256, j * BK);
+                    tma_load_2d(dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * BK);
+                    tma_load_2d(dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * BK);
+                }
             }
         }
     } else if (warp == 10) {
         if (elect_one()) {
-            for (int j = 0; j < n_kv; ++j) {
-                const int s = j % kFwdStages;
-                if (!mbar_wait(&v_empty[s], ((j / kFwdStages) & 1) ^ 1, abort_flag, args.status, 0x11)) break;
-                uint8_t* dv = smem + L::kV + s * 2 * L::kSlab;
-                mbar_arrive_expect_tx(&v_full[s], 2 * L::kSlab);
-                tma_load_2d(dv, &tmap_kv, &v_full[s], head * 256 + 128, j * BK);
-                tma_load_2d(dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * BK);
+            uint32_t T = 0;
+            bool ok = true;
+            for (uint32_t n = 0; ok; ++n) {
+                const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
+                if (!ok || item < 0) break;
+                int q0, head, n_kv;
+                item_geometry(item, q0, head, n_kv);
+                for (int j = 0; j < n_kv; ++j, ++T) {
+                    const uint32_t s = T % kFwdStages;
+                    ok = mbar_wait(&v_empty[s], ((T / kFwdStages) & 1u) ^ 1u, abort_flag, args.status, 0x11);
+                    if (!ok) break;
+                    uint8_t* dv = smem + L::kV + s * 2 * L::kSlab;
+                    mbar_arrive_expect_tx(&v_full[s], 2 * L::kSlab);
+                    tma_load_2d(dv, &tmap_kv, &v_full[s], head * 256 + 128, j * BK);
+                    tma_load_2d(dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * BK);
+                }
             }
         }
     } else if (warp == 9) {
@@ -153,8 +191,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             // while the MMAs block, and the bounded wait runs only when the probe came back false.
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, BK, 0, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);
-            auto qk_mmas = [&](int j) {
-                const int s = j % kFwdStages;
+            auto qk_mmas = [&](uint32_t T) {
+                const uint32_t s = T % kFwdStages;
                 const uint32_t sk = smem_u32(smem + L::kK + s * 3 * L::kSlab);
 #pragma unroll
                 for (int kk = 0; kk < 12; ++kk)
@@ -163,172 +201,75 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 mma_commit(&k_empty[s]);
                 mma_commit(&s_full[s]);
             };
-            bool ok = mbar_wait(q_ready, 0, abort_flag, args.status, 0x22);
-            for (int j = 0; j < 3 && j < n_kv && ok; ++j) {
-                ok = mbar_wait(&k_full[j], 0, abort_flag, args.status, 0x23);
-                tc_fence_after_sync();
-                if (ok) qk_mmas(j);
-            }
-            bool v_ok = false, p_ok = false;      // probes of v_full / p_full for tile j
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const int s = j % kFwdStages, g = j & 1;
-                const uint32_t ph = (j / kFwdStages) & 1;
-                if (!v_ok) ok = mbar_wait(&v_full[s], ph, abort_flag, args.status, 0x20);
-                if (ok && !p_ok) ok = mbar_wait(&p_full[g], (j >> 1) & 1, abort_flag, args.status, 0x21);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const bool more = j + 3 < n_kv;
-                const bool k_ok = more && mbar_try_wait(&k_full[s], ph ^ 1);   // K_{j+3} lands in the stage K_j left
-                const uint32_t sv = smem_u32(smem + L::kV + s * 2 * L::kSlab);
-#pragma unroll
-                for (int kk = 0; kk < BK / 16; ++kk)   // A = P_j: packed bf16, 8 TMEM columns per 16 keys
-                    mma_ts(tmem_o, tmem_base + s * BK + kk * 8, desc_mn_major(sv + kk * 2048, L::kSlab), idesc_pv,
-                           (j > 0 || kk > 0) ? 1u : 0u);
-                mma_commit(&v_empty[s]);
-                mma_commit(&pv_done[g]);
-                v_ok = p_ok = false;
-                if (more) {
-                    if (!k_ok) ok = mbar_wait(&k_full[s], ph ^ 1, abort_flag, args.status, 0x23);
+            uint32_t T0 = 0;
+            bool ok = true;
+            for (uint32_t n = 0; ok; ++n) {
+                const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
+                if (!ok || item < 0) break;
+                int q0, head, n_kv;
+                item_geometry(item, q0, head, n_kv);
+                ok = mbar_wait(q_ready, n & 1u, abort_flag, args.status, 0x22);
+                for (int j = 0; j < 3 && j < n_kv && ok; ++j) {
+                    const uint32_t T = T0 + j;
+                    ok = mbar_wait(&k_full[T % kFwdStages], (T / kFwdStages) & 1u, abort_flag, args.status, 0x23);
+                    tc_fence_after_sync();
+                    if (ok) qk_mmas(T);
+                }
+                // the item's first P V overwrites O: the previous item's must have been drained
+                if (ok && n > 0) ok = mbar_wait(o_empty, (n - 1) & 1u, abort_flag, args.status, 0x24);
+                bool v_ok = false, p_ok = false;      // probes of v_full / p_full for tile j
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const uint32_t T = T0 + j;
+                    const uint32_t s = T % kFwdStages, g = T & 1u;
+                    const uint32_t ph = (T / kFwdStages) & 1u;
+                    if (!v_ok) ok = mbar_wait(&v_full[s], ph, abort_flag, args.status, 0x20);
+                    if (ok && !p_ok) ok = mbar_wait(&p_full[g], (T >> 1) & 1u, abort_flag, args.status, 0x21);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const int s1 = (j + 1) % kFwdStages;
-                    v_ok = mbar_try_wait(&v_full[s1], ((j + 1) / kFwdStages) & 1);
-                    p_ok = mbar_try_wait(&p_full[g ^ 1], ((j + 1) >> 1) & 1);
-                    qk_mmas(j + 3);
+                    const bool more = j + 3 < n_kv;
+                    const bool k_ok = more && mbar_try_wait(&k_full[s], ph ^ 1u);   // K of tile T+3 lands in the stage tile T left
+                    const uint32_t sv = smem_u32(smem + L::kV + s * 2 * L::kSlab);
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk)   // A = P: packed bf16, 8 TMEM columns per 16 keys
+                        mma_ts(tmem_o, tmem_base + s * BK + kk * 8, desc_mn_major(sv + kk * 2048, L::kSlab), idesc_pv,
+                               (j > 0 || kk > 0) ? 1u : 0u);
+                    mma_commit(&v_empty[s]);
+                    mma_commit(&pv_done[g]);
+                    v_ok = p_ok = false;
+                    if (more) {
+                        if (!k_ok) ok = mbar_wait(&k_full[s], ph ^ 1u, abort_flag, args.status, 0x23);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        v_ok = mbar_try_wait(&v_full[(T + 1) % kFwdStages], ((T + 1) / kFwdStages) & 1u);
+                        p_ok = mbar_try_wait(&p_full[g ^ 1u], ((T + 1) >> 1) & 1u);
+                        qk_mmas(T + 3);
+                    }
                 }
+                if (ok) mma_commit(all_done);
+                T0 += static_cast<uint32_t>(n_kv);
             }
-            if (ok) mma_commit(all_done);
         }
     } else {
-        const int g = warp >> 2;                      // softmax warpgroup: key tiles j with (j & 1) == g
+        const int g = warp >> 2;                      // softmax warpgroup: tiles whose running count has parity g
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;          // row inside the tile == TMEM lane
-        const int sq_idx = q0 + row;                  // global query index
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-        if (g == 0) {   // this thread's query row (192 bf16 = 96 packed words) goes to TMEM once, as the A operand of S
-            const bool q_valid = sq_idx < args.S;
-            const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(sq_idx) * args.h + head) * 192);
-#pragma unroll 1
-            for (int c = 0; c < 3; ++c) {
-                uint32_t w[32];
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                    const uint4 x = q_valid ? src[c * 8 + v] : make_uint4(0u, 0u, 0u, 0u);
-                    w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
-                }
-                __syncwarp();
-                tmem_st_x32(tmem_q + lane_addr + c * 32, w);
-            }
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(q_ready);
-        }
-        float m_mine = -INFINITY;                     // reference max (scaled, log2 domain) l_part refers to
-        float l_part = 0.f;                           // this group's part of the row sum
-        bool ok = true;
-        for (int j = g; j < n_kv; j += 2) {
-            const int b = j % kFwdStages;
-            const uint32_t tmem_s = tmem_base + lane_addr + b * BK;
-            ok = mbar_wait_warp(&s_full[b], (j / kFwdStages) & 1, abort_flag, args.status, 0x30);
-            if (!ok) break;
+        auto read_item = [&](uint32_t n, bool& ok) -> int {
+            ok = mbar_wait_warp(&ring.full[n & 1u], (n >> 1) & 1u, abort_flag, args.status, 0xA1);
+            if (!ok) return -1;
+            const int it = ring.item[n & 1u];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ring.empty[n & 1u]);
+            return it;
+        };
+        // O of a finished item (all of its MMAs are known complete): each group drains half of the columns
+        auto drain = [&](int sq_idx, int head, float m_fin, float l_run) {
             tc_fence_after_sync();
-            uint32_t sv[BK];
-#pragma unroll
-            for (int c = 0; c < BK / 32; ++c) tmem_ld_x32(tmem_s + c * 32, sv + c * 32);
-            tmem_ld_wait();
-
-            const int t_last = j * BK + BK - 1;
-            if ((kCausal && t_last > q0) || t_last >= args.S) {   // the causal edge can cross two tiles
-#pragma unroll
-                for (int c = 0; c < BK; ++c) {
-                    const int t = j * BK + c;
-                    if ((kCausal && t > sq_idx) || t >= args.S) sv[c] = __float_as_uint(-INFINITY);
-                }
-            }
-            // eight independent chains (three-input max: two elements per instruction)
-            float mxs[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) mxs[e] = fmaxf(__uint_as_float(sv[e]), __uint_as_float(sv[8 + e]));
-#pragma unroll
-            for (int c = 16; c < BK; c += 16)
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    mxs[e] = fmax3(mxs[e], __uint_as_float(sv[c + e]), __uint_as_float(sv[c + 8 + e]));
-            const float mx = fmaxf(fmax3(mxs[0], mxs[1], mxs[2]), fmax3(fmax3(mxs[3], mxs[4], mxs[5]), mxs[6], mxs[7]));
-
-            // The reference maximum as the other group left it after tile j-1.  Tile 0 holds an unmasked key
-            // for every row, so the reference is finite from there on; a later tile may be masked out for a
-            // row altogether (mx = -inf), which leaves the reference alone and yields P = 0.
-            float m_old = -INFINITY;
-            if (j > 0) {
-                ok = mbar_wait_warp(&max_done[g ^ 1], ((j - 1) >> 1) & 1, abort_flag, args.status, 0x33);
-                if (!ok) break;
-                m_old = mref[row];
-            }
-            const float m_cand = fmaxf(m_old, mx * args.scale_log2);
-            // Lazy rescale: keep the old reference unless it fell behind by more than 2^8.
-            const bool move = (m_cand - m_old) > 8.0f;
-            const float m_new = move ? m_cand : m_old;
-            if (move) mref[row] = m_new;
-            mbar_arrive(&max_done[g]);
-            const float alpha = move ? fast_exp2(m_old - m_new) : 1.0f;               // for O (all earlier tiles)
-            const float beta = (m_mine == m_new) ? 1.0f : fast_exp2(m_mine - m_new);   // for this group's sum
-            m_mine = m_new;
-
-            float sums[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            uint32_t pk[BK / 2];
-#pragma unroll
-            for (int c = 0; c < BK / 2; ++c) {
-                const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * c]), args.scale_log2, -m_new));
-                const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * c + 1]), args.scale_log2, -m_new));
-                sums[c & 7] += p0 + p1;
-                pk[c] = pack_bf16x2(p0, p1);
-            }
-            const float sum = ((sums[0] + sums[1]) + (sums[2] + sums[3])) + ((sums[4] + sums[5]) + (sums[6] + sums[7]));
-            l_part = l_part * beta + sum;
-
-            if (j > 0 && __any_sync(0xffffffffu, move)) {
-                // O must be at rest: P_{j-1} V_{j-1} finished (the previous phase of its barrier, tile j-3,
-                // is known complete because S_j was issued after it), P_j V_j not issued before p_full below.
-                ok = mbar_wait_warp(&pv_done[g ^ 1], ((j - 1) >> 1) & 1, abort_flag, args.status, 0x31);
-                if (!ok) break;
-                tc_fence_after_sync();
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int v = 0; v < 32; ++v) o[v] = __float_as_uint(__uint_as_float(o[v]) * alpha);
-                    tmem_st_x32(tmem_o + lane_addr + c * 32, o);
-                }
-            }
-            tmem_st_x32(tmem_s, pk);
-            tmem_st_x16(tmem_s + 32, pk + 32);
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(&p_full[g]);
-        }
-        // Bring this group's sum to the final reference (set by the owner of the last tile) and add the
-        // two groups' sums.
-        const int last = n_kv - 1;
-        if (ok && (last & 1) != g) ok = mbar_wait_warp(&max_done[g ^ 1], (last >> 1) & 1, abort_flag, args.status, 0x34);
-        float m_fin = 0.f;
-        if (ok) {
-            m_fin = mref[row];
-            lsum[g * 128 + row] = l_part * ((m_mine == m_fin) ? 1.0f : fast_exp2(m_mine - m_fin));
-            mbar_arrive(l_ready);
-            ok = mbar_wait_warp(l_ready, 0, abort_flag, args.status, 0x35);
-        }
-        if (ok) ok = mbar_wait_warp(all_done, 0, abort_flag, args.status, 0x32);
-        if (ok) {
-            tc_fence_after_sync();
-            const float l_run = lsum[row] + lsum[128 + row];
             const float inv_l = 1.0f / l_run;
             const bool valid = sq_idx < args.S;
             __nv_bfloat16* dst = args.out + (static_cast<size_t>(sq_idx) * args.h + head) * 128;
 #pragma unroll 1
-            for (int c = 2 * g; c < 2 * g + 2; ++c) {     // each group drains half of the O columns
+            for (int c = 2 * g; c < 2 * g + 2; ++c) {
                 uint32_t o[32];
                 __syncwarp();
                 tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
@@ -347,11 +288,156 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             }
             if (valid && g == 0)
                 args.lse[static_cast<size_t>(sq_idx) * args.h + head] = (m_fin + log2f(l_run)) * 0.6931471805599453f;
+            __syncwarp();
+            tc_fence_before_sync();
+            mbar_arrive(o_empty);
+        };
+        uint32_t T0 = 0;
+        bool ok = true;
+        int item = read_item(0, ok);
+        int prev_sq_idx = 0, prev_head = 0;
+        float prev_m_fin = 0.f, prev_l_run = 1.f;
+        for (uint32_t n = 0; ok && item >= 0; ++n) {
+            int q0, head, n_kv;
+            item_geometry(item, q0, head, n_kv);
+            const int sq_idx = q0 + row;              // global query index
+            if (g == 0) {   // this thread's query row (192 bf16 = 96 packed words) goes to TMEM once, as the A operand of S
+                            // (the previous item's MMAs, which read the old tile, are known complete)
+                const bool q_valid = sq_idx < args.S;
+                const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(sq_idx) * args.h + head) * 192);
+#pragma unroll 1
+                for (int c = 0; c < 3; ++c) {
+                    uint32_t w[32];
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const uint4 x = q_valid ? src[c * 8 + v] : make_uint4(0u, 0u, 0u, 0u);
+                        w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
+                    }
+                    __syncwarp();
+                    tmem_st_x32(tmem_q + lane_addr + c * 32, w);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(q_ready);
+            }
+            if (n > 0) drain(prev_sq_idx, prev_head, prev_m_fin, prev_l_run);
+            float m_mine = -INFINITY;                     // reference max (scaled, log2 domain) l_part refers to
+            float l_part = 0.f;                           // this group's part of the row sum
+            for (int j = 0; j < n_kv; ++j) {
+                const uint32_t T = T0 + j;
+                if ((T & 1u) != static_cast<uint32_t>(g)) continue;
+                const uint32_t b = T % kFwdStages;
+                const uint32_t tmem_s = tmem_base + lane_addr + b * BK;
+                ok = mbar_wait_warp(&s_full[b], (T / kFwdStages) & 1u, abort_flag, args.status, 0x30);
+                if (!ok) break;
+                tc_fence_after_sync();
+                uint32_t sv[BK];
+#pragma unroll
+                for (int c = 0; c < BK / 32; ++c) tmem_ld_x32(tmem_s + c * 32, sv + c * 32);
+                tmem_ld_wait();
+
+                const int t_last = j * BK + BK - 1;
+                if ((kCausal && t_last > q0) || t_last >= args.S) {   // the causal edge can cross two tiles
+#pragma unroll
+                    for (int c = 0; c < BK; ++c) {
+                        const int t = j * BK + c;
+                        if ((kCausal && t > sq_idx) || t >= args.S) sv[c] = __float_as_uint(-INFINITY);
+                    }
+                }
+                // eight independent chains (three-input max: two elements per instruction)
+                float mxs[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) mxs[e] = fmaxf(__uint_as_float(sv[e]), __uint_as_float(sv[8 + e]));
+#pragma unroll
+                for (int c = 16; c < BK; c += 16)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        mxs[e] = fmax3(mxs[e], __uint_as_float(sv[c + e]), __uint_as_float(sv[c + 8 + e]));
+                const float mx = fmaxf(fmax3(mxs[0], mxs[1], mxs[2]), fmax3(fmax3(mxs[3], mxs[4], mxs[5]), mxs[6], mxs[7]));
+
+                // The reference maximum as the other group left it after the item's previous tile.  The item's
+                // first tile holds an unmasked key for every row, so the reference is finite from there on; a
+                // later tile may be masked out for a row altogether (mx = -inf), which leaves the reference alone
+                // and yields P = 0.
+                float m_old = -INFINITY;
+                if (j > 0) {
+                    ok = mbar_wait_warp(&max_done[g ^ 1], ((T - 1) >> 1) & 1u, abort_flag, args.status, 0x33);
+                    if (!ok) break;
+                    m_old = mref[row];
+                }
+                const float m_cand = fmaxf(m_old, mx * args.scale_log2);
+                // Lazy rescale: keep the old reference unless it fell behind by more than 2^8.
+                const bool move = (m_cand - m_old) > 8.0f;
+                const float m_new = move ? m_cand : m_old;
+                if (move) mref[row] = m_new;
+                mbar_arrive(&max_done[g]);
+                const float alpha = move ? fast_exp2(m_old - m_new) : 1.0f;               // for O (all earlier tiles)
+                const float beta = (m_mine == m_new) ? 1.0f : fast_exp2(m_mine - m_new);   // for this group's sum
+                m_mine = m_new;
+
+                float sums[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                uint32_t pk[BK / 2];
+#pragma unroll
+                for (int c = 0; c < BK / 2; ++c) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * c]), args.scale_log2, -m_new));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * c + 1]), args.scale_log2, -m_new));
+                    sums[c & 7] += p0 + p1;
+                    pk[c] = pack_bf16x2(p0, p1);
+                }
+                const float sum = ((sums[0] + sums[1]) + (sums[2] + sums[3])) + ((sums[4] + sums[5]) + (sums[6] + sums[7]));
+                l_part = l_part * beta + sum;
+
+                if (j > 0 && __any_sync(0xffffffffu, move)) {
+                    // O must be at rest: P V of the previous tile finished (the previous phase of its barrier, tile
+                    // T-3, is known complete because S of this tile was issued after it), P V of this tile is not
+                    // issued before p_full below.
+                    ok = mbar_wait_warp(&pv_done[g ^ 1], ((T - 1) >> 1) & 1u, abort_flag, args.status, 0x31);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int v = 0; v < 32; ++v) o[v] = __float_as_uint(__uint_as_float(o[v]) * alpha);
+                        tmem_st_x32(tmem_o + lane_addr + c * 32, o);
+                    }
+                }
+                tmem_st_x32(tmem_s, pk);
+                tmem_st_x16(tmem_s + 32, pk + 32);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(&p_full[g]);
+            }
+            if (!ok) break;
+            // Bring this group's sum to the final reference (set by the owner of the item's last tile) and add
+            // the two groups' sums.
+            const uint32_t last = T0 + static_cast<uint32_t>(n_kv) - 1u;
+            if ((last & 1u) != static_cast<uint32_t>(g))
+                ok = mbar_wait_warp(&max_done[g ^ 1], (last >> 1) & 1u, abort_flag, args.status, 0x34);
+            if (!ok) break;
+            const float m_fin = mref[row];
+            float* lsum_n = lsum + (n & 1u) * 256;
+            lsum_n[g * 128 + row] = l_part * ((m_mine == m_fin) ? 1.0f : fast_exp2(m_mine - m_fin));
+            mbar_arrive(l_ready);
+            ok = mbar_wait_warp(l_ready, n & 1u, abort_flag, args.status, 0x35);
+            if (!ok) break;
+            prev_l_run = lsum_n[row] + lsum_n[128 + row];
+            prev_m_fin = m_fin;
+            prev_sq_idx = sq_idx;
+            prev_head = head;
+            ok = mbar_wait_warp(all_done, n & 1u, abort_flag, args.status, 0x32);
+            if (!ok) break;
+            T0 += static_cast<uint32_t>(n_kv);
+            item = read_item(n + 1, ok);
+            if (ok && item < 0) drain(prev_sq_idx, prev_head, prev_m_fin, prev_l_run);
         }
     }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 9) { tc_fence_after_sync(); tmem_dealloc(tmem_base, 512); }
+    clock_probe_end(args.clock_probe);
 }
 
 }  // namespace laga

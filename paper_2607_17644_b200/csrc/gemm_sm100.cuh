@@ -22,6 +22,8 @@ struct GemmArgs {
     void* C;              // bf16 [M, ldc] (EPI_BF16) or fp32 [M, ldc] (EPI_ATOMIC_F32)
     int ldc;
     unsigned int* status;
+    float4* zero_begin;   // optional: zero_count float4 elements cleared by this launch before it starts
+    size_t zero_count;    // (the buffer the NEXT kernel accumulates into: saves a separate memset)
 };
 
 enum { EPI_BF16 = 0, EPI_ATOMIC_F32 = 1 };
@@ -66,6 +68,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tma_prefetch_desc(&tmap_b);
     }
     if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+    for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < args.zero_count;
+         z += static_cast<size_t>(gridDim.x) * blockDim.x)
+        args.zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();

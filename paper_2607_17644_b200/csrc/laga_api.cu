@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <initializer_list>
+#include <mutex>
 #include <vector>
 
 #include "attn_bwd_sm100.cuh"
@@ -59,31 +61,93 @@ bool make_tmap_bf16(CUtensorMap* map, const void* base, uint64_t inner_elems, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int check_device() {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return LAGA_ERR_CUDA;
-    static int cached_dev = -1, cached_major = 0;
-    if (cached_dev != dev) {
-        int major = 0;
-        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-            return LAGA_ERR_CUDA;
-        cached_dev = dev;
-        cached_major = major;
-    }
-    return cached_major == 10 ? LAGA_OK : LAGA_ERR_UNSUPPORTED;
+// ---- launch status slot ---------------------------------------------------------------------------
+// The first kStatusBytes of every workspace: word 0 is the device status word; the work counters of the
+// persistent attention kernels and their clock probes follow.  The first kStatusClearBytes (all of
+// that) are cleared at the start of every entry point.
+constexpr size_t kStatusClearBytes = 256;
+constexpr size_t kCounterOffsetWords = 4;     // words 4, 5, 6: forward, dK/dV and dQ kernel work counters
+constexpr size_t kProbeOffsetBytes = 64;      // three ClockProbe records (forward, dK/dV, dQ)
+enum { kSlotFwd = 0, kSlotDkv = 1, kSlotDq = 2 };
+
+unsigned* slot_counter(unsigned* status, int slot) { return status + kCounterOffsetWords + slot; }
+ClockProbe* slot_probe(unsigned* status, int slot) {
+    return reinterpret_cast<ClockProbe*>(reinterpret_cast<uint8_t*>(status) + kProbeOffsetBytes) + slot;
 }
 
-// Number of SMs of the current device (cached per device); 148 if the query fails.
+int launch_status() { return cudaGetLastError() == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA; }
+
+// ---- per-device facts, looked up once per device (thread-safe) ------------------------------------
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+    std::once_flag once;
+    int rc = LAGA_ERR_CUDA;
+    int sms = 148;
+    std::once_flag scratch_once;
+    unsigned char* builtin_scratch = nullptr;
+};
+DeviceInfo g_devices[kMaxDevices];
+
+template <typename Kernel>
+bool allow_smem(Kernel kernel, int bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+void init_device(DeviceInfo* info, int dev) {
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return;
+    if (major != 10) { info->rc = LAGA_ERR_UNSUPPORTED; return; }
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) info->sms = sms;
+    // every kernel of the library asks for more than the default 48 KB of dynamic shared memory: opt in once
+    using G = GemmSmem<256, 4>;
+    bool ok = allow_smem(gemm_sm100_kernel<256, 4, false, true, EPI_BF16>, G::kTotalBytes) &&
+              allow_smem(gemm_sm100_kernel<256, 4, false, false, EPI_BF16>, G::kTotalBytes) &&
+              allow_smem(gemm_sm100_kernel<256, 4, true, true, EPI_ATOMIC_F32>, G::kTotalBytes) &&
+              allow_smem(attn_fwd_sm100_kernel<true>, AttnFwdSmem::kTotalBytes) &&
+              allow_smem(attn_fwd_sm100_kernel<false>, AttnFwdSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_dkv_sm100_kernel<true>, AttnBwdDkvSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_dkv_sm100_kernel<false>, AttnBwdDkvSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_dq_sm100_kernel<true>, AttnBwdDqSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_dq_sm100_kernel<false>, AttnBwdDqSmem::kTotalBytes);
+    info->rc = ok ? LAGA_OK : LAGA_ERR_CUDA;
+    if (!ok) (void)cudaGetLastError();
+}
+
+// The current device's record; LAGA_ERR_UNSUPPORTED if it is not an sm_100 part.
+int current_device(DeviceInfo** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LAGA_ERR_CUDA;
+    DeviceInfo* info = &g_devices[dev];
+    std::call_once(info->once, init_device, info, dev);
+    *out = info;
+    return info->rc;
+}
+
+int check_device() {
+    DeviceInfo* info = nullptr;
+    return current_device(&info);
+}
+
 int sm_count() {
-    static int cached_dev = -1, cached_sms = 148;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cached_dev != dev) {
-        int sms = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) cached_sms = sms;
-        cached_dev = dev;
+    DeviceInfo* info = nullptr;
+    return current_device(&info) == LAGA_OK ? info->sms : 148;
+}
+
+// Every data pointer must be device memory of the CURRENT device (or managed memory): a kernel given
+// another device's pointer would fault, or silently use the wrong memory where peers are mapped.
+int check_pointers(std::initializer_list<const void*> ptrs) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LAGA_ERR_CUDA;
+    for (const void* p : ptrs) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return LAGA_ERR_INVALID_ARG;
+        }
+        if (attr.type == cudaMemoryTypeManaged) continue;
+        if (attr.type != cudaMemoryTypeDevice || attr.device != dev) return LAGA_ERR_INVALID_ARG;
     }
-    return cached_sms;
+    return LAGA_OK;
 }
 
 // Persistent kernels launch one CTA per SM (fewer if there are fewer tiles).
@@ -92,27 +156,57 @@ unsigned persistent_grid(int total_tiles) {
     return static_cast<unsigned>(total_tiles < sms ? (total_tiles < 1 ? 1 : total_tiles) : sms);
 }
 
-template <typename Kernel>
-int set_smem(Kernel kernel, int bytes) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
-               ? LAGA_OK
-               : LAGA_ERR_CUDA;
+// ---- tensor-map cache ------------------------------------------------------------------------------
+// Encoding a tensor map is a driver call of a microsecond or two and an entry point needs up to five; for
+// short sequences that is a visible part of the host time per call.  A map is a pure function of
+// (base, extents, stride, box), so recently used ones are kept (64 entries, replaced round-robin).
+struct TmapKey {
+    const void* base;
+    uint64_t inner, rows, stride;
+    uint32_t box_rows;
+    bool operator==(const TmapKey& o) const {
+        return base == o.base && inner == o.inner && rows == o.rows && stride == o.stride && box_rows == o.box_rows;
+    }
+};
+struct TmapCache {
+    static constexpr int kEntries = 64;
+    std::mutex mutex;
+    TmapKey keys[kEntries] = {};
+    CUtensorMap maps[kEntries];
+    bool used[kEntries] = {};
+    int next = 0;
+};
+TmapCache g_tmaps;
+
+bool cached_tmap_bf16(CUtensorMap* map, const void* base, uint64_t inner_elems, uint64_t rows, uint64_t row_stride_bytes,
+                      uint32_t box_rows) {
+    const TmapKey key{base, inner_elems, rows, row_stride_bytes, box_rows};
+    std::lock_guard<std::mutex> lock(g_tmaps.mutex);
+    for (int i = 0; i < TmapCache::kEntries; ++i)
+        if (g_tmaps.used[i] && g_tmaps.keys[i] == key) { *map = g_tmaps.maps[i]; return true; }
+    if (!make_tmap_bf16(map, base, inner_elems, rows, row_stride_bytes, box_rows)) return false;
+    const int slot = g_tmaps.next;
+    g_tmaps.next = (slot + 1) % TmapCache::kEntries;
+    g_tmaps.keys[slot] = key;
+    g_tmaps.maps[slot] = *map;
+    g_tmaps.used[slot] = true;
+    return true;
 }
 
-int launch_status() { return cudaGetLastError() == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA; }
-
-// Measurement aid (laga_profile_kernel): caller-provided CUDA events recorded around launches of one
-// kernel, cycling through the registered pairs.
+// ---- measurement aid (laga_profile_kernel) ---------------------------------------------------------
+// Caller-provided CUDA events recorded around launches of one kernel, cycling through the registered pairs.
 struct ProfileSlot {
     std::vector<cudaEvent_t> starts, stops;
     unsigned long long launches = 0;
 };
 ProfileSlot g_profile[LAGA_KERNEL_COUNT];
+std::mutex g_profile_mutex;
 
 struct ScopedKernelEvents {
     cudaEvent_t stop = nullptr;
     cudaStream_t stream;
     ScopedKernelEvents(int kernel_id, cudaStream_t st) : stream(st) {
+        std::lock_guard<std::mutex> lock(g_profile_mutex);
         ProfileSlot& slot = g_profile[kernel_id];
         if (!slot.starts.empty()) {
             const size_t i = static_cast<size_t>(slot.launches++ % slot.starts.size());
@@ -125,6 +219,17 @@ struct ScopedKernelEvents {
     }
 };
 
+// How many of the h heads the persistent attention kernels sweep position by position instead of head by
+// head (see work_sched.cuh): as many as keep the swept heads' streamed operands (640 bytes per token and
+// head: K_nope, V and the rope band on one side, Q and dO on the other) within half of the 126 MB L2.
+WorkSchedule make_schedule(int n_tiles, int S, int h, unsigned* counter) {
+    const long long per_head = static_cast<long long>(S) * 640;
+    long long banded = (64ll << 20) / (per_head > 0 ? per_head : 1);
+    if (banded < 1) banded = 1;
+    if (banded > h) banded = h;
+    return WorkSchedule{n_tiles, h, static_cast<int>(banded), n_tiles * h, counter};
+}
+
 // ---- Algorithm 1 step 4: KV[S, N] = c_kv[S, d_c] . W[d_c, N] ------------------------------------
 int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
                       cudaStream_t stream) {
@@ -132,10 +237,9 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
     auto kernel = gemm_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
     using L = GemmSmem<BN, STAGES>;
     CUtensorMap ta, tb;
-    if (!make_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
-    if (!make_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
-    if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-    GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status};
+    if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
+    if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
+    GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status, nullptr, 0};
     dim3 grid(persistent_grid((N / BN) * ((S + 127) / 128)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
@@ -143,35 +247,33 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
 
 // ---- Section 5.2, back through step 4 -----------------------------------------------------------
 // dc_kv[S, d_c] = dKV[S, N] . W^T          (A = dKV K-major, B = W rows d_c / inner N: K-major)
-int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, unsigned* status,
-                cudaStream_t stream) {
+// `clear` (optional) is an fp32 buffer of clear_floats elements this launch zeroes on its way in: the dW
+// GEMM that follows accumulates into it with atomics.
+int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float* clear, size_t clear_floats,
+                unsigned* status, cudaStream_t stream) {
     constexpr int BN = 256, STAGES = 4;
     auto kernel = gemm_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
     using L = GemmSmem<BN, STAGES>;
     CUtensorMap ta, tb;
-    if (!make_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
-    if (!make_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN)) return LAGA_ERR_CUDA;
-    if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-    GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status};
+    if (!cached_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN)) return LAGA_ERR_CUDA;
+    GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status, reinterpret_cast<float4*>(clear), clear_floats / 4};
     dim3 grid(persistent_grid((kDc / BN) * ((S + 127) / 128)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
 
-// dW[d_c, N] (+)= c_kv^T . dKV   (both operands read with the token index as K: MN-major), split over
-// the sequence with fp32 atomic accumulation.
-int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool accumulate, bool deterministic,
+// dW[d_c, N] += c_kv^T . dKV   (both operands read with the token index as K: MN-major), split over
+// the sequence with fp32 atomic accumulation into a buffer the caller of this function has cleared
+// (launch_dckv does it) or wants added to.
+int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool deterministic,
               unsigned* status, cudaStream_t stream) {
     constexpr int BN = 256, STAGES = 4;
     auto kernel = gemm_sm100_kernel<BN, STAGES, true, true, EPI_ATOMIC_F32>;
     using L = GemmSmem<BN, STAGES>;
     CUtensorMap ta, tb;
-    if (!make_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 64)) return LAGA_ERR_CUDA;
-    if (!make_tmap_bf16(&tb, dkv, N, S, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;
-    if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-    if (!accumulate &&
-        cudaMemsetAsync(dw, 0, sizeof(float) * static_cast<size_t>(kDc) * N, stream) != cudaSuccess)
-        return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 64)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tb, dkv, N, S, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;
     // Split the sequence so that tiles x splits fills whole waves of the persistent grid: the smallest
     // split count (fewest atomics) whose last wave is at least 90 % full, else the best found.
     const int tiles = (kDc / 128) * (N / BN);
@@ -187,7 +289,7 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool a
     }
     const int per_split = (k_tiles + splits - 1) / splits;
     splits = (k_tiles + per_split - 1) / per_split;
-    GemmArgs a{kDc, N, S, per_split, splits, dw, N, status};
+    GemmArgs a{kDc, N, S, per_split, splits, dw, N, status, nullptr, 0};
     dim3 grid(persistent_grid(tiles * splits), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
@@ -199,20 +301,16 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
     using L = AttnFwdSmem;
     const int N = h * (kDn + kDv);
     CUtensorMap tkv, tpe;   // boxes of 64 columns x one key tile of rows
-    if (!make_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, kFwdKeys)) return LAGA_ERR_CUDA;
-    if (!make_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, kFwdKeys)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, kFwdKeys)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, kFwdKeys)) return LAGA_ERR_CUDA;
+    const int n_tiles = (S + 127) / 128;
     AttnFwdArgs a{S, h, softmax_scale * 1.4426950408889634f, reinterpret_cast<const __nv_bfloat16*>(q),
-                  reinterpret_cast<__nv_bfloat16*>(out), lse, status};
-    dim3 grid((S + 127) / 128, h, 1);
-    if (causal) {
-        auto kernel = attn_fwd_sm100_kernel<true>;
-        if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a); }
-    } else {
-        auto kernel = attn_fwd_sm100_kernel<false>;
-        if (set_smem(kernel, L::kTotalBytes) != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream); kernel<<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a); }
-    }
+                  reinterpret_cast<__nv_bfloat16*>(out), lse, status,
+                  make_schedule(n_tiles, S, h, slot_counter(status, kSlotFwd)), slot_probe(status, kSlotFwd)};
+    dim3 grid(persistent_grid(n_tiles * h), 1, 1);
+    ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream);
+    if (causal) attn_fwd_sm100_kernel<true><<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a);
+    else attn_fwd_sm100_kernel<false><<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a);
     return launch_status();
 }
 
@@ -245,45 +343,40 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
                     cudaStream_t stream) {
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
-    {   // delta and the transposed, padded softmax statistics
+    {   // delta and the transposed, padded softmax statistics; clears the rope-gradient accumulator on the way
         const long long items = static_cast<long long>(S_pad) * h;   // eight lanes per (row, head)
         const unsigned blocks = static_cast<unsigned>((items * 8 + 255) / 256);
         ScopedKernelEvents ev(LAGA_KERNEL_BWD_DELTA, stream);
         bwd_delta_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(out),
                                                      reinterpret_cast<const __nv_bfloat16*>(dout), lse, S, h, S_pad,
-                                                     stat_l2, stat_delta);
+                                                     stat_l2, stat_delta, reinterpret_cast<float4*>(dkpe_acc),
+                                                     static_cast<size_t>(S) * kDr / 4);
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     }
-    if (cudaMemsetAsync(dkpe_acc, 0, static_cast<size_t>(S) * kDr * sizeof(float), stream) != cudaSuccess)
-        return LAGA_ERR_CUDA;
     const uint64_t q_row = static_cast<uint64_t>(h) * 192, do_row = static_cast<uint64_t>(h) * 128;
-    CUtensorMap tq, tkv, tpe, tq64, tdo64;   // boxes of 64 columns x 128 rows (x 64 rows for the dkv query tiles)
-    if (!make_tmap_bf16(&tq, q, q_row, S, q_row * 2, 128) || !make_tmap_bf16(&tq64, q, q_row, S, q_row * 2, 64) ||
-        !make_tmap_bf16(&tdo64, dout, do_row, S, do_row * 2, 64) ||
-        !make_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, 128) ||
-        !make_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, 128))
+    CUtensorMap tq, tkv, tpe, tdo;   // boxes of 64 columns x 128 rows
+    if (!cached_tmap_bf16(&tq, q, q_row, S, q_row * 2, 128) || !cached_tmap_bf16(&tdo, dout, do_row, S, do_row * 2, 128) ||
+        !cached_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, 128) ||
+        !cached_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, 128))
         return LAGA_ERR_CUDA;
-    dim3 grid((S + 127) / 128, h, 1);
+    const int n_tiles = (S + 127) / 128;
+    dim3 grid(persistent_grid(n_tiles * h), 1, 1);
     AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
-                     reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, dk_rope_per_head, status};
+                     reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, dk_rope_per_head, status,
+                     make_schedule(n_tiles, S, h, slot_counter(status, kSlotDkv)), slot_probe(status, kSlotDkv)};
     AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad,
-                    reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status};
-    if (causal) {
-        auto k1 = attn_bwd_dkv_sm100_kernel<true>;
-        auto k2 = attn_bwd_dq_sm100_kernel<true>;
-        if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
-            return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv, tpe, a); }
-        if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b); }
-    } else {
-        auto k1 = attn_bwd_dkv_sm100_kernel<false>;
-        auto k2 = attn_bwd_dq_sm100_kernel<false>;
-        if (set_smem(k1, AttnBwdDkvSmem::kTotalBytes) != LAGA_OK || set_smem(k2, AttnBwdDqSmem::kTotalBytes) != LAGA_OK)
-            return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream); k1<<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq64, tdo64, tkv, tpe, a); }
-        if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-        { ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream); k2<<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b); }
+                    reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status,
+                    make_schedule(n_tiles, S, h, slot_counter(status, kSlotDq)), slot_probe(status, kSlotDq)};
+    {
+        ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream);
+        if (causal) attn_bwd_dkv_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
+        else attn_bwd_dkv_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
+    }
+    if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+    {
+        ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream);
+        if (causal) attn_bwd_dq_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
+        else attn_bwd_dq_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     {
@@ -317,7 +410,12 @@ __global__ void selftest_bounded_wait_kernel(unsigned* status, unsigned long lon
     if (ok && threadIdx.x == 0) atomicExch(status, 0xdeadu);   // cannot happen: nothing arrives
 }
 
-int zero_status(void* status_word, cudaStream_t stream) {
+// Clears the status word and the work counters of a workspace's status slot.
+int zero_status(void* status_slot, cudaStream_t stream) {
+    return cudaMemsetAsync(status_slot, 0, kStatusClearBytes, stream) == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA;
+}
+// A bare status word handed to a step entry point (no counters behind it).
+int zero_status_word(void* status_word, cudaStream_t stream) {
     return cudaMemsetAsync(status_word, 0, sizeof(unsigned), stream) == cudaSuccess ? LAGA_OK : LAGA_ERR_CUDA;
 }
 
@@ -325,7 +423,7 @@ int zero_status(void* status_word, cudaStream_t stream) {
 
 extern "C" {
 
-int laga_version(void) { return 100; }
+int laga_version(void) { return 200; }
 
 const char* laga_status_string(int status) {
     switch (status) {
@@ -335,6 +433,7 @@ const char* laga_status_string(int status) {
         case LAGA_ERR_WORKSPACE_TOO_SMALL: return "LAGA_ERR_WORKSPACE_TOO_SMALL";
         case LAGA_ERR_CUDA: return "LAGA_ERR_CUDA";
         case LAGA_ERR_DEVICE_TIMEOUT: return "LAGA_ERR_DEVICE_TIMEOUT";
+        case LAGA_ERR_DEVICE_CHECK: return "LAGA_ERR_DEVICE_CHECK";
         default: return "LAGA_ERR_UNKNOWN";
     }
 }
@@ -356,8 +455,9 @@ int laga_up_project(const void* c_kv, const void* w_kv_b, int S, int h, int d_c,
     if (!geometry_supported(d_c, d_nope, kDr, d_v)) return LAGA_ERR_UNSUPPORTED;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({c_kv, w_kv_b, kv, status_word})) != LAGA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((rc = zero_status(status_word, st)) != LAGA_OK) return rc;
+    if ((rc = zero_status_word(status_word, st)) != LAGA_OK) return rc;
     return launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, static_cast<unsigned*>(status_word), st);
 }
 
@@ -371,13 +471,16 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
     if (!geometry_supported(d_c, d_nope, kDr, d_v)) return LAGA_ERR_UNSUPPORTED;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({dkv, c_kv, w_kv_b, dc_kv, dw_kv_b, status_word})) != LAGA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned* status = static_cast<unsigned*>(status_word);
     const int N = h * (kDn + kDv);
-    if ((rc = zero_status(status_word, st)) != LAGA_OK) return rc;
-    if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
-    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0,
-                     (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st);
+    const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
+    if ((rc = zero_status_word(status_word, st)) != LAGA_OK) return rc;
+    if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,
+                          accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st)) != LAGA_OK)
+        return rc;
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st);
 }
 
 int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
@@ -394,6 +497,7 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
         return LAGA_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({q, c_kv, k_pe, w_kv_b, out, lse, workspace})) != LAGA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned* status = static_cast<unsigned*>(workspace);
     void* kv = static_cast<uint8_t*>(workspace) + kStatusBytes;
@@ -417,10 +521,13 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
         return LAGA_ERR_INVALID_ARG;
     if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
     const bool deterministic = (flags & LAGA_FLAG_DETERMINISTIC) != 0;
+    const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
     const BwdWorkspace w = bwd_workspace_layout(S, h, deterministic);
     if (workspace_bytes < w.total) return LAGA_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({q, c_kv, k_pe, w_kv_b, out, lse, dout, dq, dc_kv, dk_pe, dw_kv_b, workspace})) != LAGA_OK)
+        return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t* base = static_cast<uint8_t*>(workspace);
     unsigned* status = reinterpret_cast<unsigned*>(base);
@@ -437,8 +544,10 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
                               deterministic ? reinterpret_cast<float*>(base + w.dk_rope_per_head) : nullptr, w.S_pad, status,
                               st)) != LAGA_OK)
         return rc;
-    if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, status, st)) != LAGA_OK) return rc;
-    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_ACCUM_DW) != 0, deterministic, status, st);
+    if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,
+                          accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st)) != LAGA_OK)
+        return rc;
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, deterministic, status, st);
 }
 
 // ---- forward without caller-provided scratch ----------------------------------------------------
@@ -451,20 +560,22 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kStatusBytes + 
 // Device address of g_builtin_scratch on the current device.  In host code the symbol's name is only
 // a handle, never an address a kernel may use: the address comes from cudaGetSymbolAddress, looked up
 // once per device with that device current.
-static int builtin_scratch_address(unsigned char** ptr) {
-    constexpr int kMaxDevices = 64;
-    static unsigned char* cached[kMaxDevices] = {};
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LAGA_ERR_CUDA;
-    if (!cached[dev]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) {
-            (void)cudaGetLastError();
-            return LAGA_ERR_CUDA;
-        }
-        cached[dev] = static_cast<unsigned char*>(p);
+static void lookup_builtin_scratch(DeviceInfo* info) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) {
+        (void)cudaGetLastError();
+        return;
     }
-    *ptr = cached[dev];
+    info->builtin_scratch = static_cast<unsigned char*>(p);
+}
+
+static int builtin_scratch_address(unsigned char** ptr) {
+    DeviceInfo* info = nullptr;
+    const int rc = current_device(&info);
+    if (rc != LAGA_OK) return rc;
+    std::call_once(info->scratch_once, lookup_builtin_scratch, info);
+    if (!info->builtin_scratch) return LAGA_ERR_CUDA;
+    *ptr = info->builtin_scratch;
     return LAGA_OK;
 }
 
@@ -481,13 +592,15 @@ int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, 
     if (static_cast<size_t>(S) * h * (kDn + kDv) * 2 > kBuiltinKvBytes) return LAGA_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({q, c_kv, k_pe, w_kv_b, out, lse})) != LAGA_OK) return rc;
     unsigned char* base = nullptr;
     if ((rc = builtin_scratch_address(&base)) != LAGA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned* status = reinterpret_cast<unsigned*>(base);
     void* kv = base + kStatusBytes;
-    // The array keeps whatever the previous call left: the status word must start at zero; KV rows
-    // [0, S) are fully overwritten by the up-projection before the attention kernel reads them.
+    // The array keeps whatever the previous call left: the status slot (status word and work counter) must
+    // start at zero; KV rows [0, S) are fully overwritten by the up-projection before the attention kernel
+    // reads them.
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
     if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
     return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st);
@@ -498,7 +611,7 @@ int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stre
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if ((rc = zero_status(status_word, st)) != LAGA_OK) return rc;
+    if ((rc = zero_status_word(status_word, st)) != LAGA_OK) return rc;
     selftest_bounded_wait_kernel<<<1, 64, 0, st>>>(static_cast<unsigned*>(status_word),
                                                    static_cast<unsigned long long>(budget_us) * 1000ull);
     return launch_status();
@@ -507,14 +620,36 @@ int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stre
 int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs) {
     if (kernel_id < 0 || kernel_id >= LAGA_KERNEL_COUNT || n_pairs < 0) return LAGA_ERR_INVALID_ARG;
     if (n_pairs > 0 && (!start_events || !stop_events)) return LAGA_ERR_INVALID_ARG;
+    for (int i = 0; i < n_pairs; ++i)
+        if (!start_events[i] || !stop_events[i]) return LAGA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
     ProfileSlot& slot = g_profile[kernel_id];
     slot.starts.clear();
     slot.stops.clear();
     slot.launches = 0;
     for (int i = 0; i < n_pairs; ++i) {
-        if (!start_events[i] || !stop_events[i]) { slot.starts.clear(); slot.stops.clear(); return LAGA_ERR_INVALID_ARG; }
         slot.starts.push_back(static_cast<cudaEvent_t>(start_events[i]));
         slot.stops.push_back(static_cast<cudaEvent_t>(stop_events[i]));
+    }
+    return LAGA_OK;
+}
+
+int laga_query_kernel_clocks(const void* workspace, void* stream, double* sm_mhz, double* kernel_ms) {
+    if (!workspace || !sm_mhz || !kernel_ms) return LAGA_ERR_INVALID_ARG;
+    ClockProbe probes[3];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(probes, static_cast<const uint8_t*>(workspace) + kProbeOffsetBytes, sizeof(probes),
+                        cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return LAGA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return LAGA_ERR_CUDA;
+    for (int k = 0; k < LAGA_KERNEL_COUNT; ++k) sm_mhz[k] = kernel_ms[k] = 0.0;
+    const int ids[3] = {LAGA_KERNEL_ATTN_FWD, LAGA_KERNEL_ATTN_BWD_DKV, LAGA_KERNEL_ATTN_BWD_DQ};
+    for (int i = 0; i < 3; ++i) {
+        const ClockProbe& p = probes[i];
+        if (p.ns_end <= p.ns_begin || p.cycles_end <= p.cycles_begin) continue;   // that kernel has not run on this workspace
+        const double ns = static_cast<double>(p.ns_end - p.ns_begin);
+        sm_mhz[ids[i]] = static_cast<double>(p.cycles_end - p.cycles_begin) / ns * 1e3;
+        kernel_ms[ids[i]] = ns * 1e-6;
     }
     return LAGA_OK;
 }
@@ -528,7 +663,9 @@ int laga_query_status(const void* workspace, void* stream, unsigned* detail) {
     if (cudaStreamSynchronize(st) != cudaSuccess) return LAGA_ERR_CUDA;
     if (detail) *detail = word;
     if (word == 0) return LAGA_OK;
-    return (word & 0xff000000u) == kStatusTimeout ? LAGA_ERR_DEVICE_TIMEOUT : LAGA_ERR_CUDA;
+    if ((word & 0xff000000u) == kStatusTimeout) return LAGA_ERR_DEVICE_TIMEOUT;
+    if ((word & 0xff000000u) == kStatusCheck) return LAGA_ERR_DEVICE_CHECK;
+    return LAGA_ERR_CUDA;
 }
 
 }  // extern "C"

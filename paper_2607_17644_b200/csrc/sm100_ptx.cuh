@@ -15,6 +15,7 @@ namespace laga {
 // ------------------------------------------------------------------------------------------------
 constexpr unsigned int kStatusOk = 0u;
 constexpr unsigned int kStatusTimeout = 0x54000000u;   // | site id in the low bits
+constexpr unsigned int kStatusCheck = 0x43000000u;     // a device-side self-check failed; | site id
 
 // Wall-clock budget of a single mbarrier wait.  Kernels here run for milliseconds; a wait that has
 // not completed after this long means a protocol bug, and the kernel unwinds instead of hanging.

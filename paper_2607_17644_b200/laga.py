@@ -17,6 +17,7 @@ ERR_UNSUPPORTED = -2
 ERR_WORKSPACE_TOO_SMALL = -3
 ERR_CUDA = -4
 ERR_DEVICE_TIMEOUT = -5
+ERR_DEVICE_CHECK = -6
 FLAG_ACCUM_DW = 1
 FLAG_DETERMINISTIC = 2
 FLAG_KV_SAVED = 4
@@ -37,6 +38,7 @@ SIGNATURES = {
     "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
     "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
     "laga_profile_kernel": (_ci, [_ci, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _ci]),
+    "laga_query_kernel_clocks": (_ci, [_vp, _vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "laga_selftest_bounded_wait": (_ci, [_vp, _cu, _vp]),
     "laga_fwd_builtin_scratch": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp]),
 }
@@ -82,8 +84,8 @@ def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
-def _stream(stream):
-    s = torch.cuda.current_stream() if stream is None else stream
+def _stream(stream, device):
+    s = torch.cuda.current_stream(device) if stream is None else stream
     return ctypes.c_void_p(s.cuda_stream)
 
 
@@ -92,6 +94,23 @@ def _dev(t: torch.Tensor, dtype, shape, name):
         raise ValueError(f"{name}: expected contiguous CUDA {dtype} tensor of shape {tuple(shape)}, "
                          f"got {t.dtype} {tuple(t.shape)} on {t.device}")
     return t
+
+
+def same_device(*tensors) -> torch.device:
+    """All tensors of a call must live on ONE device: the library launches on the current device, so the
+    call runs under that device (see ``_on``) and a tensor from anywhere else is refused here, before the
+    C side would refuse its pointer."""
+    present = [t for t in tensors if t is not None]
+    dev = present[0].device
+    for t in present[1:]:
+        if t.device != dev:
+            raise ValueError(f"tensors of one call are on different devices: {dev} and {t.device}")
+    return dev
+
+
+def _on(device):
+    """Context that makes `device` current for the duration of a library call."""
+    return torch.cuda.device(device)
 
 
 def _geometry(q, c_kv, k_pe, w_kv_b, d_v):
@@ -124,22 +143,24 @@ def fwd(q, c_kv, k_pe, w_kv_b, d_v=128, softmax_scale=None, causal=True, out=Non
         stream=None):
     """laga_fwd: returns (out bf16 [S,h,d_v], lse fp32 [S,h], workspace).  Enqueues only."""
     S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
+    dev = same_device(q, c_kv, k_pe, w_kv_b, out, lse, workspace)
     if softmax_scale is None:
         softmax_scale = (d_nope + d_rope) ** -0.5
     if out is None:
-        out = torch.empty(S, h, d_v, dtype=torch.bfloat16, device=q.device)
+        out = torch.empty(S, h, d_v, dtype=torch.bfloat16, device=dev)
     if lse is None:
-        lse = torch.empty(S, h, dtype=torch.float32, device=q.device)
+        lse = torch.empty(S, h, dtype=torch.float32, device=dev)
     _dev(out, torch.bfloat16, (S, h, d_v), "out")
     _dev(lse, torch.float32, (S, h), "lse")
     need = fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v)
     if need == 0:
         raise LagaError(ERR_UNSUPPORTED, "laga_fwd_workspace_bytes")
     if workspace is None:
-        workspace = alloc_workspace(need, q.device)
-    rc = lib().laga_fwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope, d_v,
-                        float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse), _ptr(workspace),
-                        workspace.numel(), 0, _stream(stream))
+        workspace = alloc_workspace(need, dev)
+    with _on(dev):
+        rc = lib().laga_fwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope, d_v,
+                            float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse), _ptr(workspace),
+                            workspace.numel(), 0, _stream(stream, dev))
     _check(rc, "laga_fwd")
     return out, lse, workspace
 
@@ -152,16 +173,19 @@ def fwd_builtin_scratch(q, c_kv, k_pe, w_kv_b, out, lse, d_v=128, softmax_scale=
     S * h must not exceed BUILTIN_SCRATCH_MAX_TOKEN_HEADS; larger problems raise
     LAGA_ERR_WORKSPACE_TOO_SMALL.  Calls on one stream may follow each other freely; calls that could
     overlap on the GPU share the array and must be ordered by the caller.  The first call on a device
-    resolves the array's address and should happen outside stream capture.
+    resolves the array's address (and may be the call that makes the CUDA runtime load the library's
+    device code, array included): it belongs in initialisation, outside any stream capture.
     """
     S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
+    dev = same_device(q, c_kv, k_pe, w_kv_b, out, lse)
     if softmax_scale is None:
         softmax_scale = (d_nope + d_rope) ** -0.5
     _dev(out, torch.bfloat16, (S, h, d_v), "out")
     _dev(lse, torch.float32, (S, h), "lse")
-    rc = lib().laga_fwd_builtin_scratch(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope,
-                                        d_v, float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse),
-                                        _stream(stream))
+    with _on(dev):
+        rc = lib().laga_fwd_builtin_scratch(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope,
+                                            d_rope, d_v, float(softmax_scale), int(bool(causal)), _ptr(out),
+                                            _ptr(lse), _stream(stream, dev))
     _check(rc, "laga_fwd_builtin_scratch")
 
 
@@ -169,12 +193,12 @@ def bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout, d_v=128, softmax_scale=None, caus
         dk_pe=None, dw_kv_b=None, workspace=None, flags=0, stream=None):
     """laga_bwd: returns (dq, dc_kv, dk_pe, dw_kv_b, workspace).  Enqueues only."""
     S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
+    dev = same_device(q, c_kv, k_pe, w_kv_b, out, lse, dout, dq, dc_kv, dk_pe, dw_kv_b, workspace)
     if softmax_scale is None:
         softmax_scale = (d_nope + d_rope) ** -0.5
     _dev(out, torch.bfloat16, (S, h, d_v), "out")
     _dev(lse, torch.float32, (S, h), "lse")
     _dev(dout, torch.bfloat16, (S, h, d_v), "dout")
-    dev = q.device
     dq = torch.empty_like(q) if dq is None else _dev(dq, torch.bfloat16, q.shape, "dq")
     dc_kv = torch.empty_like(c_kv) if dc_kv is None else _dev(dc_kv, torch.bfloat16, c_kv.shape, "dc_kv")
     dk_pe = torch.empty_like(k_pe) if dk_pe is None else _dev(dk_pe, torch.bfloat16, k_pe.shape, "dk_pe")
@@ -188,9 +212,11 @@ def bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout, d_v=128, softmax_scale=None, caus
         raise LagaError(ERR_UNSUPPORTED, "laga_bwd_workspace_bytes")
     if workspace is None:
         workspace = alloc_workspace(need, dev)
-    rc = lib().laga_bwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), _ptr(out), _ptr(lse), _ptr(dout), S, h,
-                        d_c, d_nope, d_rope, d_v, float(softmax_scale), int(bool(causal)), _ptr(dq), _ptr(dc_kv),
-                        _ptr(dk_pe), _ptr(dw_kv_b), _ptr(workspace), workspace.numel(), flags, _stream(stream))
+    with _on(dev):
+        rc = lib().laga_bwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), _ptr(out), _ptr(lse), _ptr(dout), S, h,
+                            d_c, d_nope, d_rope, d_v, float(softmax_scale), int(bool(causal)), _ptr(dq), _ptr(dc_kv),
+                            _ptr(dk_pe), _ptr(dw_kv_b), _ptr(workspace), workspace.numel(), flags,
+                            _stream(stream, dev))
     _check(rc, "laga_bwd")
     return dq, dc_kv, dk_pe, dw_kv_b, workspace
 
@@ -201,12 +227,14 @@ def up_project(c_kv, w_kv_b, h, d_nope=128, d_v=128, kv=None, status_word=None, 
     n = h * (d_nope + d_v)
     _dev(c_kv, torch.bfloat16, (S, d_c), "c_kv")
     _dev(w_kv_b, torch.bfloat16, (d_c, n), "w_kv_b")
-    kv = torch.empty(S, n, dtype=torch.bfloat16, device=c_kv.device) if kv is None else kv
+    dev = same_device(c_kv, w_kv_b, kv, status_word)
+    kv = torch.empty(S, n, dtype=torch.bfloat16, device=dev) if kv is None else kv
     _dev(kv, torch.bfloat16, (S, n), "kv")
     if status_word is None:
-        status_word = torch.zeros(1, dtype=torch.int32, device=c_kv.device)
-    rc = lib().laga_up_project(_ptr(c_kv), _ptr(w_kv_b), S, h, d_c, d_nope, d_v, _ptr(kv), _ptr(status_word),
-                               _stream(stream))
+        status_word = torch.zeros(1, dtype=torch.int32, device=dev)
+    with _on(dev):
+        rc = lib().laga_up_project(_ptr(c_kv), _ptr(w_kv_b), S, h, d_c, d_nope, d_v, _ptr(kv), _ptr(status_word),
+                                   _stream(stream, dev))
     _check(rc, "laga_up_project")
     return kv, status_word
 
@@ -219,14 +247,16 @@ def kv_backward(dkv, c_kv, w_kv_b, h, d_nope=128, d_v=128, dc_kv=None, dw_kv_b=N
     _dev(dkv, torch.bfloat16, (S, n), "dkv")
     _dev(c_kv, torch.bfloat16, (S, d_c), "c_kv")
     _dev(w_kv_b, torch.bfloat16, (d_c, n), "w_kv_b")
+    dev = same_device(dkv, c_kv, w_kv_b, dc_kv, dw_kv_b, status_word)
     dc_kv = torch.empty_like(c_kv) if dc_kv is None else _dev(dc_kv, torch.bfloat16, c_kv.shape, "dc_kv")
     if dw_kv_b is None:
-        dw_kv_b = torch.empty(d_c, n, dtype=torch.float32, device=c_kv.device)
+        dw_kv_b = torch.empty(d_c, n, dtype=torch.float32, device=dev)
     _dev(dw_kv_b, torch.float32, (d_c, n), "dw_kv_b")
     if status_word is None:
-        status_word = torch.zeros(1, dtype=torch.int32, device=c_kv.device)
-    rc = lib().laga_kv_backward(_ptr(dkv), _ptr(c_kv), _ptr(w_kv_b), S, h, d_c, d_nope, d_v, _ptr(dc_kv),
-                                _ptr(dw_kv_b), flags, _ptr(status_word), _stream(stream))
+        status_word = torch.zeros(1, dtype=torch.int32, device=dev)
+    with _on(dev):
+        rc = lib().laga_kv_backward(_ptr(dkv), _ptr(c_kv), _ptr(w_kv_b), S, h, d_c, d_nope, d_v, _ptr(dc_kv),
+                                    _ptr(dw_kv_b), flags, _ptr(status_word), _stream(stream, dev))
     _check(rc, "laga_kv_backward")
     return dc_kv, dw_kv_b, status_word
 
@@ -242,18 +272,33 @@ def profile_kernel(kernel: str, start_events=(), stop_events=()):
     _check(lib().laga_profile_kernel(KERNELS[kernel], starts, stops, n), "laga_profile_kernel")
 
 
+def query_kernel_clocks(workspace, stream=None) -> dict:
+    """laga_query_kernel_clocks: synchronises the stream; returns {kernel name: (SM MHz, kernel ms)} for
+    the attention kernels the last call on `workspace` ran (measured inside the kernels themselves)."""
+    mhz = (ctypes.c_double * len(KERNELS))()
+    ms = (ctypes.c_double * len(KERNELS))()
+    with _on(workspace.device):
+        rc = lib().laga_query_kernel_clocks(_ptr(workspace), _stream(stream, workspace.device), mhz, ms)
+    _check(rc, "laga_query_kernel_clocks")
+    return {name: (float(mhz[i]), float(ms[i])) for name, i in KERNELS.items() if mhz[i] > 0.0}
+
+
 def selftest_bounded_wait(budget_us: int = 1000, stream=None):
     """laga_selftest_bounded_wait: run the kernel whose waits cannot complete; returns the status word
     tensor to pass to query_status (expected: ERR_DEVICE_TIMEOUT, detail 0x54007e57)."""
     word = torch.zeros(1, dtype=torch.int32, device="cuda")
-    _check(lib().laga_selftest_bounded_wait(_ptr(word), int(budget_us), _stream(stream)), "laga_selftest_bounded_wait")
+    with _on(word.device):
+        rc = lib().laga_selftest_bounded_wait(_ptr(word), int(budget_us), _stream(stream, word.device))
+    _check(rc, "laga_selftest_bounded_wait")
     return word
 
 
 def query_status(workspace_or_word, stream=None) -> tuple[int, int]:
     """laga_query_status: synchronises the stream; returns (status code, raw device word)."""
     detail = ctypes.c_uint(0)
-    rc = lib().laga_query_status(_ptr(workspace_or_word), _stream(stream), ctypes.byref(detail))
+    dev = workspace_or_word.device
+    with _on(dev):
+        rc = lib().laga_query_status(_ptr(workspace_or_word), _stream(stream, dev), ctypes.byref(detail))
     return int(rc), int(detail.value)
 
 

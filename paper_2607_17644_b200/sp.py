@@ -12,7 +12,7 @@ shard H_r = {r n_h/P, ..., (r+1) n_h/P - 1} inside it:
 Backward: the gradient of step 6 is a head-scatter all-to-all of d_out, the gradient of step 2 a
 sequence-scatter all-to-all of dq, the gradient of step 3 a reduce-scatter of the ranks' partial
 dc_kv and dk_pe, and the W_kv_b gradient -- complete for H_r's columns on rank r, zero elsewhere --
-is summed over the group.  Only the exchanges are here; every contraction is in ``compute``.
+is summed over the group (an all-gather of the column shards).  Only the exchanges are here; every contraction is in ``compute``.
 
 No kernel of this repository reads peer memory: a gathered tensor lands in this GPU's memory first
 and the hot path reads it from there.  On this build's single-GPU test pool the exchanges are covered
@@ -26,7 +26,7 @@ import torch
 import torch.distributed as dist
 
 
-# ---- communication volume (Section 6, communication table) ---------------------------------------
+# ---- communication volume (Section 4, Evaluation: communication-volume table) --------------------
 @dataclass(frozen=True)
 class CommDims:
     n_h: int = 128
@@ -114,15 +114,16 @@ def shard_columns(w_kv_b: torch.Tensor, n_h: int, group=None) -> torch.Tensor:
     return w_kv_b[:, r * h * per_head:(r + 1) * h * per_head].contiguous()
 
 
-def all_reduce_dw(dw_shard: torch.Tensor, n_h: int, group=None) -> torch.Tensor:
-    """The head-axis all-reduce of Section 5.2: rank r's gradient covers H_r's columns of the replicated
-    W_kv_b and is zero elsewhere; the sum over the group is the full gradient."""
-    P, r = _world(group)
-    cols = dw_shard.shape[1]
-    full = torch.zeros(dw_shard.shape[0], cols * P, dtype=dw_shard.dtype, device=dw_shard.device)
-    full[:, r * cols:(r + 1) * cols] = dw_shard
-    dist.all_reduce(full, group=group)
-    return full
+def all_gather_dw(dw_shard: torch.Tensor, n_h: int, group=None) -> torch.Tensor:
+    """The head-axis reduction of the W_kv_b gradient (Section 5.2).  Rank r's gradient is complete for H_r's
+    columns of the replicated W_kv_b and identically zero elsewhere, so the sum over the group is the
+    concatenation of the column shards: an all-gather moves 1/P of what an all-reduce of zero-padded full
+    matrices would.  Returns the full [d_c, n_h (d_nope + d_v)] gradient (identical on every rank)."""
+    P, _ = _world(group)
+    d_c, cols = dw_shard.shape
+    gathered = torch.empty(P * d_c, cols, dtype=dw_shard.dtype, device=dw_shard.device)   # rank-major row blocks
+    dist.all_gather_into_tensor(gathered, dw_shard.contiguous(), group=group)
+    return gathered.view(P, d_c, cols).permute(1, 0, 2).reshape(d_c, P * cols).contiguous()
 
 
 # ---- one attention block under SP ----------------------------------------------------------------
@@ -163,4 +164,4 @@ def sp_backward(ctx, dout_local, compute, group=None):
     dout = head_scatter_all_to_all(dout_local, group)
     dq, dc_kv, dk_pe, dw = compute.bwd(q, c_kv, k_pe, w, out, lse, dout, causal)
     return (seq_scatter_all_to_all(dq, group), seq_reduce_scatter(dc_kv, group), seq_reduce_scatter(dk_pe, group),
-            all_reduce_dw(dw, n_h, group))
+            all_gather_dw(dw, n_h, group))

@@ -119,3 +119,14 @@ def test_binding_rejects_cpu_tensors(laga):
     w = torch.zeros(512, 512, dtype=torch.bfloat16)
     with pytest.raises(ValueError):
         laga.fwd(q, c, k, w)
+
+
+def test_binding_refuses_tensors_on_different_devices(laga):
+    """One call, one device: the check runs before anything reaches the C side (here with a CPU and a
+    meta tensor, which need no GPU)."""
+    import torch
+    a = torch.zeros(4)
+    b = torch.zeros(4, device="meta")
+    with pytest.raises(ValueError, match="different devices"):
+        laga.same_device(a, b)
+    assert laga.same_device(a, None, torch.ones(2)) == a.device

@@ -72,3 +72,27 @@ def test_max_over_ranks_with_two_gloo_ranks():
     fl = bench.flops(CONFIGS["c2"])
     total = fl["fwd"] + fl["bwd"]
     assert abs(2 * total / (results[0] * 1e-3) / 1e12 - 2 * total / 15e-3 / 1e12) < 1e-9
+
+
+def test_gpus_n_without_a_launcher_starts_n_ranks():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment must itself start two ranks (one per
+    GPU on the real run) and print ONE line whose n_gpus is 2 with the max over the ranks' times.  --dry-run
+    swaps the GPU work for a made-up step time (10 ms on rank 0, 15 ms on rank 1) over gloo."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"], env=env,
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip().startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["ms_per_step"] == 15.0 and d["scaling"] == "weak"
+
+
+def test_error_metrics_and_sample():
+    g = torch.tensor([1.0, 2.0, 4.0])
+    r = torch.tensor([1.0, 2.0, 3.0], dtype=torch.float64)
+    m = bench.error_metrics(g, r)
+    assert m["max_abs"] == 1.0 and abs(m["rel_l2"] - 1.0 / 14 ** 0.5) < 1e-12
+    assert abs(m["scaled_max_abs"] - 1.0 / (14 / 3) ** 0.5) < 1e-12
+    sub, tensors = bench.oracle_sample(100, "c1")
+    assert sub.S == 100 and sub.h == 1 and tuple(tensors[0].shape) == (100, 1, 192) and tuple(tensors[3].shape) == (512, 256)

@@ -124,7 +124,8 @@ def test_round_bf16_matches_single_rounding(oracle):
 
 @pytest.mark.parametrize("sh", [TOY, SMALL], ids=["toy", "small"])
 def test_head_shard_concatenation(oracle, sh):
-    """Paper Prop. 1: a head shard's up-projection is a column slice of the full one, so running the
+    """Section 5.1: step 4 computes, for the heads of a shard, the same per-head linear maps as the full
+    up-projection, i.e. a head shard's up-projection is a column slice of the full one, so running the
     shards separately reproduces the full-head run; shared-tensor gradients add across shards."""
     sh = LagaShape(S=sh.S, h=4, d_c=sh.d_c, d_nope=sh.d_nope, d_rope=sh.d_rope, d_v=sh.d_v)
     q, c_kv, k_pe, w, dout = make_inputs(sh, 15)

@@ -51,6 +51,44 @@ def test_two_calls_in_a_row_match_laga_fwd(laga):
     _check_same(*second)
 
 
+def test_matches_the_oracle_directly(laga, oracle):
+    """One comparison that does not go through laga_fwd at all: the entry point against the fp64 oracle."""
+    from parity import TOL_LSE, check_tensor, max_abs
+    sh = LagaShape(S=700, h=3)
+    tensors = make_inputs(sh, 36, with_dout=False)
+    q, c_kv, k_pe, w = (t.cuda() for t in tensors[:4])
+    out = torch.full((sh.S, sh.h, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((sh.S, sh.h), float("nan"), dtype=torch.float32, device="cuda")
+    laga.fwd_builtin_scratch(q, c_kv, k_pe, w, out, lse)
+    torch.cuda.synchronize()
+    ref_out, ref_lse = oracle.fwd(*tensors[:4], sh.d_v, sh.softmax_scale, causal=True, kv_round_bf16=True)
+    check_tensor("out", out, ref_out)
+    assert max_abs(lse, ref_lse) <= TOL_LSE
+
+
+def test_the_call_allocates_no_device_memory(laga):
+    """After one warm call (which may make the CUDA runtime load the library's device code, the scratch
+    array included), further calls must leave the device's free memory and torch's allocator untouched,
+    at two different shapes."""
+    shapes = [LagaShape(S=512, h=4), LagaShape(S=1000, h=2)]
+    cases = []
+    for i, sh in enumerate(shapes):
+        q, c_kv, k_pe, w = (t.cuda() for t in make_inputs(sh, 40 + i, with_dout=False)[:4])
+        out = torch.empty(sh.S, sh.h, 128, dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty(sh.S, sh.h, dtype=torch.float32, device="cuda")
+        cases.append((q, c_kv, k_pe, w, out, lse))
+    laga.fwd_builtin_scratch(*cases[0])                      # warm: module load, address lookup
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    allocated_before, reserved_before = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for case in cases + cases:
+        laga.fwd_builtin_scratch(*case)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert torch.cuda.memory_allocated() == allocated_before and torch.cuda.memory_reserved() == reserved_before
+    assert free_after == free_before, f"device free memory moved by {free_before - free_after} bytes"
+
+
 def test_back_to_back_on_one_stream_without_sync(laga):
     """Two enqueues with no host synchronisation between them: stream order alone must be enough."""
     sh_a, sh_b = LagaShape(S=640, h=2), LagaShape(S=512, h=5)
