@@ -40,7 +40,7 @@ KERNELS_PER_STEP = 9   # fwd: up_project, attn_fwd; bwd: up_project, delta, dkv,
 # capture summarised in profiles/ncu_dram_c2_attn_bwd_dkv.txt.  For other workloads the figure is scaled
 # by S*h (the kernel reads its inputs and writes its outputs once; tiles are re-read from L2, not DRAM)
 # and flagged as scaled.
-DKV_DRAM_BYTES_C2 = None          # filled in from the capture; None until one exists
+DKV_DRAM_BYTES_C2 = 337137408 + 112096000          # dram__bytes_read.sum + dram__bytes_write.sum of one launch
 DKV_DRAM_C2_TOKEN_HEADS = 16384 * 16
 
 
