@@ -226,9 +226,70 @@ def run_dry(args):
         dist.destroy_process_group()
 
 
+def run_c4(args):
+    """Benchmark configuration 4: the absorbed form (Section 3.2, baseline B2) on configuration 2's inputs,
+    forward, as hand-written kernels (laga_absorbed_fwd), beside the LAGA forward on the same inputs: time,
+    useful TFLOP/s (the explicit form's 640 FLOP per causal pair and head plus one up-projection -- the work
+    the result needs), executed TFLOP/s (what the absorbed kernels actually run) and the scratch each form
+    keeps alive.  One GPU; the absorbed form has no backward here."""
+    from paper_2607_17644_b200 import laga
+    laga.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    sh = CONFIGS["c4"]
+    fl = flops(sh)
+    pairs = sh.S * (sh.S + 1) // 2
+    q, c_kv, k_pe, w, _ = (t.to(dev) if t is not None else None for t in make_inputs(sh, CONFIG_SEEDS["c4"], with_dout=False))
+    out = torch.empty(sh.S, sh.h, sh.d_v, dtype=torch.bfloat16, device=dev)
+    lse = torch.empty(sh.S, sh.h, dtype=torch.float32, device=dev)
+    out_l, lse_l = torch.empty_like(out), torch.empty_like(lse)
+    ws_a = laga.alloc_workspace(laga.absorbed_fwd_workspace_bytes(sh.S, sh.h), dev)
+    ws_l = laga.alloc_workspace(laga.fwd_workspace_bytes(sh.S, sh.h), dev)
+    K, W = args.steps, max(args.warmup, 3)
+
+    def timed(fn):
+        for _ in range(W):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(K):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / K
+
+    abs_ms = timed(lambda: laga.absorbed_fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_a))
+    laga_ms = timed(lambda: laga.fwd(q, c_kv, k_pe, w, out=out_l, lse=lse_l, workspace=ws_l))
+    laga.check_status(ws_a, where="laga_absorbed_fwd")
+    laga.check_status(ws_l, where="laga_fwd")
+    executed = 2 * sh.h * pairs * (2 * (sh.d_c + sh.d_rope) + sh.d_c) + 2 * 2 * sh.S * sh.h * sh.d_nope * sh.d_c   # both halves' scores + P V, two batched GEMMs
+    nominal = 2 * sh.h * pairs * ((sh.d_c + sh.d_rope) + sh.d_c) + 2 * 2 * sh.S * sh.h * sh.d_nope * sh.d_c
+    peaks = measured_peaks()
+    line = {"metric": "absorbed_form_fwd_useful_tflops", "value": fl["fwd"] / (abs_ms * 1e-3) / 1e12, "unit": UNIT,
+            "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": abs_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "c4: absorbed form on c2's inputs (S=16384, h_local=16, causal), forward",
+                       "l2_policy": "inputs and scratch larger than L2 (q_abs and the latent accumulator alone are 537 MB)"},
+            "absorbed": {"ms": abs_ms, "useful_tflops": fl["fwd"] / (abs_ms * 1e-3) / 1e12,
+                         "executed_tflops": executed / (abs_ms * 1e-3) / 1e12,
+                         "executed_flops": executed, "nominal_flops_of_the_form": nominal, "useful_flops": fl["fwd"],
+                         "executed_frac_of_burst_peak": executed / (abs_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                         "scratch_bytes": ws_a.numel()},
+            "laga": {"ms": laga_ms, "tflops": fl["fwd"] / (laga_ms * 1e-3) / 1e12, "scratch_bytes": ws_l.numel()},
+            "absorbed_over_laga": {"time": abs_ms / laga_ms, "scratch": ws_a.numel() / ws_l.numel(),
+                                   "extra_scratch_bytes": ws_a.numel() - ws_l.numel()},
+            "max_abs_diff_between_forms": {"out": float((out.float() - out_l.float()).abs().max()),
+                                           "lse": float((lse - lse_l).abs().max())},
+            "gpu_launches": 3 * K}
+    print(json.dumps(line), flush=True)
+
+
 def run_cuda(args):
     from paper_2607_17644_b200 import laga
     laga.lib()
+    if args.workload == "c4":
+        return run_c4(args)
     world, rank, local_rank = dist_setup(args.gpus)
     dev = torch.device("cuda", torch.cuda.current_device())
     sh = CONFIGS[args.workload]
@@ -596,7 +657,8 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing and parity leg")
     ap.add_argument("--workload", choices=sorted(CONFIGS), default=WORKLOAD,
-                    help="benchmark configuration (default c2, the headline; others are for profiling)")
+                    help="benchmark configuration (default c2, the headline; c4 = the absorbed form beside the LAGA "
+                         "forward on c2's inputs; others are for profiling)")
     ap.add_argument("--compare-eager", action="store_true",
                     help="also time the explicit and absorbed forms in eager PyTorch (N=1; tens of GB at c2)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=16384,

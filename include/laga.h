@@ -127,6 +127,26 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
                      void* stream);
 
 /*
+ * The ABSORBED form of the same forward (Section 3.2, baseline B2), for comparison with laga_fwd: the
+ * paper's point is what this form costs in training.  Same inputs, outputs and meaning as laga_fwd (the two
+ * forms are algebraically identical: q_nope . (W_uk^T c) = (W_uk q_nope) . c), different association:
+ *   q_abs[s,i,:] = W_uk[i] q_nope[s,i,:]                 (d_c wide: a batched GEMM over the heads)
+ *   scores       = softmax_scale * ( q_abs . c_kv^T + q_rope . k_pe^T )     (576-deep, against the latent itself)
+ *   o_lat[s,i,:] = softmax(scores) c_kv                  (d_c-wide accumulator per token and head)
+ *   out[s,i,:]   = W_uv[i]^T o_lat[s,i,:]                (a second batched GEMM)
+ * where W_uk[i] / W_uv[i] are the K / V column blocks of head i in w_kv_b.  No per-head K or V is formed;
+ * instead q_abs and o_lat, S*h*d_c bf16 elements each, live in `workspace` (laga_absorbed_fwd_workspace_bytes):
+ * at S=16384, h=16 that is 537 MB against the 134 MB of laga_fwd.  The attention kernel splits the 512
+ * latent columns over two CTAs and computes the scores in both, so it executes 3328 FLOP per (query, key)
+ * pair (2176 nominal for this form, 640 for the explicit form).  Forward only.
+ * Errors and conventions as laga_fwd; `flags` must be 0.
+ */
+size_t laga_absorbed_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v);
+int laga_absorbed_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
+                      int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out, float* lse,
+                      void* workspace, size_t workspace_bytes, unsigned flags, void* stream);
+
+/*
  * laga_fwd for callers that have no scratch to give.  (The paper has no counterpart: this is a
  * packaging convenience of the library, not a step of the method.)
  *
@@ -186,7 +206,10 @@ int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stre
 #define LAGA_KERNEL_DKPE_REDUCE 5   /* dk_pe: bf16 rounding of the head-summed rope-column sums */
 #define LAGA_KERNEL_DCKV_GEMM 6     /* dc_kv = dKV . W^T                                       */
 #define LAGA_KERNEL_DW_GEMM 7       /* dW = c_kv^T . dKV                                       */
-#define LAGA_KERNEL_COUNT 8
+#define LAGA_KERNEL_Q_ABSORB 8      /* absorbed form: q_abs = W_uk q_nope (batched over heads)   */
+#define LAGA_KERNEL_ATTN_ABSORBED 9 /* absorbed form: latent-space attention                     */
+#define LAGA_KERNEL_V_PROJECT 10    /* absorbed form: out = W_uv o_lat (batched over heads)      */
+#define LAGA_KERNEL_COUNT 11
 int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs);
 
 /*

@@ -4,6 +4,10 @@
 //     KV    [S, N]   = c_kv [S, d_c] . W [d_c, N]          A K-major,  B MN-major, bf16 out
 //     dc_kv [S, d_c] = dKV  [S, N]   . W^T                 A K-major,  B K-major,  bf16 out
 //     dW    [d_c, N] = c_kv^T . dKV                        A MN-major, B MN-major, fp32 atomic out (split-K)
+// and, batched over the heads of the shard, for the two projections of the absorbed form (Section 3.2):
+//     q_abs [S, h, d_c]  = q_nope [S, h, d_n] . W_uk[h]^T  A K-major,  B K-major,  bf16 out
+//     out   [S, h, d_v]  = o_lat  [S, h, d_c] . W_uv[h]    A K-major,  B MN-major, bf16 out
+// (a batch shifts the operands' innermost TMA coordinate and the output's column by a fixed step).
 //
 // Persistent: one CTA per SM walks the 128 x BN output tiles (n fastest, so neighbouring CTAs share
 // the A tile through L2).  Warp 0 issues TMA loads, warp 1 issues the MMAs, warps 2..5 drain the
@@ -24,6 +28,9 @@ struct GemmArgs {
     unsigned int* status;
     float4* zero_begin;   // optional: zero_count float4 elements cleared by this launch before it starts
     size_t zero_count;    // (the buffer the NEXT kernel accumulates into: saves a separate memset)
+    int batches;          // >= 1; batch b adds b * a_step / b_step to the operands' innermost (contiguous)
+    int a_step, b_step;   // TMA coordinate and b * c_step to the output column
+    int c_step;
 };
 
 enum { EPI_BF16 = 0, EPI_ATOMIC_F32 = 1 };
@@ -55,7 +62,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_n = args.N / BN;
     const int tiles_m = (args.M + 127) / 128;
-    const int total_tiles = tiles_n * tiles_m * args.n_splits;
+    const int tiles_per_batch = tiles_n * tiles_m * args.n_splits;
+    const int total_tiles = tiles_per_batch * args.batches;
     const int total_k_tiles = (args.K + 63) / 64;
     constexpr uint32_t kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
 
@@ -87,9 +95,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             uint32_t kc = 0;   // running k-iteration count: stage = kc % STAGES, phase = (kc / STAGES) & 1
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int n0 = (t % tiles_n) * BN, m0 = ((t / tiles_n) % tiles_m) * 128;
+                const int batch = t / tiles_per_batch, tb = t - batch * tiles_per_batch;
+                const int n0 = (tb % tiles_n) * BN, m0 = ((tb / tiles_n) % tiles_m) * 128;
+                const int a_off = batch * args.a_step, b_off = batch * args.b_step;
                 int kt_begin, n_kt;
-                k_range(t / (tiles_n * tiles_m), kt_begin, n_kt);
+                k_range(tb / (tiles_n * tiles_m), kt_begin, n_kt);
                 for (int i = 0; i < n_kt; ++i, ++kc) {
                     const int s = kc % STAGES;
                     ok = mbar_wait(&empty_bar[s], ((kc / STAGES) & 1) ^ 1, abort_flag, args.status, 0x100);
@@ -99,16 +109,16 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     mbar_arrive_expect_tx(&full_bar[s], L::kStageBytes);
                     const int k0 = (kt_begin + i) * 64;
                     if (A_MN) {   // global A is [K rows, M contiguous]: two slabs of 64 K-rows x 64 M
-                        tma_load_2d(sa, &tmap_a, &full_bar[s], m0, k0);
-                        tma_load_2d(sa + 8192, &tmap_a, &full_bar[s], m0 + 64, k0);
+                        tma_load_2d(sa, &tmap_a, &full_bar[s], a_off + m0, k0);
+                        tma_load_2d(sa + 8192, &tmap_a, &full_bar[s], a_off + m0 + 64, k0);
                     } else {      // global A is [M rows, K contiguous]: one slab of 128 rows x 64 K
-                        tma_load_2d(sa, &tmap_a, &full_bar[s], k0, m0);
+                        tma_load_2d(sa, &tmap_a, &full_bar[s], a_off + k0, m0);
                     }
                     if (B_MN) {
                         for (int j = 0; j < BN / 64; ++j)
-                            tma_load_2d(sb + j * 8192, &tmap_b, &full_bar[s], n0 + j * 64, k0);
+                            tma_load_2d(sb + j * 8192, &tmap_b, &full_bar[s], b_off + n0 + j * 64, k0);
                     } else {
-                        tma_load_2d(sb, &tmap_b, &full_bar[s], k0, n0);
+                        tma_load_2d(sb, &tmap_b, &full_bar[s], b_off + k0, n0);
                     }
                 }
             }
@@ -120,7 +130,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
                 int kt_begin, n_kt;
-                k_range(t / (tiles_n * tiles_m), kt_begin, n_kt);
+                k_range((t % tiles_per_batch) / (tiles_n * tiles_m), kt_begin, n_kt);
                 const uint32_t buf = it & 1;
                 ok = mbar_wait(&acc_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, args.status, 0x201);
                 if (!ok) break;
@@ -151,9 +161,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         uint32_t it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-            const int n0 = (t % tiles_n) * BN, m0 = ((t / tiles_n) % tiles_m) * 128;
+            const int batch = t / tiles_per_batch, tb = t - batch * tiles_per_batch;
+            const int n0 = batch * args.c_step + (tb % tiles_n) * BN, m0 = ((tb / tiles_n) % tiles_m) * 128;
             int kt_begin, n_kt;
-            k_range(t / (tiles_n * tiles_m), kt_begin, n_kt);
+            k_range(tb / (tiles_n * tiles_m), kt_begin, n_kt);
             const uint32_t buf = it & 1;
             const int row = m0 + quarter * 32 + lane;
             ok = mbar_wait_warp(&acc_full[buf], (it >> 1) & 1, abort_flag, args.status, 0x300);

@@ -10,6 +10,7 @@
 #include <mutex>
 #include <vector>
 
+#include "attn_absorbed_sm100.cuh"
 #include "attn_bwd_sm100.cuh"
 #include "attn_fwd_sm100.cuh"
 #include "gemm_sm100.cuh"
@@ -103,6 +104,9 @@ void init_device(DeviceInfo* info, int dev) {
     bool ok = allow_smem(gemm_sm100_kernel<256, 4, false, true, EPI_BF16>, G::kTotalBytes) &&
               allow_smem(gemm_sm100_kernel<256, 4, false, false, EPI_BF16>, G::kTotalBytes) &&
               allow_smem(gemm_sm100_kernel<256, 4, true, true, EPI_ATOMIC_F32>, G::kTotalBytes) &&
+              allow_smem(gemm_sm100_kernel<128, 4, false, true, EPI_BF16>, GemmSmem<128, 4>::kTotalBytes) &&
+              allow_smem(attn_absorbed_fwd_sm100_kernel<true>, AttnAbsorbedSmem::kTotalBytes) &&
+              allow_smem(attn_absorbed_fwd_sm100_kernel<false>, AttnAbsorbedSmem::kTotalBytes) &&
               allow_smem(attn_fwd_sm100_kernel<true>, AttnFwdSmem::kTotalBytes) &&
               allow_smem(attn_fwd_sm100_kernel<false>, AttnFwdSmem::kTotalBytes) &&
               allow_smem(attn_bwd_dkv_sm100_kernel<true>, AttnBwdDkvSmem::kTotalBytes) &&
@@ -239,7 +243,7 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
     if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
-    GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status, nullptr, 0};
+    GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status, nullptr, 0, 1, 0, 0, 0};
     dim3 grid(persistent_grid((N / BN) * ((S + 127) / 128)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
@@ -257,7 +261,7 @@ int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN)) return LAGA_ERR_CUDA;
-    GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status, reinterpret_cast<float4*>(clear), clear_floats / 4};
+    GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status, reinterpret_cast<float4*>(clear), clear_floats / 4, 1, 0, 0, 0};
     dim3 grid(persistent_grid((kDc / BN) * ((S + 127) / 128)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
@@ -289,7 +293,7 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool d
     }
     const int per_split = (k_tiles + splits - 1) / splits;
     splits = (k_tiles + per_split - 1) / per_split;
-    GemmArgs a{kDc, N, S, per_split, splits, dw, N, status, nullptr, 0};
+    GemmArgs a{kDc, N, S, per_split, splits, dw, N, status, nullptr, 0, 1, 0, 0, 0};
     dim3 grid(persistent_grid(tiles * splits), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
@@ -391,6 +395,57 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
                 dkpe_acc, S, reinterpret_cast<__nv_bfloat16*>(dk_pe));
         }
     }
+    return launch_status();
+}
+
+// ---- absorbed form (Section 3.2, baseline B2): comparison path --------------------------------------
+// q_abs[S, h, d_c] = q_nope[S, h, d_n] . W_uk[h]^T, batched over the heads: head i reads columns
+// [192 i, 192 i + 128) of q and columns [256 i, 256 i + 128) of W (rows = latent index = the GEMM's N).
+int launch_q_absorb(const void* q, const void* w, int S, int h, void* q_abs, unsigned* status, cudaStream_t stream) {
+    constexpr int BN = 256, STAGES = 4;
+    auto kernel = gemm_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
+    using L = GemmSmem<BN, STAGES>;
+    const uint64_t q_row = static_cast<uint64_t>(h) * (kDn + kDr), w_row = static_cast<uint64_t>(h) * (kDn + kDv);
+    CUtensorMap ta, tb;
+    if (!cached_tmap_bf16(&ta, q, q_row, S, q_row * 2, 128)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tb, w, w_row, kDc, w_row * 2, BN)) return LAGA_ERR_CUDA;
+    GemmArgs a{S, kDc, kDn, kDn / 64, 1, q_abs, h * kDc, status, nullptr, 0, h, kDn + kDr, kDn + kDv, kDc};
+    dim3 grid(persistent_grid((kDc / BN) * ((S + 127) / 128) * h), 1, 1);
+    { ScopedKernelEvents ev(LAGA_KERNEL_Q_ABSORB, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
+    return launch_status();
+}
+
+// out[S, h, d_v] = o_lat[S, h, d_c] . W_uv[h], batched over the heads: head i reads columns
+// [512 i, 512 i + 512) of o_lat and columns [256 i + 128, 256 i + 256) of W (rows = latent index = the GEMM's K).
+int launch_v_project(const void* o_lat, const void* w, int S, int h, void* out, unsigned* status, cudaStream_t stream) {
+    constexpr int BN = 128, STAGES = 4;
+    auto kernel = gemm_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
+    using L = GemmSmem<BN, STAGES>;
+    const uint64_t o_row = static_cast<uint64_t>(h) * kDc, w_row = static_cast<uint64_t>(h) * (kDn + kDv);
+    CUtensorMap ta, tb;
+    if (!cached_tmap_bf16(&ta, o_lat, o_row, S, o_row * 2, 128)) return LAGA_ERR_CUDA;
+    // the map starts at W's column d_nope: column 0 of the map is V channel 0 of head 0
+    if (!cached_tmap_bf16(&tb, static_cast<const uint8_t*>(w) + kDn * 2, w_row - kDn, kDc, w_row * 2, 64)) return LAGA_ERR_CUDA;
+    GemmArgs a{S, kDv, kDc, kDc / 64, 1, out, h * kDv, status, nullptr, 0, h, kDc, kDn + kDv, kDv};
+    dim3 grid(persistent_grid(((S + 127) / 128) * h), 1, 1);
+    { ScopedKernelEvents ev(LAGA_KERNEL_V_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
+    return launch_status();
+}
+
+int launch_attn_absorbed(const void* q, const void* q_abs, const void* c_kv, const void* k_pe, int S, int h,
+                         float softmax_scale, int causal, void* o_lat, float* lse, unsigned* status, cudaStream_t stream) {
+    using L = AttnAbsorbedSmem;
+    const uint64_t qa_row = static_cast<uint64_t>(h) * kDc, q_row = static_cast<uint64_t>(h) * (kDn + kDr);
+    CUtensorMap tqa, tq, tc, tpe;
+    if (!cached_tmap_bf16(&tqa, q_abs, qa_row, S, qa_row * 2, 128) || !cached_tmap_bf16(&tq, q, q_row, S, q_row * 2, 128) ||
+        !cached_tmap_bf16(&tc, c_kv, kDc, S, kDc * 2, kAbsKeys) || !cached_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, kAbsKeys))
+        return LAGA_ERR_CUDA;
+    AttnAbsorbedArgs a{S, h, softmax_scale * 1.4426950408889634f, reinterpret_cast<const __nv_bfloat16*>(q_abs),
+                       reinterpret_cast<__nv_bfloat16*>(o_lat), lse, status};
+    dim3 grid((S + 127) / 128, 2 * h, 1);
+    ScopedKernelEvents ev(LAGA_KERNEL_ATTN_ABSORBED, stream);
+    if (causal) attn_absorbed_fwd_sm100_kernel<true><<<grid, kAbsThreads, L::kTotalBytes, stream>>>(tqa, tq, tc, tpe, a);
+    else attn_absorbed_fwd_sm100_kernel<false><<<grid, kAbsThreads, L::kTotalBytes, stream>>>(tqa, tq, tc, tpe, a);
     return launch_status();
 }
 
@@ -604,6 +659,39 @@ int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, 
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
     if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
     return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st);
+}
+
+size_t laga_absorbed_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v) {
+    if (S < 1 || h < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
+    return kStatusBytes + 2 * align_up(static_cast<size_t>(S) * h * d_c * 2, 1024);
+}
+
+int laga_absorbed_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
+                      int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out, float* lse,
+                      void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+    if (!q || !c_kv || !k_pe || !w_kv_b || !out || !lse || !workspace || S < 1 || h < 1)
+        return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(c_kv) || !aligned16(k_pe) || !aligned16(w_kv_b) || !aligned16(out) ||
+        !aligned16(lse) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return LAGA_ERR_INVALID_ARG;
+    if (flags != 0 || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
+    if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
+    if (workspace_bytes < laga_absorbed_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v))
+        return LAGA_ERR_WORKSPACE_TOO_SMALL;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({q, c_kv, k_pe, w_kv_b, out, lse, workspace})) != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    unsigned* status = reinterpret_cast<unsigned*>(base);
+    const size_t lat_bytes = align_up(static_cast<size_t>(S) * h * kDc * 2, 1024);
+    void* q_abs = base + kStatusBytes;
+    void* o_lat = base + kStatusBytes + lat_bytes;
+    if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
+    if ((rc = launch_q_absorb(q, w_kv_b, S, h, q_abs, status, st)) != LAGA_OK) return rc;
+    if ((rc = launch_attn_absorbed(q, q_abs, c_kv, k_pe, S, h, softmax_scale, causal, o_lat, lse, status, st)) != LAGA_OK)
+        return rc;
+    return launch_v_project(o_lat, w_kv_b, S, h, out, status, st);
 }
 
 int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stream) {

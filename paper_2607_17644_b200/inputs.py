@@ -51,6 +51,7 @@ CONFIGS = {
     "c3_sp2": LagaShape(S=8192, h=64),
     "c3_sp4": LagaShape(S=8192, h=32),
     "c3_sp8": LagaShape(S=8192, h=16),
+    "c4": LagaShape(S=16384, h=16),     # the absorbed form on c2's inputs (same shapes, same seed)
 }
 CONFIG_SEEDS = {"c0": 1000, "c1": 1001, "c2": 1002, "c3_sp1": 1003, "c3_sp2": 1003, "c3_sp4": 1003,
                 "c3_sp8": 1003, "c4": 1002}

@@ -34,6 +34,8 @@ SIGNATURES = {
     "laga_bwd_workspace_bytes": (_sz, [_ci] * 6 + [_cu]),
     "laga_fwd": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
     "laga_bwd": (_ci, [_vp] * 7 + [_ci] * 6 + [_cf, _ci] + [_vp] * 4 + [_vp, _sz, _cu, _vp]),
+    "laga_absorbed_fwd_workspace_bytes": (_sz, [_ci] * 6),
+    "laga_absorbed_fwd": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
     "laga_up_project": (_ci, [_vp, _vp] + [_ci] * 5 + [_vp, _vp, _vp]),
     "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
     "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
@@ -44,7 +46,7 @@ SIGNATURES = {
 }
 BUILTIN_SCRATCH_MAX_TOKEN_HEADS = 32768   # S * h limit of laga_fwd_builtin_scratch (16 MiB of bf16 KV)
 KERNELS = {"up_project": 0, "attn_fwd": 1, "bwd_delta": 2, "attn_bwd_dkv": 3, "attn_bwd_dq": 4,
-           "dkpe_reduce": 5, "dckv_gemm": 6, "dw_gemm": 7}
+           "dkpe_reduce": 5, "dckv_gemm": 6, "dw_gemm": 7, "q_absorb": 8, "attn_absorbed": 9, "v_project": 10}
 
 
 class LagaError(RuntimeError):
@@ -162,6 +164,36 @@ def fwd(q, c_kv, k_pe, w_kv_b, d_v=128, softmax_scale=None, causal=True, out=Non
                             float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse), _ptr(workspace),
                             workspace.numel(), 0, _stream(stream, dev))
     _check(rc, "laga_fwd")
+    return out, lse, workspace
+
+
+def absorbed_fwd_workspace_bytes(S, h, d_c=512, d_nope=128, d_rope=64, d_v=128) -> int:
+    return int(lib().laga_absorbed_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v))
+
+
+def absorbed_fwd(q, c_kv, k_pe, w_kv_b, d_v=128, softmax_scale=None, causal=True, out=None, lse=None, workspace=None,
+                 stream=None):
+    """laga_absorbed_fwd: the absorbed form of the forward (comparison path).  Returns (out, lse, workspace)."""
+    S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
+    dev = same_device(q, c_kv, k_pe, w_kv_b, out, lse, workspace)
+    if softmax_scale is None:
+        softmax_scale = (d_nope + d_rope) ** -0.5
+    if out is None:
+        out = torch.empty(S, h, d_v, dtype=torch.bfloat16, device=dev)
+    if lse is None:
+        lse = torch.empty(S, h, dtype=torch.float32, device=dev)
+    _dev(out, torch.bfloat16, (S, h, d_v), "out")
+    _dev(lse, torch.float32, (S, h), "lse")
+    need = absorbed_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v)
+    if need == 0:
+        raise LagaError(ERR_UNSUPPORTED, "laga_absorbed_fwd_workspace_bytes")
+    if workspace is None:
+        workspace = alloc_workspace(need, dev)
+    with _on(dev):
+        rc = lib().laga_absorbed_fwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope, d_v,
+                                     float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse), _ptr(workspace),
+                                     workspace.numel(), 0, _stream(stream, dev))
+    _check(rc, "laga_absorbed_fwd")
     return out, lse, workspace
 
 
