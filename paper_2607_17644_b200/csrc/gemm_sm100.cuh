@@ -212,4 +212,202 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     if (warp == 1) { tc_fence_after_sync(); tmem_dealloc(tmem_base, kTmemCols); }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same GEMM on CTA PAIRS (cluster of two, tcgen05 cta_group::2): a pair owns 256 x BN output tiles,
+// each CTA holds its own 128 rows of A and half of the BN columns of B, so a CTA fills (and the MMAs read)
+// 16 + 16 KB per 64-deep k-stage instead of 16 + 32 KB for the same 128 x BN outputs per CTA.  With K = 512
+// the one-CTA kernel is bound by those fills (it moves 384 KB from L2 for every 33 MFLOP tile).
+// Roles per CTA as above; only the even CTA's warp 1 issues MMAs and commits, to barriers in both CTAs.
+// The full barriers live in the even CTA and count the bytes of both CTAs' loads; the odd CTA's epilogue
+// warps release the accumulator buffer with arrivals on the even CTA's barrier.
+template <int BN, int STAGES>
+struct GemmPairSmem {
+    static constexpr int kABytes = 128 * 64 * 2;
+    static constexpr int kBBytes = (BN / 2) * 64 * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarrierOffset = STAGES * kStageBytes;
+    static constexpr int kTotalBytes = kBarrierOffset + 256;
+};
+
+template <int BN, int STAGES, bool A_MN, bool B_MN, int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
+gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                       const GemmArgs args) {
+    using L = GemmPairSmem<BN, STAGES>;
+    static_assert(2 * BN <= 512 && BN % 128 == 0, "two accumulators must fit in TMEM; each CTA holds whole 64-column slabs");
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::kBarrierOffset);   // used in the even CTA only
+    uint64_t* empty_bar = full_bar + STAGES;   // both CTAs: the stage's MMAs have completed
+    uint64_t* acc_full = empty_bar + STAGES;   // [2] both CTAs
+    uint64_t* acc_empty = acc_full + 2;        // [2] even CTA: 256 arrivals (both CTAs' epilogue threads)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int tiles_n = args.N / BN;
+    const int tiles_m = (args.M + 255) / 256;
+    const int tiles_per_batch = tiles_n * tiles_m * args.n_splits;
+    const int total_tiles = tiles_per_batch * args.batches;
+    const int total_k_tiles = (args.K + 63) / 64;
+    constexpr uint32_t kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 256); }
+        abort_flag->value = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_b);
+        if ((smem_u32(smem) & 1023u) != 0u) {
+            abort_flag->value = 1;
+            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD4u);
+        }
+    }
+    if (warp == 1) { tmem_alloc_pair(tmem_slot, kTmemCols); tmem_relinquish_pair(); }
+    for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < args.zero_count;
+         z += static_cast<size_t>(gridDim.x) * blockDim.x)
+        args.zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync();            // the peer's barriers exist before anything can arrive on them
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const bool run = abort_flag->value == 0u;   // (the layout is the same in both CTAs: they agree)
+
+    auto k_range = [&](int split, int& kt_begin, int& n_kt) {
+        kt_begin = split * args.k_tiles_per_split;
+        const int kt_end = min(total_k_tiles, kt_begin + args.k_tiles_per_split);
+        n_kt = max(0, kt_end - kt_begin);
+    };
+
+    if (!run) {
+        // fall through to the common exit
+    } else if (warp == 0) {
+        if (elect_one()) {
+            uint32_t kc = 0;
+            bool ok = true;
+            for (int t = pair; t < total_tiles && ok; t += n_pairs) {
+                const int batch = t / tiles_per_batch, tb = t - batch * tiles_per_batch;
+                const int n0 = (tb % tiles_n) * BN + static_cast<int>(rank) * (BN / 2);
+                const int m0 = ((tb / tiles_n) % tiles_m) * 256 + static_cast<int>(rank) * 128;
+                const int a_off = batch * args.a_step, b_off = batch * args.b_step;
+                int kt_begin, n_kt;
+                k_range(tb / (tiles_n * tiles_m), kt_begin, n_kt);
+                for (int i = 0; i < n_kt; ++i, ++kc) {
+                    const int s = kc % STAGES;
+                    ok = mbar_wait(&empty_bar[s], ((kc / STAGES) & 1) ^ 1, abort_flag, args.status, 0x110);
+                    if (!ok) break;
+                    uint8_t* sa = smem + s * L::kStageBytes;
+                    uint8_t* sb = sa + L::kABytes;
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * L::kStageBytes);   // both CTAs' bytes
+                    const uint32_t bar = cluster_map(&full_bar[s], 0);
+                    const int k0 = (kt_begin + i) * 64;
+                    if (A_MN) {
+                        tma_load_2d_pair(sa, &tmap_a, bar, a_off + m0, k0);
+                        tma_load_2d_pair(sa + 8192, &tmap_a, bar, a_off + m0 + 64, k0);
+                    } else {
+                        tma_load_2d_pair(sa, &tmap_a, bar, a_off + k0, m0);
+                    }
+                    if (B_MN) {
+                        for (int j = 0; j < BN / 128; ++j)
+                            tma_load_2d_pair(sb + j * 8192, &tmap_b, bar, b_off + n0 + j * 64, k0);
+                    } else {
+                        tma_load_2d_pair(sb, &tmap_b, bar, b_off + k0, n0);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (rank == 0 && elect_one()) {
+            constexpr uint32_t idesc = make_idesc_bf16(256, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+            uint32_t kc = 0, it = 0;
+            bool ok = true;
+            for (int t = pair; t < total_tiles && ok; t += n_pairs, ++it) {
+                int kt_begin, n_kt;
+                k_range((t % tiles_per_batch) / (tiles_n * tiles_m), kt_begin, n_kt);
+                const uint32_t buf = it & 1;
+                ok = mbar_wait(&acc_empty[buf], ((it >> 1) & 1) ^ 1, abort_flag, args.status, 0x211);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t tmem_acc = tmem_base + buf * BN;
+                for (int i = 0; i < n_kt; ++i, ++kc) {
+                    const int s = kc % STAGES;
+                    ok = mbar_wait(&full_bar[s], (kc / STAGES) & 1, abort_flag, args.status, 0x210);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_u32(smem + s * L::kStageBytes);
+                    const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t da = A_MN ? desc_mn_major(sa + k * 2048, 8192) : desc_k_major(sa + k * 32);
+                        const uint64_t db = B_MN ? desc_mn_major(sb + k * 2048, 8192) : desc_k_major(sb + k * 32);
+                        mma_ss_pair(tmem_acc, da, db, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    }
+                    mma_commit_pair(&empty_bar[s], 3);
+                }
+                if (ok) mma_commit_pair(&acc_full[buf], 3);
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+        const uint32_t acc_empty_leader[2] = {cluster_map(&acc_empty[0], 0), cluster_map(&acc_empty[1], 0)};
+        uint32_t it = 0;
+        bool ok = true;
+        for (int t = pair; t < total_tiles && ok; t += n_pairs, ++it) {
+            const int batch = t / tiles_per_batch, tb = t - batch * tiles_per_batch;
+            const int n0 = batch * args.c_step + (tb % tiles_n) * BN;
+            const int m0 = ((tb / tiles_n) % tiles_m) * 256 + static_cast<int>(rank) * 128;
+            int kt_begin, n_kt;
+            k_range(tb / (tiles_n * tiles_m), kt_begin, n_kt);
+            const uint32_t buf = it & 1;
+            const int row = m0 + quarter * 32 + lane;
+            ok = mbar_wait_warp(&acc_full[buf], (it >> 1) & 1, abort_flag, args.status, 0x310);
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (n_kt > 0) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t r[32];
+                    __syncwarp();
+                    tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 32, r);
+                    tmem_ld_wait();
+                    if (row < args.M) {
+                        if (EPI == EPI_BF16) {
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(args.C) +
+                                                 static_cast<size_t>(row) * args.ldc + n0 + c * 32;
+                            uint4* dst4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                uint4 o;
+                                o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                                o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                                o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                                o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                                dst4[v] = o;
+                            }
+                        } else {
+                            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.C) +
+                                                                    static_cast<size_t>(row) * args.ldc + n0 + c * 32);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                atomicAdd(dst + v, make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                                                               __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3])));
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            tc_fence_before_sync();
+            mbar_arrive_cluster(acc_empty_leader[buf]);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync();            // neither CTA frees TMEM or leaves while the peer may still use it or its barriers
+    if (warp == 1) { tc_fence_after_sync(); tmem_dealloc_pair(tmem_base, kTmemCols); }
+}
+
 }  // namespace laga

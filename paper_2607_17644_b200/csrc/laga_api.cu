@@ -80,6 +80,7 @@ int launch_status() { return cudaGetLastError() == cudaSuccess ? LAGA_OK : LAGA_
 
 // ---- per-device facts, looked up once per device (thread-safe) ------------------------------------
 constexpr int kMaxDevices = 64;
+constexpr int kGemmStages = 6;      // 64-deep k-stages of the CTA-pair GEMM (32 KB each)
 struct DeviceInfo {
     std::once_flag once;
     int rc = LAGA_ERR_CUDA;
@@ -100,10 +101,10 @@ void init_device(DeviceInfo* info, int dev) {
     if (major != 10) { info->rc = LAGA_ERR_UNSUPPORTED; return; }
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) info->sms = sms;
     // every kernel of the library asks for more than the default 48 KB of dynamic shared memory: opt in once
-    using G = GemmSmem<256, 4>;
-    bool ok = allow_smem(gemm_sm100_kernel<256, 4, false, true, EPI_BF16>, G::kTotalBytes) &&
-              allow_smem(gemm_sm100_kernel<256, 4, false, false, EPI_BF16>, G::kTotalBytes) &&
-              allow_smem(gemm_sm100_kernel<256, 4, true, true, EPI_ATOMIC_F32>, G::kTotalBytes) &&
+    using G = GemmPairSmem<256, kGemmStages>;
+    bool ok = allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, false, true, EPI_BF16>, G::kTotalBytes) &&
+              allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, false, false, EPI_BF16>, G::kTotalBytes) &&
+              allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, true, true, EPI_ATOMIC_F32>, G::kTotalBytes) &&
               allow_smem(gemm_sm100_kernel<128, 4, false, true, EPI_BF16>, GemmSmem<128, 4>::kTotalBytes) &&
               allow_smem(attn_absorbed_fwd_sm100_kernel<true>, AttnAbsorbedSmem::kTotalBytes) &&
               allow_smem(attn_absorbed_fwd_sm100_kernel<false>, AttnAbsorbedSmem::kTotalBytes) &&
@@ -158,6 +159,12 @@ int check_pointers(std::initializer_list<const void*> ptrs) {
 unsigned persistent_grid(int total_tiles) {
     const int sms = sm_count();
     return static_cast<unsigned>(total_tiles < sms ? (total_tiles < 1 ? 1 : total_tiles) : sms);
+}
+
+// The CTA-pair GEMM launches whole pairs: one pair per two SMs (fewer if there are fewer 256-row tiles).
+unsigned pair_grid(int total_tiles) {
+    const int pairs = sm_count() / 2;
+    return 2u * static_cast<unsigned>(total_tiles < pairs ? (total_tiles < 1 ? 1 : total_tiles) : pairs);
 }
 
 // ---- tensor-map cache ------------------------------------------------------------------------------
@@ -237,14 +244,14 @@ WorkSchedule make_schedule(int n_tiles, int S, int h, unsigned* counter) {
 // ---- Algorithm 1 step 4: KV[S, N] = c_kv[S, d_c] . W[d_c, N] ------------------------------------
 int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
                       cudaStream_t stream) {
-    constexpr int BN = 256, STAGES = 4;
-    auto kernel = gemm_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
-    using L = GemmSmem<BN, STAGES>;
+    constexpr int BN = 256, STAGES = kGemmStages;
+    auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
+    using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
     if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
     GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status, nullptr, 0, 1, 0, 0, 0};
-    dim3 grid(persistent_grid((N / BN) * ((S + 127) / 128)), 1, 1);
+    dim3 grid(pair_grid((N / BN) * ((S + 255) / 256)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
@@ -255,14 +262,14 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
 // GEMM that follows accumulates into it with atomics.
 int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float* clear, size_t clear_floats,
                 unsigned* status, cudaStream_t stream) {
-    constexpr int BN = 256, STAGES = 4;
-    auto kernel = gemm_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
-    using L = GemmSmem<BN, STAGES>;
+    constexpr int BN = 256, STAGES = kGemmStages;
+    auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
+    using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
-    if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN / 2)) return LAGA_ERR_CUDA;
     GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status, reinterpret_cast<float4*>(clear), clear_floats / 4, 1, 0, 0, 0};
-    dim3 grid(persistent_grid((kDc / BN) * ((S + 127) / 128)), 1, 1);
+    dim3 grid(pair_grid((kDc / BN) * ((S + 255) / 256)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
@@ -272,17 +279,17 @@ int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float
 // (launch_dckv does it) or wants added to.
 int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool deterministic,
               unsigned* status, cudaStream_t stream) {
-    constexpr int BN = 256, STAGES = 4;
-    auto kernel = gemm_sm100_kernel<BN, STAGES, true, true, EPI_ATOMIC_F32>;
-    using L = GemmSmem<BN, STAGES>;
+    constexpr int BN = 256, STAGES = kGemmStages;
+    auto kernel = gemm_pair_sm100_kernel<BN, STAGES, true, true, EPI_ATOMIC_F32>;
+    using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 64)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tb, dkv, N, S, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;
     // Split the sequence so that tiles x splits fills whole waves of the persistent grid: the smallest
     // split count (fewest atomics) whose last wave is at least 90 % full, else the best found.
-    const int tiles = (kDc / 128) * (N / BN);
+    const int tiles = (kDc / 256) * (N / BN);
     const int k_tiles = (S + 63) / 64;
-    const int sms = sm_count();
+    const int sms = sm_count() / 2;       // CTA pairs
     int splits = 1;
     double best = 0.0;
     for (int s = 1; s <= 16 && s <= k_tiles && !deterministic; ++s) {   // one split: one add per element
@@ -294,7 +301,7 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool d
     const int per_split = (k_tiles + splits - 1) / splits;
     splits = (k_tiles + per_split - 1) / per_split;
     GemmArgs a{kDc, N, S, per_split, splits, dw, N, status, nullptr, 0, 1, 0, 0, 0};
-    dim3 grid(persistent_grid(tiles * splits), 1, 1);
+    dim3 grid(pair_grid(tiles * splits), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
@@ -402,15 +409,15 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
 // q_abs[S, h, d_c] = q_nope[S, h, d_n] . W_uk[h]^T, batched over the heads: head i reads columns
 // [192 i, 192 i + 128) of q and columns [256 i, 256 i + 128) of W (rows = latent index = the GEMM's N).
 int launch_q_absorb(const void* q, const void* w, int S, int h, void* q_abs, unsigned* status, cudaStream_t stream) {
-    constexpr int BN = 256, STAGES = 4;
-    auto kernel = gemm_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
-    using L = GemmSmem<BN, STAGES>;
+    constexpr int BN = 256, STAGES = kGemmStages;
+    auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
+    using L = GemmPairSmem<BN, STAGES>;
     const uint64_t q_row = static_cast<uint64_t>(h) * (kDn + kDr), w_row = static_cast<uint64_t>(h) * (kDn + kDv);
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, q, q_row, S, q_row * 2, 128)) return LAGA_ERR_CUDA;
-    if (!cached_tmap_bf16(&tb, w, w_row, kDc, w_row * 2, BN)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tb, w, w_row, kDc, w_row * 2, BN / 2)) return LAGA_ERR_CUDA;
     GemmArgs a{S, kDc, kDn, kDn / 64, 1, q_abs, h * kDc, status, nullptr, 0, h, kDn + kDr, kDn + kDv, kDc};
-    dim3 grid(persistent_grid((kDc / BN) * ((S + 127) / 128) * h), 1, 1);
+    dim3 grid(pair_grid((kDc / BN) * ((S + 255) / 256) * h), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_Q_ABSORB, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
     return launch_status();
 }
