@@ -14,6 +14,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 ROOT = os.path.dirname(PKG_DIR)
 LIB_PATH = os.path.join(PKG_DIR, "liblaga.so")
+DEBUG_LIB_PATH = os.path.join(PKG_DIR, "liblaga_debug.so")   # the checked build (-DLAGA_DEBUG), see sm100_ptx.cuh
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "--expt-relaxed-constexpr"]
@@ -24,21 +25,25 @@ def sources():
             sorted(glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))))
 
 
-def build(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
+def build(force: bool = False, verbose: bool = False, extra_flags=(), debug: bool = False) -> str:
+    """Build the library (debug=True: the checked build, whose kernels verify their own index arithmetic
+    and report LAGA_ERR_DEVICE_CHECK instead of making a bad access; selected at run time by LAGA_DEBUG=1)."""
     cus, deps = sources()
+    target = DEBUG_LIB_PATH if debug else LIB_PATH
     newest = max(os.path.getmtime(p) for p in cus + deps)
-    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= newest:
-        return LIB_PATH
+    if not force and os.path.exists(target) and os.path.getmtime(target) >= newest:
+        return target
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
-    cmd = [nvcc, *NVCC_FLAGS, *extra_flags, "-o", tmp, *cus]
+    tmp = target + f".tmp{os.getpid()}"
+    cmd = [nvcc, *NVCC_FLAGS, *(("-DLAGA_DEBUG=1",) if debug else ()), *extra_flags, "-o", tmp, *cus]
     if verbose:
         print(" ".join(cmd), file=sys.stderr)
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, target)
+    return target
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose=True,
-                extra_flags=("-Xptxas", "-v") if "--ptxas-v" in sys.argv else ()))
+    flags = ("-Xptxas", "-v") if "--ptxas-v" in sys.argv else ()
+    print(build(force="--force" in sys.argv, verbose=True, extra_flags=flags))
+    print(build(force="--force" in sys.argv, verbose=True, extra_flags=flags, debug=True))

@@ -67,7 +67,8 @@ attn_absorbed_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_qabs, co
     uint64_t* p_full = bars + 12;    // [2]  P of tile T has replaced it
     uint64_t* pv_done = bars + 14;   // [2]  O += P V of tile T has completed
     uint64_t* all_done = bars + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+    uint64_t* quiesce_bar = bars + 17;   // abort path only: the MMA lane's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -86,6 +87,7 @@ attn_absorbed_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_qabs, co
             mbar_init(&s_full[s], 1); mbar_init(&p_full[s], 128); mbar_init(&pv_done[s], 1);
         }
         mbar_init(all_done, 1);
+        mbar_init(quiesce_bar, 1);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_qabs); tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_ckv); tma_prefetch_desc(&tmap_kpe);
@@ -106,24 +108,29 @@ attn_absorbed_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_qabs, co
         // misaligned shared memory: nothing was started, fall through to the common exit
     } else if (warp == 4) {
         if (elect_one()) {
+            ArmedBarriers armed(bars);
             mbar_arrive_expect_tx(q_full, 5 * L::kQSlab);
+            armed.arm(q_full, 0);
             for (int c = 0; c < 4; ++c)
-                tma_load_2d(smem + L::kQ + c * L::kQSlab, &tmap_qabs, q_full, head * 512 + other_col + c * 64, q0);
-            tma_load_2d(smem + L::kQ + 4 * L::kQSlab, &tmap_q, q_full, head * 192 + 128, q0);      // rope band of q
+                tma_load_2d_chk(args.status, smem + L::kQ + c * L::kQSlab, &tmap_qabs, q_full, head * 512 + other_col + c * 64, q0);
+            tma_load_2d_chk(args.status, smem + L::kQ + 4 * L::kQSlab, &tmap_q, q_full, head * 192 + 128, q0);      // rope band of q
             for (int j = 0; j < n_kv; ++j) {
                 const int s = j & 1;
                 const uint32_t ph = ((j >> 1) & 1) ^ 1;
                 uint8_t* stage = smem + L::kK + s * 9 * L::kKSlab;
                 if (!mbar_wait(&a_empty[s], ph, abort_flag, args.status, 0xB0)) break;
                 mbar_arrive_expect_tx(&a_full[s], 5 * L::kKSlab);
+                armed.arm(&a_full[s], ph ^ 1);
                 for (int c = 0; c < 4; ++c)
-                    tma_load_2d(stage + c * L::kKSlab, &tmap_ckv, &a_full[s], other_col + c * 64, j * BK);
-                tma_load_2d(stage + 4 * L::kKSlab, &tmap_kpe, &a_full[s], 0, j * BK);
+                    tma_load_2d_chk(args.status, stage + c * L::kKSlab, &tmap_ckv, &a_full[s], other_col + c * 64, j * BK);
+                tma_load_2d_chk(args.status, stage + 4 * L::kKSlab, &tmap_kpe, &a_full[s], 0, j * BK);
                 if (!mbar_wait(&b_empty[s], ph, abort_flag, args.status, 0xB1)) break;
                 mbar_arrive_expect_tx(&b_full[s], 4 * L::kKSlab);
+                armed.arm(&b_full[s], ph ^ 1);
                 for (int c = 0; c < 4; ++c)
-                    tma_load_2d(stage + (5 + c) * L::kKSlab, &tmap_ckv, &b_full[s], own_col + c * 64, j * BK);
+                    tma_load_2d_chk(args.status, stage + (5 + c) * L::kKSlab, &tmap_ckv, &b_full[s], own_col + c * 64, j * BK);
             }
+            if (abort_flag->value != 0u) armed.quiesce();
         }
     } else if (warp == 5) {
         if (elect_one()) {
@@ -167,6 +174,7 @@ attn_absorbed_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_qabs, co
                 mma_commit(&pv_done[s]);
             }
             if (ok) mma_commit(all_done);
+            if (abort_flag->value != 0u) { mma_commit(quiesce_bar); mbar_wait_quiesce(quiesce_bar, 0); }
         }
     } else {
         const int row = warp * 32 + lane;             // row inside the tile == TMEM lane
@@ -267,7 +275,7 @@ attn_absorbed_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_qabs, co
                 __syncwarp();
                 tmem_ld_x32(tmem_base + lane_addr + c * 32, o);
                 tmem_ld_wait();
-                if (valid) {
+                if (valid && device_check(aligned16_dev(dst) && head < args.h, args.status, 0xE60000u | c)) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         uint4 w;

@@ -169,7 +169,8 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     uint64_t* acc_full = bars + 16;   // the item's dK / dV are complete
     uint64_t* acc_empty = bars + 17;  // both groups have drained them
     ItemRing ring{bars + 18, bars + 20, reinterpret_cast<volatile int*>(bars + 22)};
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 23);
+    uint64_t* quiesce_bar = bars + 23;   // abort path only: the MMA lane's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -183,6 +184,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         mbar_init(p_full, 256); mbar_init(dv_done, 1); mbar_init(ds_full, 256); mbar_init(dk_done, 1);
         mbar_init(acc_full, 1); mbar_init(acc_empty, 256);
         for (int s = 0; s < 2; ++s) { mbar_init(&ring.full[s], 1); mbar_init(&ring.empty[s], 9); }
+        mbar_init(quiesce_bar, 1);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_do);
@@ -216,6 +218,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         if (elect_one()) {
             uint32_t T = 0;                      // running tile count of this CTA: ring positions and phases
             bool ok = true;
+            ArmedBarriers armed(bars);
             for (uint32_t n = 0; ok; ++n) {
                 const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
@@ -224,30 +227,34 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 ok = mbar_wait(kv_empty, (n & 1u) ^ 1u, abort_flag, args.status, 0x41);
                 if (!ok) break;
                 mbar_arrive_expect_tx(kv_full, 5 * L::kSlab);
-                tma_load_2d(smem + L::kK, &tmap_kv, kv_full, head * 256, t0);
-                tma_load_2d(smem + L::kK + L::kSlab, &tmap_kv, kv_full, head * 256 + 64, t0);
-                tma_load_2d(smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, t0);
-                tma_load_2d(smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, t0);
-                tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, kv_full, head * 256 + 192, t0);
+                armed.arm(kv_full, n & 1u);
+                tma_load_2d_chk(args.status, smem + L::kK, &tmap_kv, kv_full, head * 256, t0);
+                tma_load_2d_chk(args.status, smem + L::kK + L::kSlab, &tmap_kv, kv_full, head * 256 + 64, t0);
+                tma_load_2d_chk(args.status, smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, t0);
+                tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, t0);
+                tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, kv_full, head * 256 + 192, t0);
                 for (int j = 0; j < n_iter; ++j, ++T) {
                     const uint32_t sq = T % L::kQStages;
                     const int q0 = (j_begin + j) * 128;
                     ok = mbar_wait(&q_empty[sq], ((T / L::kQStages) & 1u) ^ 1u, abort_flag, args.status, 0x40);
                     if (!ok) break;
                     mbar_arrive_expect_tx(&q_full[sq], 3 * L::kSlab + 1024);
+                    armed.arm(&q_full[sq], (T / L::kQStages) & 1u);
                     uint8_t* dst_q = smem + L::kQ + sq * 3 * L::kSlab;
                     for (int c = 0; c < 3; ++c)
-                        tma_load_2d(dst_q + c * L::kSlab, &tmap_q, &q_full[sq], head * 192 + c * 64, q0);
+                        tma_load_2d_chk(args.status, dst_q + c * L::kSlab, &tmap_q, &q_full[sq], head * 192 + c * 64, q0);
                     float* stat = reinterpret_cast<float*>(smem + L::kStat + sq * 1024);
                     bulk_load_1d(stat, args.stat_l2 + static_cast<size_t>(head) * args.S_pad + q0, 512, &q_full[sq]);
                     bulk_load_1d(stat + 128, args.stat_delta + static_cast<size_t>(head) * args.S_pad + q0, 512, &q_full[sq]);
                     ok = mbar_wait(do_empty, (T & 1u) ^ 1u, abort_flag, args.status, 0x42);
                     if (!ok) break;
                     mbar_arrive_expect_tx(do_full, 2 * L::kSlab);
+                    armed.arm(do_full, T & 1u);
                     for (int c = 0; c < 2; ++c)
-                        tma_load_2d(smem + L::kDo + c * L::kSlab, &tmap_do, do_full, head * 128 + c * 64, q0);
+                        tma_load_2d_chk(args.status, smem + L::kDo + c * L::kSlab, &tmap_do, do_full, head * 128 + c * 64, q0);
                 }
             }
+            if (abort_flag->value != 0u) armed.quiesce();
         }
     } else if (warp == 1) {
         if (elect_one()) {
@@ -330,6 +337,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (ok) mma_commit(acc_full);
                 T0 += static_cast<uint32_t>(n_iter);
             }
+            if (abort_flag->value != 0u) { mma_commit(quiesce_bar); mbar_wait_quiesce(quiesce_bar, 0); }
         }
     } else {
         const int g = (warp - 2) >> 2;               // consumer warpgroup: query columns [64g, 64g+64) of every tile
@@ -444,6 +452,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 tmem_ld_x32(tmem_dk + lane_addr + c * 32, r);
                 tmem_ld_wait();
                 if (!valid) continue;
+                if (!device_check(head < args.h && aligned16_dev(dkv_row) && aligned16_dev(dkr_row), args.status, 0xE40000u | c)) continue;
                 if (c == 4 || c == 5) {
 #pragma unroll
                     for (int v = 0; v < 8; ++v) {
@@ -535,7 +544,8 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     uint64_t* acc_full = bars + 15;   // the item's dQ is complete
     uint64_t* acc_empty = bars + 16;  // both groups have drained it
     ItemRing ring{bars + 17, bars + 19, reinterpret_cast<volatile int*>(bars + 21)};
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
+    uint64_t* quiesce_bar = bars + 22;   // abort path only: the MMA lane's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 23);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -549,6 +559,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         mbar_init(s_full, 1); mbar_init(s_read, 256); mbar_init(dp_full, 1); mbar_init(ds_full, 256);
         mbar_init(acc_full, 1); mbar_init(acc_empty, 256);
         for (int s = 0; s < 2; ++s) { mbar_init(&ring.full[s], 1); mbar_init(&ring.empty[s], 9); }
+        mbar_init(quiesce_bar, 1);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
@@ -582,14 +593,16 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         if (elect_one()) {
             uint32_t T0 = 0;
             bool ok = true;
+            ArmedBarriers armed(bars);
             auto load_k = [&](uint32_t T, int j, int head) -> bool {
                 const uint32_t st = T % kDqKStages;
                 if (!mbar_wait(&k_empty[st], ((T / kDqKStages) & 1u) ^ 1u, abort_flag, args.status, 0x70)) return false;
                 mbar_arrive_expect_tx(&k_full[st], 3 * L::kSlab);
+                armed.arm(&k_full[st], (T / kDqKStages) & 1u);
                 uint8_t* sk = smem + L::kK + st * 3 * L::kSlab;
-                tma_load_2d(sk, &tmap_kv, &k_full[st], head * 256, j * 128);
-                tma_load_2d(sk + L::kSlab, &tmap_kv, &k_full[st], head * 256 + 64, j * 128);
-                tma_load_2d(sk + 2 * L::kSlab, &tmap_kpe, &k_full[st], 0, j * 128);
+                tma_load_2d_chk(args.status, sk, &tmap_kv, &k_full[st], head * 256, j * 128);
+                tma_load_2d_chk(args.status, sk + L::kSlab, &tmap_kv, &k_full[st], head * 256 + 64, j * 128);
+                tma_load_2d_chk(args.status, sk + 2 * L::kSlab, &tmap_kpe, &k_full[st], 0, j * 128);
                 return true;
             };
             for (uint32_t n = 0; ok; ++n) {
@@ -600,8 +613,9 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 ok = mbar_wait(q_empty, (n & 1u) ^ 1u, abort_flag, args.status, 0x72);
                 if (!ok) break;
                 mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
+                armed.arm(q_full, n & 1u);
                 for (int c = 0; c < 3; ++c)
-                    tma_load_2d(smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
+                    tma_load_2d_chk(args.status, smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
                 ok = load_k(T0, 0, head);
                 for (int j = 0; j < n_iter && ok; ++j) {
                     const uint32_t T = T0 + j;
@@ -610,11 +624,13 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     ok = mbar_wait(v_empty, (T & 1u) ^ 1u, abort_flag, args.status, 0x71);
                     if (!ok) break;
                     mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
-                    tma_load_2d(smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
-                    tma_load_2d(smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
+                    armed.arm(v_full, T & 1u);
+                    tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
+                    tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
                 }
                 T0 += static_cast<uint32_t>(n_iter);
             }
+            if (abort_flag->value != 0u) armed.quiesce();
         }
     } else if (warp == 1) {
         if (elect_one()) {
@@ -682,6 +698,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 if (ok) mma_commit(acc_full);
                 T0 += static_cast<uint32_t>(n_iter);
             }
+            if (abort_flag->value != 0u) { mma_commit(quiesce_bar); mbar_wait_quiesce(quiesce_bar, 0); }
         }
     } else {
         const int g = (warp - 2) >> 2;               // consumer group: key columns [64g, 64g+64) of the tile
@@ -709,6 +726,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 tmem_ld_x32(tmem_dq + lane_addr + c * 32, r);
                 tmem_ld_wait();
                 if (!valid) continue;
+                if (!device_check(head < args.h && aligned16_dev(dst), args.status, 0xE50000u | c)) continue;
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
                     uint4 w;

@@ -93,7 +93,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     uint64_t* l_ready = bars + 23;   // both groups have stored their row sums
     uint64_t* o_empty = bars + 24;   // both groups have drained O
     ItemRing ring{bars + 25, bars + 27, reinterpret_cast<volatile int*>(bars + 29)};
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 30);
+    uint64_t* quiesce_bar = bars + 30;   // abort path only: the MMA lane's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 31);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
     float* mref = reinterpret_cast<float*>(smem + L::kMref);
     float* lsum = reinterpret_cast<float*>(smem + L::kLsum);
@@ -113,6 +114,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
         mbar_init(all_done, 1);
         mbar_init(l_ready, 256);
         mbar_init(o_empty, 256);
+        mbar_init(quiesce_bar, 1);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
@@ -145,6 +147,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
         if (elect_one()) {
             uint32_t T = 0;
             bool ok = true;
+            ArmedBarriers armed(bars);
             for (uint32_t n = 0; ok; ++n) {
                 const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
@@ -156,16 +159,19 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     if (!ok) break;
                     uint8_t* dk = smem + L::kK + s * 3 * L::kSlab;
                     mbar_arrive_expect_tx(&k_full[s], 3 * L::kSlab);
-                    tma_load_2d(dk, &tmap_kv, &k_full[s], head * 256, j * BK);
-                    tma_load_2d(dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * BK);
-                    tma_load_2d(dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * BK);
+                    armed.arm(&k_full[s], (T / kFwdStages) & 1u);
+                    tma_load_2d_chk(args.status, dk, &tmap_kv, &k_full[s], head * 256, j * BK);
+                    tma_load_2d_chk(args.status, dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * BK);
+                    tma_load_2d_chk(args.status, dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * BK);
                 }
             }
+            if (abort_flag->value != 0u) armed.quiesce();
         }
     } else if (warp == 10) {
         if (elect_one()) {
             uint32_t T = 0;
             bool ok = true;
+            ArmedBarriers armed(bars);
             for (uint32_t n = 0; ok; ++n) {
                 const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
@@ -177,10 +183,12 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     if (!ok) break;
                     uint8_t* dv = smem + L::kV + s * 2 * L::kSlab;
                     mbar_arrive_expect_tx(&v_full[s], 2 * L::kSlab);
-                    tma_load_2d(dv, &tmap_kv, &v_full[s], head * 256 + 128, j * BK);
-                    tma_load_2d(dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * BK);
+                    armed.arm(&v_full[s], (T / kFwdStages) & 1u);
+                    tma_load_2d_chk(args.status, dv, &tmap_kv, &v_full[s], head * 256 + 128, j * BK);
+                    tma_load_2d_chk(args.status, dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * BK);
                 }
             }
+            if (abort_flag->value != 0u) armed.quiesce();
         }
     } else if (warp == 9) {
         if (elect_one()) {
@@ -248,6 +256,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 if (ok) mma_commit(all_done);
                 T0 += static_cast<uint32_t>(n_kv);
             }
+            if (abort_flag->value != 0u) { mma_commit(quiesce_bar); mbar_wait_quiesce(quiesce_bar, 0); }
         }
     } else {
         const int g = warp >> 2;                      // softmax warpgroup: tiles whose running count has parity g
@@ -274,7 +283,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 __syncwarp();
                 tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
                 tmem_ld_wait();
-                if (valid) {
+                if (valid && device_check(aligned16_dev(dst) && head < args.h && sq_idx >= 0, args.status, 0xE30000u | c)) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         uint4 w;

@@ -56,7 +56,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     uint64_t* empty_bar = full_bar + STAGES;
     uint64_t* acc_full = empty_bar + STAGES;   // [2]
     uint64_t* acc_empty = acc_full + 2;        // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* quiesce_bar = acc_empty + 2;     // abort path only: the MMA lane's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(quiesce_bar + 1);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -70,6 +71,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+        mbar_init(quiesce_bar, 1);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_a);
@@ -94,6 +96,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (elect_one()) {
             uint32_t kc = 0;   // running k-iteration count: stage = kc % STAGES, phase = (kc / STAGES) & 1
             bool ok = true;
+            ArmedBarriers armed(full_bar);
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const int batch = t / tiles_per_batch, tb = t - batch * tiles_per_batch;
                 const int n0 = (tb % tiles_n) * BN, m0 = ((tb / tiles_n) % tiles_m) * 128;
@@ -107,21 +110,23 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     uint8_t* sa = smem + s * L::kStageBytes;
                     uint8_t* sb = sa + L::kABytes;
                     mbar_arrive_expect_tx(&full_bar[s], L::kStageBytes);
+                    armed.arm(&full_bar[s], (kc / STAGES) & 1);
                     const int k0 = (kt_begin + i) * 64;
                     if (A_MN) {   // global A is [K rows, M contiguous]: two slabs of 64 K-rows x 64 M
-                        tma_load_2d(sa, &tmap_a, &full_bar[s], a_off + m0, k0);
-                        tma_load_2d(sa + 8192, &tmap_a, &full_bar[s], a_off + m0 + 64, k0);
+                        tma_load_2d_chk(args.status, sa, &tmap_a, &full_bar[s], a_off + m0, k0);
+                        tma_load_2d_chk(args.status, sa + 8192, &tmap_a, &full_bar[s], a_off + m0 + 64, k0);
                     } else {      // global A is [M rows, K contiguous]: one slab of 128 rows x 64 K
-                        tma_load_2d(sa, &tmap_a, &full_bar[s], a_off + k0, m0);
+                        tma_load_2d_chk(args.status, sa, &tmap_a, &full_bar[s], a_off + k0, m0);
                     }
                     if (B_MN) {
                         for (int j = 0; j < BN / 64; ++j)
-                            tma_load_2d(sb + j * 8192, &tmap_b, &full_bar[s], b_off + n0 + j * 64, k0);
+                            tma_load_2d_chk(args.status, sb + j * 8192, &tmap_b, &full_bar[s], b_off + n0 + j * 64, k0);
                     } else {
-                        tma_load_2d(sb, &tmap_b, &full_bar[s], b_off + k0, n0);
+                        tma_load_2d_chk(args.status, sb, &tmap_b, &full_bar[s], b_off + k0, n0);
                     }
                 }
             }
+            if (abort_flag->value != 0u) armed.quiesce();
         }
     } else if (warp == 1) {
         if (elect_one()) {
@@ -153,6 +158,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 if (ok) mma_commit(&acc_full[buf]);
             }
+            if (abort_flag->value != 0u) { mma_commit(quiesce_bar); mbar_wait_quiesce(quiesce_bar, 0); }
         }
     } else {
         // Epilogue: TMEM lane = output row within the tile, TMEM column = output column.
@@ -182,6 +188,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(args.C) +
                                                  static_cast<size_t>(row) * args.ldc + n0 + c * 32;
                             uint4* dst4 = reinterpret_cast<uint4*>(dst);
+                            if (!device_check(aligned16_dev(dst) && n0 + c * 32 + 32 <= args.ldc, args.status, 0xE10000u | c)) continue;
 #pragma unroll
                             for (int v = 0; v < 4; ++v) {
                                 uint4 o;
@@ -194,6 +201,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         } else {
                             float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.C) +
                                                                     static_cast<size_t>(row) * args.ldc + n0 + c * 32);
+                            if (!device_check(aligned16_dev(dst) && n0 + c * 32 + 32 <= args.ldc, args.status, 0xE20000u | c)) continue;
 #pragma unroll
                             for (int v = 0; v < 8; ++v)
                                 atomicAdd(dst + v, make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
@@ -240,7 +248,8 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     uint64_t* empty_bar = full_bar + STAGES;   // both CTAs: the stage's MMAs have completed
     uint64_t* acc_full = empty_bar + STAGES;   // [2] both CTAs
     uint64_t* acc_empty = acc_full + 2;        // [2] even CTA: 256 arrivals (both CTAs' epilogue threads)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* quiesce_bar = acc_empty + 2;     // abort path only: the MMA lane's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(quiesce_bar + 1);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -256,6 +265,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 256); }
+        mbar_init(quiesce_bar, 1);
         abort_flag->value = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmap_a);
@@ -288,6 +298,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         if (elect_one()) {
             uint32_t kc = 0;
             bool ok = true;
+            ArmedBarriers armed(full_bar);
             for (int t = pair; t < total_tiles && ok; t += n_pairs) {
                 const int batch = t / tiles_per_batch, tb = t - batch * tiles_per_batch;
                 const int n0 = (tb % tiles_n) * BN + static_cast<int>(rank) * (BN / 2);
@@ -301,23 +312,26 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                     if (!ok) break;
                     uint8_t* sa = smem + s * L::kStageBytes;
                     uint8_t* sb = sa + L::kABytes;
-                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * L::kStageBytes);   // both CTAs' bytes
+                    if (rank == 0) { mbar_arrive_expect_tx(&full_bar[s], 2 * L::kStageBytes); armed.arm(&full_bar[s], (kc / STAGES) & 1); }   // both CTAs' bytes
                     const uint32_t bar = cluster_map(&full_bar[s], 0);
                     const int k0 = (kt_begin + i) * 64;
                     if (A_MN) {
-                        tma_load_2d_pair(sa, &tmap_a, bar, a_off + m0, k0);
-                        tma_load_2d_pair(sa + 8192, &tmap_a, bar, a_off + m0 + 64, k0);
+                        tma_load_2d_pair_chk(args.status, sa, &tmap_a, bar, a_off + m0, k0);
+                        tma_load_2d_pair_chk(args.status, sa + 8192, &tmap_a, bar, a_off + m0 + 64, k0);
                     } else {
-                        tma_load_2d_pair(sa, &tmap_a, bar, a_off + k0, m0);
+                        tma_load_2d_pair_chk(args.status, sa, &tmap_a, bar, a_off + k0, m0);
                     }
                     if (B_MN) {
                         for (int j = 0; j < BN / 128; ++j)
-                            tma_load_2d_pair(sb + j * 8192, &tmap_b, bar, b_off + n0 + j * 64, k0);
+                            tma_load_2d_pair_chk(args.status, sb + j * 8192, &tmap_b, bar, b_off + n0 + j * 64, k0);
                     } else {
-                        tma_load_2d_pair(sb, &tmap_b, bar, b_off + k0, n0);
+                        tma_load_2d_pair_chk(args.status, sb, &tmap_b, bar, b_off + k0, n0);
                     }
                 }
             }
+            // (the final cluster barrier keeps the odd CTA's shared memory alive until the even CTA has seen
+            // these barriers complete or given up on them)
+            if (abort_flag->value != 0u) armed.quiesce();
         }
     } else if (warp == 1) {
         if (rank == 0 && elect_one()) {
@@ -349,6 +363,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 }
                 if (ok) mma_commit_pair(&acc_full[buf], 3);
             }
+            if (abort_flag->value != 0u) { mma_commit_pair(quiesce_bar, 1); mbar_wait_quiesce(quiesce_bar, 0); }
         }
     } else {
         const int quarter = warp & 3;
@@ -379,6 +394,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                             __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(args.C) +
                                                  static_cast<size_t>(row) * args.ldc + n0 + c * 32;
                             uint4* dst4 = reinterpret_cast<uint4*>(dst);
+                            if (!device_check(aligned16_dev(dst) && n0 + c * 32 + 32 <= args.ldc, args.status, 0xE10000u | c)) continue;
 #pragma unroll
                             for (int v = 0; v < 4; ++v) {
                                 uint4 o;
@@ -391,6 +407,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         } else {
                             float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.C) +
                                                                     static_cast<size_t>(row) * args.ldc + n0 + c * 32);
+                            if (!device_check(aligned16_dev(dst) && n0 + c * 32 + 32 <= args.ldc, args.status, 0xE20000u | c)) continue;
 #pragma unroll
                             for (int v = 0; v < 8; ++v)
                                 atomicAdd(dst + v, make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),

@@ -106,6 +106,55 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, A
 }
 
 // ------------------------------------------------------------------------------------------------
+// Checked build.  Compiled with -DLAGA_DEBUG, every TMA issue and every global store of the kernels first
+// verifies its own index arithmetic (coordinate alignment, row / column bounds, pointer alignment).  A
+// failed check records kStatusCheck | site in the status word and the access is SKIPPED: the kernel runs
+// on (a skipped load shows up as a bounded-wait timeout at worst), nothing traps, and the host reads
+// LAGA_ERR_DEVICE_CHECK with the site from laga_query_status.  In the normal build the checks vanish.
+// ------------------------------------------------------------------------------------------------
+#ifdef LAGA_DEBUG
+constexpr bool kDeviceChecks = true;
+#else
+constexpr bool kDeviceChecks = false;
+#endif
+__device__ __forceinline__ bool device_check(bool cond, unsigned int* status, uint32_t site) {
+    if (!kDeviceChecks || cond) return true;
+    if (status) atomicCAS(status, kStatusOk, kStatusCheck | (site & 0xffffffu));
+    return false;
+}
+__device__ __forceinline__ bool aligned16_dev(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0u; }
+
+// ------------------------------------------------------------------------------------------------
+// Unwinding after a wait gave up.  A role that leaves its loop early may still have asynchronous work in
+// flight that targets this CTA's shared memory or TMEM: TMA copies it armed, MMAs it issued.  Before the CTA
+// frees TMEM and exits, the producer lane waits (1 ms at most per barrier, whatever the abort flag says) for
+// the copies it armed, and the MMA lane commits to a barrier of its own and waits for that.
+// ------------------------------------------------------------------------------------------------
+constexpr unsigned long long kQuiesceBudgetNs = 1000000ull;
+__device__ __forceinline__ void mbar_wait_quiesce(uint64_t* bar, uint32_t parity) {
+    const unsigned long long t0 = global_timer_ns();
+    while (!mbar_try_wait(bar, parity))
+        if (global_timer_ns() - t0 > kQuiesceBudgetNs) return;
+}
+// The barriers a producer lane has armed with expect_tx, with the parity of the phase each was last armed
+// for: two bit masks over the CTA's barrier array (all barriers of a kernel sit in one array of fewer than
+// 64), so the record lives in registers.
+struct ArmedBarriers {
+    uint64_t* base;
+    uint64_t armed = 0ull, parity = 0ull;
+    __device__ __forceinline__ explicit ArmedBarriers(uint64_t* barrier_array) : base(barrier_array) {}
+    __device__ __forceinline__ void arm(uint64_t* b, uint32_t ph) {
+        const uint64_t bit = 1ull << static_cast<uint32_t>(b - base);
+        armed |= bit;
+        parity = (ph & 1u) ? (parity | bit) : (parity & ~bit);
+    }
+    __device__ __forceinline__ void quiesce() const {
+        for (uint32_t i = 0; i < 64u; ++i)
+            if ((armed >> i) & 1ull) mbar_wait_quiesce(base + i, static_cast<uint32_t>((parity >> i) & 1ull));
+    }
+};
+
+// ------------------------------------------------------------------------------------------------
 // TMA (tiled bulk tensor copies global -> shared, completion on an mbarrier)
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
@@ -118,6 +167,14 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
+}
+
+// The same with the checked build's self-check: x on a 16-byte boundary (the hardware raises an illegal
+// instruction otherwise), y not negative, destination slab 1024-byte aligned.
+__device__ __forceinline__ void tma_load_2d_chk(unsigned int* status, void* smem_dst, const CUtensorMap* map, uint64_t* bar,
+                                                int x, int y) {
+    if (device_check((x & 7) == 0 && x >= 0 && y >= 0 && (smem_u32(smem_dst) & 1023u) == 0u, status, 0xE00000u | (x & 0xffff)))
+        tma_load_2d(smem_dst, map, bar, x, y);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -287,6 +344,11 @@ __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorM
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y)
         : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair_chk(unsigned int* status, void* smem_dst, const CUtensorMap* map,
+                                                     uint32_t bar_cluster_addr, int x, int y) {
+    if (device_check((x & 7) == 0 && x >= 0 && y >= 0 && (smem_u32(smem_dst) & 1023u) == 0u, status, 0xE00000u | (x & 0xffff)))
+        tma_load_2d_pair(smem_dst, map, bar_cluster_addr, x, y);
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t n_cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)), "r"(n_cols)

@@ -22,7 +22,10 @@ FLAG_ACCUM_DW = 1
 FLAG_DETERMINISTIC = 2
 FLAG_KV_SAVED = 4
 
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblaga.so")
+# LAGA_DEBUG=1 selects the checked build of the same kernels (liblaga_debug.so): every TMA issue and global
+# store verifies its index arithmetic first and reports LAGA_ERR_DEVICE_CHECK instead of a bad access.
+DEBUG = os.environ.get("LAGA_DEBUG", "0") not in ("", "0")
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblaga_debug.so" if DEBUG else "liblaga.so")
 _lib = None
 
 # name -> (restype, argtypes); mirrors include/laga.h one to one

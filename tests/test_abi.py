@@ -130,3 +130,14 @@ def test_binding_refuses_tensors_on_different_devices(laga):
     with pytest.raises(ValueError, match="different devices"):
         laga.same_device(a, b)
     assert laga.same_device(a, None, torch.ones(2)) == a.device
+
+
+def test_checked_build_exports_the_same_entry_points():
+    """liblaga_debug.so (-DLAGA_DEBUG: kernels that verify their own index arithmetic) is the same ABI."""
+    from paper_2607_17644_b200 import build
+    path = build.build(debug=True)
+    handle = ctypes.CDLL(path)
+    for name in declared_functions():
+        assert hasattr(handle, name), f"{name} missing from the checked build"
+    handle.laga_status_string.restype = ctypes.c_char_p
+    assert handle.laga_status_string(-6) == b"LAGA_ERR_DEVICE_CHECK"
