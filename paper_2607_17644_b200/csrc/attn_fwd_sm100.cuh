@@ -86,15 +86,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     uint64_t* v_full = bars + 7;     // [3]
     uint64_t* v_empty = bars + 10;   // [3]
     uint64_t* s_full = bars + 13;    // [3]  S of tile T is in TMEM buffer T % 3
-    uint64_t* p_full = bars + 16;    // [2]  group g has written P of its tile
-    uint64_t* pv_done = bars + 18;   // [2]  P V of a tile of group g has completed
-    uint64_t* max_done = bars + 20;  // [2]  group g has published the reference maxima of its tile
-    uint64_t* all_done = bars + 22;  // every MMA of the item has completed
-    uint64_t* l_ready = bars + 23;   // both groups have stored their row sums
-    uint64_t* o_empty = bars + 24;   // both groups have drained O
-    ItemRing ring{bars + 25, bars + 27, reinterpret_cast<volatile int*>(bars + 29)};
-    uint64_t* quiesce_bar = bars + 30;   // abort path only: the MMA lane's last commit
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 31);
+    // One barrier per SCORE BUFFER, not per softmax group: with three score tiles in flight a group can have
+    // delivered P of tile T+1 and of tile T+3 before the MMA lane (held up, say, by a late V stage) has looked
+    // at the first; a per-group barrier would then be two phases ahead of its waiter, whose parity test can
+    // no longer tell "done" from "not yet" (it waits for ever).  A buffer cannot be refilled before its
+    // previous P was consumed, so a per-buffer barrier never runs ahead.
+    uint64_t* p_full = bars + 16;    // [3]  P of tile T has replaced S in buffer T % 3
+    uint64_t* pv_done = bars + 19;   // [2]  P V of a tile of group g has completed
+    uint64_t* max_done = bars + 21;  // [2]  group g has published the reference maxima of its tile
+    uint64_t* all_done = bars + 23;  // every MMA of the item has completed
+    uint64_t* l_ready = bars + 24;   // both groups have stored their row sums
+    uint64_t* o_empty = bars + 25;   // both groups have drained O
+    ItemRing ring{bars + 26, bars + 28, reinterpret_cast<volatile int*>(bars + 30)};
+    uint64_t* quiesce_bar = bars + 31;   // abort path only: the MMA lane's last commit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 32);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
     float* mref = reinterpret_cast<float*>(smem + L::kMref);
     float* lsum = reinterpret_cast<float*>(smem + L::kLsum);
@@ -106,9 +111,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
         mbar_init(q_ready, 128);
         for (int s = 0; s < 3; ++s) {
             mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); mbar_init(&s_full[s], 1);
+            mbar_init(&p_full[s], 128);
         }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&p_full[s], 128); mbar_init(&pv_done[s], 1); mbar_init(&max_done[s], 128);
+            mbar_init(&pv_done[s], 1); mbar_init(&max_done[s], 128);
             mbar_init(&ring.full[s], 1); mbar_init(&ring.empty[s], 10);
         }
         mbar_init(all_done, 1);
@@ -231,7 +237,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     const uint32_t s = T % kFwdStages, g = T & 1u;
                     const uint32_t ph = (T / kFwdStages) & 1u;
                     if (!v_ok) ok = mbar_wait(&v_full[s], ph, abort_flag, args.status, 0x20);
-                    if (ok && !p_ok) ok = mbar_wait(&p_full[g], (T >> 1) & 1u, abort_flag, args.status, 0x21);
+                    if (ok && !p_ok) ok = mbar_wait(&p_full[s], ph, abort_flag, args.status, 0x21);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const bool more = j + 3 < n_kv;
@@ -249,7 +255,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                         if (!ok) break;
                         tc_fence_after_sync();
                         v_ok = mbar_try_wait(&v_full[(T + 1) % kFwdStages], ((T + 1) / kFwdStages) & 1u);
-                        p_ok = mbar_try_wait(&p_full[g ^ 1u], ((T + 1) >> 1) & 1u);
+                        p_ok = mbar_try_wait(&p_full[(T + 1) % kFwdStages], ((T + 1) / kFwdStages) & 1u);
                         qk_mmas(T + 3);
                     }
                 }
@@ -417,7 +423,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 tmem_st_x16(tmem_s + 32, pk + 32);
                 tmem_st_wait();
                 tc_fence_before_sync();
-                mbar_arrive(&p_full[g]);
+                mbar_arrive(&p_full[b]);
             }
             if (!ok) break;
             // Bring this group's sum to the final reference (set by the owner of the item's last tile) and add
