@@ -233,14 +233,22 @@ struct GemmPairSmem {
     static constexpr int kABytes = 128 * 64 * 2;
     static constexpr int kBBytes = (BN / 2) * 64 * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kBarrierOffset = STAGES * kStageBytes;
+    static constexpr int kStoreOffset = STAGES * kStageBytes;     // bf16 epilogue: 4 warps x 2 buffers x (32 rows x 128 B)
+    static constexpr int kStoreBytes = 4 * 2 * 4096;
+    static constexpr int kBarrierOffset = kStoreOffset + kStoreBytes;
     static constexpr int kTotalBytes = kBarrierOffset + 256;
 };
 
+// bf16 epilogue: every lane owns one output row; writing it straight to global memory costs one wavefront
+// per lane and 16-byte store (the rows are kilobytes apart), which for a 128 x 256 tile is as many load/store
+// cycles as the tile's MMAs take.  Instead each warp packs 64 columns of its 32 rows into a 128-byte-swizzled
+// 4 KB box in shared memory (4-way bank conflicts instead of 32 wavefronts) and one lane hands the box to TMA
+// (`tmap_c`: the output as [rows, ldc] bf16, box 64 x 32); two boxes per warp alternate so that packing the
+// next one overlaps the store of the last.  TMA clips rows past M.
 template <int BN, int STAGES, bool A_MN, bool B_MN, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
 gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                       const GemmArgs args) {
+                       const __grid_constant__ CUtensorMap tmap_c, const GemmArgs args) {
     using L = GemmPairSmem<BN, STAGES>;
     static_assert(2 * BN <= 512 && BN % 128 == 0, "two accumulators must fit in TMEM; each CTA holds whole 64-column slabs");
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -369,6 +377,8 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         const int quarter = warp & 3;
         const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
         const uint32_t acc_empty_leader[2] = {cluster_map(&acc_empty[0], 0), cluster_map(&acc_empty[1], 0)};
+        uint8_t* store_base = smem + L::kStoreOffset + quarter * 2 * 4096;   // this warp's two output boxes
+        uint32_t boxes = 0;
         uint32_t it = 0;
         bool ok = true;
         for (int t = pair; t < total_tiles && ok; t += n_pairs, ++it) {
@@ -383,28 +393,41 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             if (!ok) break;
             tc_fence_after_sync();
             if (n_kt > 0) {
+                if (EPI == EPI_BF16) {
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t r[32];
-                    __syncwarp();
-                    tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 32, r);
-                    tmem_ld_wait();
-                    if (row < args.M) {
-                        if (EPI == EPI_BF16) {
-                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(args.C) +
-                                                 static_cast<size_t>(row) * args.ldc + n0 + c * 32;
-                            uint4* dst4 = reinterpret_cast<uint4*>(dst);
-                            if (!device_check(aligned16_dev(dst) && n0 + c * 32 + 32 <= args.ldc, args.status, 0xE10000u | c)) continue;
+                    for (int c = 0; c < BN / 64; ++c, ++boxes) {
+                        uint32_t r[64];
+                        __syncwarp();
+                        tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 64, r);
+                        tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 64 + 32, r + 32);
+                        tmem_ld_wait();
+                        uint8_t* box = store_base + (boxes & 1u) * 4096;
+                        if (lane == 0) tma_store_wait_read<1>();       // the box used two stores ago has been read
+                        __syncwarp();
 #pragma unroll
-                            for (int v = 0; v < 4; ++v) {
-                                uint4 o;
-                                o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-                                o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-                                o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-                                o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-                                dst4[v] = o;
-                            }
-                        } else {
+                        for (int v = 0; v < 8; ++v) {                   // 16-byte chunk v of this lane's 128-byte row
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                            o.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                            o.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                            o.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                            *reinterpret_cast<uint4*>(box + lane * 128 + ((v ^ (lane & 7)) << 4)) = o;
+                        }
+                        fence_async_shared();
+                        __syncwarp();
+                        if (lane == 0 && device_check(((n0 + c * 64) & 7) == 0 && n0 + c * 64 + 64 <= args.ldc, args.status, 0xE70000u | c)) {
+                            tma_store_2d(&tmap_c, box, n0 + c * 64, m0 + quarter * 32);
+                            tma_store_commit();
+                        }
+                    }
+                } else {
+#pragma unroll 1
+                    for (int c = 0; c < BN / 32; ++c) {
+                        uint32_t r[32];
+                        __syncwarp();
+                        tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 32, r);
+                        tmem_ld_wait();
+                        if (row < args.M) {
                             float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.C) +
                                                                     static_cast<size_t>(row) * args.ldc + n0 + c * 32);
                             if (!device_check(aligned16_dev(dst) && n0 + c * 32 + 32 <= args.ldc, args.status, 0xE20000u | c)) continue;
@@ -420,6 +443,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             tc_fence_before_sync();
             mbar_arrive_cluster(acc_empty_leader[buf]);
         }
+        if (EPI == EPI_BF16 && lane == 0) tma_store_wait_all();   // the stores read shared memory until they complete
     }
     tc_fence_before_sync();
     __syncthreads();

@@ -250,9 +250,11 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
     if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
+    CUtensorMap tc;                                                                    // output boxes of 64 columns x 32 rows
+    if (!cached_tmap_bf16(&tc, kv, N, S, static_cast<uint64_t>(N) * 2, 32)) return LAGA_ERR_CUDA;
     GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status, nullptr, 0, 1, 0, 0, 0};
     dim3 grid(pair_grid((N / BN) * ((S + 255) / 256)), 1, 1);
-    { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
+    { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, tc, a); }
     return launch_status();
 }
 
@@ -268,9 +270,11 @@ int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN / 2)) return LAGA_ERR_CUDA;
+    CUtensorMap tc;
+    if (!cached_tmap_bf16(&tc, dc_kv, kDc, S, kDc * 2, 32)) return LAGA_ERR_CUDA;
     GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status, reinterpret_cast<float4*>(clear), clear_floats / 4, 1, 0, 0, 0};
     dim3 grid(pair_grid((kDc / BN) * ((S + 255) / 256)), 1, 1);
-    { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
+    { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, tc, a); }
     return launch_status();
 }
 
@@ -302,7 +306,7 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool d
     splits = (k_tiles + per_split - 1) / per_split;
     GemmArgs a{kDc, N, S, per_split, splits, dw, N, status, nullptr, 0, 1, 0, 0, 0};
     dim3 grid(pair_grid(tiles * splits), 1, 1);
-    { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
+    { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, ta, a); }   // (fp32 atomic epilogue: the output map is unused)
     return launch_status();
 }
 
@@ -416,9 +420,12 @@ int launch_q_absorb(const void* q, const void* w, int S, int h, void* q_abs, uns
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, q, q_row, S, q_row * 2, 128)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tb, w, w_row, kDc, w_row * 2, BN / 2)) return LAGA_ERR_CUDA;
+    CUtensorMap tc;
+    const uint64_t qa_row = static_cast<uint64_t>(h) * kDc;
+    if (!cached_tmap_bf16(&tc, q_abs, qa_row, S, qa_row * 2, 32)) return LAGA_ERR_CUDA;
     GemmArgs a{S, kDc, kDn, kDn / 64, 1, q_abs, h * kDc, status, nullptr, 0, h, kDn + kDr, kDn + kDv, kDc};
     dim3 grid(pair_grid((kDc / BN) * ((S + 255) / 256) * h), 1, 1);
-    { ScopedKernelEvents ev(LAGA_KERNEL_Q_ABSORB, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, a); }
+    { ScopedKernelEvents ev(LAGA_KERNEL_Q_ABSORB, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, tc, a); }
     return launch_status();
 }
 

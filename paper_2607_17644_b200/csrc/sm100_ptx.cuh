@@ -169,6 +169,22 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
         : "memory");
 }
 
+// TMA store of one box from shared memory (bulk async-group completion).  The shared-memory source must have
+// been written, fenced into the async proxy (fence_async_shared) and the writers synchronised before the issue.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Wait until at most `kPending` of this thread's store groups still READ their shared-memory source.
+template <int kPending>
+__device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // The same with the checked build's self-check: x on a 16-byte boundary (the hardware raises an illegal
 // instruction otherwise), y not negative, destination slab 1024-byte aligned.
 __device__ __forceinline__ void tma_load_2d_chk(unsigned int* status, void* smem_dst, const CUtensorMap* map, uint64_t* bar,
