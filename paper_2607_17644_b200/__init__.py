@@ -10,11 +10,13 @@ absence is an error: there is no CPU or eager fallback.
 """
 from .inputs import CONFIGS, CONFIG_SEEDS, LagaShape, make_inputs  # noqa: F401
 
-__all__ = ["CONFIGS", "CONFIG_SEEDS", "LagaShape", "make_inputs", "laga"]
+__all__ = ["CONFIGS", "CONFIG_SEEDS", "LagaShape", "make_inputs", "laga", "laga_attention"]
 
 
 def __getattr__(name):
+    import importlib
     if name == "laga":
-        import importlib
         return importlib.import_module(".laga", __name__)
+    if name == "laga_attention":          # the differentiable call (torch.autograd plumbing around laga.fwd / laga.bwd)
+        return importlib.import_module(".autograd", __name__).laga_attention
     raise AttributeError(name)

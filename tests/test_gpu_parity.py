@@ -416,3 +416,29 @@ def test_kernel_clock_probes(laga):
     clocks = laga.query_kernel_clocks(ws2)
     assert set(clocks) == {"attn_bwd_dkv", "attn_bwd_dq"}
     assert all(500.0 < v[0] < 2500.0 for v in clocks.values())
+
+
+def test_autograd_wrapper_gives_the_oracles_gradients(laga, oracle):
+    """laga_attention under torch.autograd: loss = <out, dO> backpropagated through the Function must return the
+    library's (and so the oracle's) gradients; the fp32 accumulation buffer variant adds on top."""
+    from paper_2607_17644_b200 import laga_attention
+    sh = LagaShape(S=777, h=3)
+    tensors = make_inputs(sh, 123)
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in tensors)
+    leaves = [t.clone().requires_grad_(True) for t in (q, c_kv, k_pe, w)]
+    out, lse = laga_attention(*leaves, return_lse=True)
+    (out.float() * dout.float()).sum().backward()
+    ref = oracle.bwd(*tensors, sh.d_v, sh.softmax_scale, kv_round_bf16=True, return_fwd=True)
+    check_tensor("out", out.detach(), ref["out"])
+    assert max_abs(lse, ref["lse"]) <= TOL_LSE
+    check_tensor("dq", leaves[0].grad, ref["dq"])
+    check_tensor("dc_kv", leaves[1].grad, ref["dc_kv"])
+    check_tensor("dk_pe", leaves[2].grad, ref["dk_pe"])
+    assert rel_l2(leaves[3].grad, ref["dw"]) <= 6e-3          # bf16 copy of the fp32 gradient (autograd wants W's dtype)
+    acc = torch.zeros(sh.d_c, sh.n_cols, dtype=torch.float32, device="cuda")
+    for _ in range(2):                                        # two micro-batches into one fp32 buffer
+        fresh = [t.clone().requires_grad_(True) for t in (q, c_kv, k_pe, w)]
+        o = laga_attention(*fresh, dw_fp32_out=acc)
+        (o.float() * dout.float()).sum().backward()
+        assert fresh[3].grad is None
+    check_dw(acc / 2, ref["dw"])
