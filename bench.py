@@ -386,6 +386,32 @@ def run_cuda(args):
     kv_saved_ms = max_over_ranks(s0.elapsed_time(s1), world) / K
     laga.check_status(ws_b, where="kv-saved step")
 
+    # ---- variant: LAGA_FLAG_FUSED_BWD, the one-pass CTA-pair backward (reported, not the headline) ---------
+    one_pass_ms = None
+    try:
+        ws_1 = laga.alloc_workspace(laga.bwd_workspace_bytes(sh.S, sh.h, flags=laga.FLAG_FUSED_BWD), dev)
+
+        def step_one_pass():
+            laga.fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_f)
+            laga.bwd(q, c_kv, k_pe, w, out, lse, dout, dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw_kv_b=dw, workspace=ws_1,
+                     flags=laga.FLAG_FUSED_BWD)
+
+        for _ in range(2):
+            step_one_pass()
+        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier(world)
+        o0.record()
+        for _ in range(K):
+            step_one_pass()
+        o1.record()
+        barrier(world)
+        one_pass_ms = max_over_ranks(o0.elapsed_time(o1), world) / K
+        laga.check_status(ws_1, where="one-pass backward step")
+        del ws_1
+        step()                                               # leave the default path's gradients in the output buffers
+    except Exception as exc:
+        one_pass_ms = f"unavailable: {type(exc).__name__}: {exc}"
+
     # ---- variant: the same step replayed from a CUDA graph (launch overhead off the critical path) -------
     graph_ms = None
     try:
@@ -550,6 +576,10 @@ def run_cuda(args):
         "variants": {"kv_saved": {"ms_per_step": kv_saved_ms, "value": world * total_flops / (kv_saved_ms * 1e-3) / 1e12,
                                   "note": "LAGA_FLAG_KV_SAVED: the backward reads the forward's K_nope/V from a shared "
                                           "workspace instead of recomputing step 4 (one launch less); not the headline"},
+                     "one_pass_bwd": {"ms_per_step": one_pass_ms,
+                                      "note": "LAGA_FLAG_FUSED_BWD: backward attention that computes every score tile once on CTA "
+                                              "pairs (1664 instead of 2304 executed FLOP per pair) with dQ summed by fp32 atomics; "
+                                              "slower as measured, kept as the opt-in alternative; not the headline"},
                      "cuda_graph": {"ms_per_step": graph_ms,
                                     "note": "the same forward+backward step captured once and replayed (11 launches per step: "
                                             "what short sequences are bound by); not the headline"}},

@@ -57,6 +57,7 @@ extern "C" {
 #define LAGA_FLAG_ACCUM_DW 1u             /* laga_bwd: add into dw_kv_b instead of overwriting it   */
 #define LAGA_FLAG_DETERMINISTIC 2u        /* laga_bwd: bitwise-repeatable dk_pe and dw_kv_b (see there) */
 #define LAGA_FLAG_KV_SAVED 4u             /* laga_bwd: the workspace still holds laga_fwd's K_nope/V (see there) */
+#define LAGA_FLAG_FUSED_BWD 8u            /* laga_bwd: one-pass backward attention on CTA pairs (see there)       */
 
 /* Library version (major*10000 + minor*100 + patch). */
 int laga_version(void);
@@ -105,6 +106,13 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
  * has written to the workspace since -- the forward leaves K_nope/V where the backward looks for them.
  * This is the explicit form's way of saving K/V for the backward; the price is that the workspace cannot
  * be shared with another layer between the two calls.  The library cannot check the promise.
+ * LAGA_FLAG_FUSED_BWD selects the one-pass backward attention: clusters of two CTAs compute each score
+ * tile once (one CTA scores, softmax and dV; its peer dK and dQ from the dS tile it receives through
+ * distributed shared memory) and dQ is summed over key tiles in an fp32 accumulator with atomic additions
+ * (S * w * 192 * 4 more workspace bytes for a window of w heads, at most 64 MB: pass the flag to
+ * laga_bwd_workspace_bytes), so dq is then not repeatable bit for bit.  It executes 5 instead of 7 tile
+ * products but is the SLOWER path on B200 as measured (its exponentials sit on one of the two SMs); it is
+ * not the default and cannot be combined with LAGA_FLAG_DETERMINISTIC (LAGA_ERR_INVALID_ARG).
  */
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
              const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
@@ -209,7 +217,9 @@ int laga_selftest_bounded_wait(void* status_word, unsigned budget_us, void* stre
 #define LAGA_KERNEL_Q_ABSORB 8      /* absorbed form: q_abs = W_uk q_nope (batched over heads)   */
 #define LAGA_KERNEL_ATTN_ABSORBED 9 /* absorbed form: latent-space attention                     */
 #define LAGA_KERNEL_V_PROJECT 10    /* absorbed form: out = W_uv o_lat (batched over heads)      */
-#define LAGA_KERNEL_COUNT 11
+#define LAGA_KERNEL_ATTN_BWD_FUSED 11 /* backward attention in one pass on CTA pairs: dK, dV, dQ sums */
+#define LAGA_KERNEL_DQ_CONVERT 12   /* dQ: scale and bf16 rounding of the fp32 sums              */
+#define LAGA_KERNEL_COUNT 13
 int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* stop_events, int n_pairs);
 
 /*

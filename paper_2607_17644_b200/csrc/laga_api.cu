@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "attn_absorbed_sm100.cuh"
+#include "attn_bwd_fused_sm100.cuh"
 #include "attn_bwd_sm100.cuh"
 #include "attn_fwd_sm100.cuh"
 #include "gemm_sm100.cuh"
@@ -68,8 +69,9 @@ bool make_tmap_bf16(CUtensorMap* map, const void* base, uint64_t inner_elems, ui
 // that) are cleared at the start of every entry point.
 constexpr size_t kStatusClearBytes = 256;
 constexpr size_t kCounterOffsetWords = 4;     // words 4, 5, 6: forward, dK/dV and dQ kernel work counters
-constexpr size_t kProbeOffsetBytes = 64;      // three ClockProbe records (forward, dK/dV, dQ)
-enum { kSlotFwd = 0, kSlotDkv = 1, kSlotDq = 2 };
+constexpr size_t kProbeOffsetBytes = 64;      // four ClockProbe records (forward, dK/dV, dQ, fused backward)
+enum { kSlotFwd = 0, kSlotDkv = 1, kSlotDq = 2, kSlotFused = 3 };
+static_assert(kProbeOffsetBytes + 4 * sizeof(ClockProbe) <= kStatusClearBytes, "the probes must lie inside the cleared part of the slot");
 
 unsigned* slot_counter(unsigned* status, int slot) { return status + kCounterOffsetWords + slot; }
 ClockProbe* slot_probe(unsigned* status, int slot) {
@@ -85,6 +87,7 @@ struct DeviceInfo {
     std::once_flag once;
     int rc = LAGA_ERR_CUDA;
     int sms = 148;
+    int fused_pairs = 74;               // CTA pairs of the fused backward that are resident at the same time
     std::once_flag scratch_once;
     unsigned char* builtin_scratch = nullptr;
 };
@@ -113,7 +116,29 @@ void init_device(DeviceInfo* info, int dev) {
               allow_smem(attn_bwd_dkv_sm100_kernel<true>, AttnBwdDkvSmem::kTotalBytes) &&
               allow_smem(attn_bwd_dkv_sm100_kernel<false>, AttnBwdDkvSmem::kTotalBytes) &&
               allow_smem(attn_bwd_dq_sm100_kernel<true>, AttnBwdDqSmem::kTotalBytes) &&
-              allow_smem(attn_bwd_dq_sm100_kernel<false>, AttnBwdDqSmem::kTotalBytes);
+              allow_smem(attn_bwd_dq_sm100_kernel<false>, AttnBwdDqSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_fused_sm100_kernel<true>, AttnBwdFusedSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_fused_sm100_kernel<false>, AttnBwdFusedSmem::kTotalBytes);
+    if (ok) {
+        // The fused backward assigns work to pairs statically, so its grid must not exceed the pairs the
+        // device keeps resident at once (SMs that cannot form a pair inside their GPC stay idle).
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(info->sms / 2 * 2), 1, 1);
+        cfg.blockDim = dim3(kBwdThreads, 1, 1);
+        cfg.dynamicSmemBytes = AttnBwdFusedSmem::kTotalBytes;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, attn_bwd_fused_sm100_kernel<true>, &cfg) == cudaSuccess && clusters > 0)
+            info->fused_pairs = clusters < info->sms / 2 ? clusters : info->sms / 2;
+        else {
+            (void)cudaGetLastError();
+            info->fused_pairs = info->sms / 2;
+        }
+    }
     info->rc = ok ? LAGA_OK : LAGA_ERR_CUDA;
     if (!ok) (void)cudaGetLastError();
 }
@@ -136,6 +161,11 @@ int check_device() {
 int sm_count() {
     DeviceInfo* info = nullptr;
     return current_device(&info) == LAGA_OK ? info->sms : 148;
+}
+
+int fused_pair_count() {
+    DeviceInfo* info = nullptr;
+    return current_device(&info) == LAGA_OK ? info->fused_pairs : 74;
 }
 
 // Every data pointer must be device memory of the CURRENT device (or managed memory): a kernel given
@@ -331,11 +361,28 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
 
 // ---- Section 5.2: backward of step 5 ------------------------------------------------------------
 struct BwdWorkspace {
-    size_t kv, dkv, stat_l2, stat_delta, dkpe_acc, dk_rope_per_head, total;
+    size_t kv, dkv, stat_l2, stat_delta, dkpe_acc, dk_rope_per_head, dq_acc, total;
     int S_pad;
+    int head_window;      // heads per launch of the fused backward; 0 = the two-kernel backward
 };
 
-BwdWorkspace bwd_workspace_layout(int S, int h, bool deterministic) {
+// The fused backward adds dQ tiles into an fp32 accumulator [S][window][192]; the window is the largest
+// even split of the heads whose accumulator stays within this budget (so that it, and the Q / dO tiles of
+// those heads, stay L2 resident while every key tile sweeps them).
+#ifndef LAGA_DQ_ACC_BUDGET_MB
+#define LAGA_DQ_ACC_BUDGET_MB 64
+#endif
+constexpr long long kDqAccBudgetBytes = static_cast<long long>(LAGA_DQ_ACC_BUDGET_MB) << 20;
+int fused_head_window(int S, int h) {
+    const long long per_head = static_cast<long long>(S) * (kDn + kDr) * sizeof(float);
+    long long fit = kDqAccBudgetBytes / per_head;
+    if (fit < 1) fit = 1;
+    if (fit > h) fit = h;
+    const int launches = static_cast<int>((h + fit - 1) / fit);
+    return (h + launches - 1) / launches;
+}
+
+BwdWorkspace bwd_workspace_layout(int S, int h, bool deterministic, bool fused) {
     BwdWorkspace w;
     const size_t kv_bytes = align_up(static_cast<size_t>(S) * h * (kDn + kDv) * 2, 1024);
     w.S_pad = (S + 127) / 128 * 128;
@@ -346,16 +393,17 @@ BwdWorkspace bwd_workspace_layout(int S, int h, bool deterministic) {
     w.stat_delta = w.stat_l2 + stat_bytes;
     w.dkpe_acc = w.stat_delta + stat_bytes;
     w.dk_rope_per_head = w.dkpe_acc + align_up(static_cast<size_t>(S) * kDr * sizeof(float), 1024);
-    w.total = w.dk_rope_per_head +
-              (deterministic ? align_up(static_cast<size_t>(h) * S * kDr * sizeof(float), 1024) : 0);
+    w.dq_acc = w.dk_rope_per_head +
+               (deterministic ? align_up(static_cast<size_t>(h) * S * kDr * sizeof(float), 1024) : 0);
+    w.head_window = fused ? fused_head_window(S, h) : 0;
+    w.total = w.dq_acc + align_up(static_cast<size_t>(S) * w.head_window * (kDn + kDr) * sizeof(float), 1024);
     return w;
 }
 
 int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void* out, const float* lse,
                     const void* dout, int S, int h, float softmax_scale, int causal, void* dq, void* dkv,
                     void* dk_pe, float* stat_l2, float* stat_delta, float* dkpe_acc, float* dk_rope_per_head, int S_pad,
-                    unsigned* status,
-                    cudaStream_t stream) {
+                    float* dq_acc, int head_window, unsigned* status, cudaStream_t stream) {
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
     {   // delta and the transposed, padded softmax statistics; clears the rope-gradient accumulator on the way
@@ -375,23 +423,51 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         !cached_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, 128))
         return LAGA_ERR_CUDA;
     const int n_tiles = (S + 127) / 128;
-    dim3 grid(persistent_grid(n_tiles * h), 1, 1);
-    AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
-                     reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, dk_rope_per_head, status,
-                     make_schedule(n_tiles, S, h, slot_counter(status, kSlotDkv)), slot_probe(status, kSlotDkv)};
-    AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad,
-                    reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status,
-                    make_schedule(n_tiles, S, h, slot_counter(status, kSlotDq)), slot_probe(status, kSlotDq)};
-    {
-        ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream);
-        if (causal) attn_bwd_dkv_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
-        else attn_bwd_dkv_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
-    }
-    if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
-    {
-        ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream);
-        if (causal) attn_bwd_dq_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
-        else attn_bwd_dq_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
+    if (head_window > 0) {
+        // One pass over the score tiles on CTA pairs, a window of heads per launch; dQ goes through dq_acc.
+        if (cudaMemsetAsync(dq_acc, 0, static_cast<size_t>(S) * head_window * (kDn + kDr) * sizeof(float), stream) != cudaSuccess)
+            return LAGA_ERR_CUDA;
+        const int pairs_max = fused_pair_count();
+        for (int head_begin = 0; head_begin < h; head_begin += head_window) {
+            const int head_count = h - head_begin < head_window ? h - head_begin : head_window;
+            const int items = n_tiles * head_count;
+            dim3 grid(2u * static_cast<unsigned>(items < pairs_max ? items : pairs_max), 1, 1);
+            AttnBwdFusedArgs f{S, h, S_pad, head_begin, head_count, scale_log2, softmax_scale, stat_l2, stat_delta,
+                               reinterpret_cast<const __nv_bfloat16*>(kv), reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc,
+                               dq_acc, status, slot_probe(status, kSlotFused)};
+            {
+                ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_FUSED, stream);
+                if (causal) attn_bwd_fused_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdFusedSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, f);
+                else attn_bwd_fused_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdFusedSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, f);
+            }
+            if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+            {
+                const size_t n = static_cast<size_t>(S) * head_count * (kDn + kDr) / 8;
+                ScopedKernelEvents ev(LAGA_KERNEL_DQ_CONVERT, stream);
+                bwd_dq_convert_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
+                    dq_acc, S, h, head_begin, head_count, softmax_scale, reinterpret_cast<__nv_bfloat16*>(dq));
+            }
+            if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+        }
+    } else {
+        dim3 grid(persistent_grid(n_tiles * h), 1, 1);
+        AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
+                         reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, dk_rope_per_head, status,
+                         make_schedule(n_tiles, S, h, slot_counter(status, kSlotDkv)), slot_probe(status, kSlotDkv)};
+        AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad,
+                        reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status,
+                        make_schedule(n_tiles, S, h, slot_counter(status, kSlotDq)), slot_probe(status, kSlotDq)};
+        {
+            ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream);
+            if (causal) attn_bwd_dkv_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
+            else attn_bwd_dkv_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
+        }
+        if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
+        {
+            ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream);
+            if (causal) attn_bwd_dq_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
+            else attn_bwd_dq_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
+        }
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     {
@@ -514,7 +590,7 @@ size_t laga_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, i
 
 size_t laga_bwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v, unsigned flags) {
     if (S < 1 || h < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
-    return bwd_workspace_layout(S, h, (flags & LAGA_FLAG_DETERMINISTIC) != 0).total;
+    return bwd_workspace_layout(S, h, (flags & LAGA_FLAG_DETERMINISTIC) != 0, (flags & LAGA_FLAG_FUSED_BWD) != 0).total;
 }
 
 int laga_up_project(const void* c_kv, const void* w_kv_b, int S, int h, int d_c, int d_nope, int d_v, void* kv,
@@ -586,12 +662,14 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
         !aligned16(lse) || !aligned16(dout) || !aligned16(dq) || !aligned16(dc_kv) || !aligned16(dk_pe) ||
         !aligned16(dw_kv_b) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return LAGA_ERR_INVALID_ARG;
-    if ((flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC | LAGA_FLAG_KV_SAVED)) || !(softmax_scale > 0.f))
+    if ((flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC | LAGA_FLAG_KV_SAVED | LAGA_FLAG_FUSED_BWD)) || !(softmax_scale > 0.f))
         return LAGA_ERR_INVALID_ARG;
     if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
     const bool deterministic = (flags & LAGA_FLAG_DETERMINISTIC) != 0;
     const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
-    const BwdWorkspace w = bwd_workspace_layout(S, h, deterministic);
+    const bool fused = (flags & LAGA_FLAG_FUSED_BWD) != 0;
+    if (fused && deterministic) return LAGA_ERR_INVALID_ARG;   // the fused kernel's dQ and dk_pe sums are order dependent
+    const BwdWorkspace w = bwd_workspace_layout(S, h, deterministic, fused);
     if (workspace_bytes < w.total) return LAGA_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
@@ -610,8 +688,8 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
     if ((rc = launch_attn_bwd(q, kv, k_pe, out, lse, dout, S, h, softmax_scale, causal, dq, dkv, dk_pe,
                               reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
                               reinterpret_cast<float*>(base + w.dkpe_acc),
-                              deterministic ? reinterpret_cast<float*>(base + w.dk_rope_per_head) : nullptr, w.S_pad, status,
-                              st)) != LAGA_OK)
+                              deterministic ? reinterpret_cast<float*>(base + w.dk_rope_per_head) : nullptr, w.S_pad,
+                              reinterpret_cast<float*>(base + w.dq_acc), w.head_window, status, st)) != LAGA_OK)
         return rc;
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,
                           accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st)) != LAGA_OK)
@@ -738,15 +816,15 @@ int laga_profile_kernel(int kernel_id, void* const* start_events, void* const* s
 
 int laga_query_kernel_clocks(const void* workspace, void* stream, double* sm_mhz, double* kernel_ms) {
     if (!workspace || !sm_mhz || !kernel_ms) return LAGA_ERR_INVALID_ARG;
-    ClockProbe probes[3];
+    ClockProbe probes[4];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(probes, static_cast<const uint8_t*>(workspace) + kProbeOffsetBytes, sizeof(probes),
                         cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return LAGA_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return LAGA_ERR_CUDA;
     for (int k = 0; k < LAGA_KERNEL_COUNT; ++k) sm_mhz[k] = kernel_ms[k] = 0.0;
-    const int ids[3] = {LAGA_KERNEL_ATTN_FWD, LAGA_KERNEL_ATTN_BWD_DKV, LAGA_KERNEL_ATTN_BWD_DQ};
-    for (int i = 0; i < 3; ++i) {
+    const int ids[4] = {LAGA_KERNEL_ATTN_FWD, LAGA_KERNEL_ATTN_BWD_DKV, LAGA_KERNEL_ATTN_BWD_DQ, LAGA_KERNEL_ATTN_BWD_FUSED};
+    for (int i = 0; i < 4; ++i) {
         const ClockProbe& p = probes[i];
         if (p.ns_end <= p.ns_begin || p.cycles_end <= p.cycles_begin) continue;   // that kernel has not run on this workspace
         const double ns = static_cast<double>(p.ns_end - p.ns_begin);

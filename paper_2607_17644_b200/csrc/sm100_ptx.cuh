@@ -361,6 +361,57 @@ __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorM
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y)
         : "memory");
 }
+// ---- distributed shared memory between the two CTAs of a cluster (used by the fused backward) ----------
+// 16-byte store into the peer's shared memory (generic proxy), at a cluster address from cluster_map().
+__device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint4 v) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+// Orders this thread's generic-proxy writes (local or peer shared memory) before later async-proxy reads
+// (tcgen05.mma operand fetches) of the same data: issue after the stores, before signalling the consumer.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// try_wait that acquires at cluster scope: the waiter goes on to read data the PEER CTA wrote.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, AbortFlag* abort_flag, unsigned int* status,
+                                                  uint32_t site, unsigned long long budget_ns = kWaitBudgetNs) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    uint32_t polls = 0;
+    while (true) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((++polls & 0xffu) == 0u) {
+            if (abort_flag->value != 0u) return false;
+            if (global_timer_ns() - t0 > budget_ns) {
+                abort_flag->value = 1u;
+                if (status) atomicCAS(status, kStatusOk, kStatusTimeout | site);
+                return false;
+            }
+        }
+    }
+}
+// tcgen05.commit (one-CTA MMAs) that arrives on the barrier at this offset in every CTA of `cta_mask`: how the
+// MMA lane of one CTA tells its PEER that the MMAs which read a buffer have completed.  Signals only; no data.
+__device__ __forceinline__ void mma_commit_to(uint64_t* bar, uint16_t cta_mask) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(cta_mask)
+                 : "memory");
+}
+// fp32 reduction into global memory without a return value (one lane, one element; a warp whose lanes hit 32
+// consecutive floats makes one 128-byte transaction).
+__device__ __forceinline__ void red_add_f32(float* addr, float v) {
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
+}
+
 __device__ __forceinline__ void tma_load_2d_pair_chk(unsigned int* status, void* smem_dst, const CUtensorMap* map,
                                                      uint32_t bar_cluster_addr, int x, int y) {
     if (device_check((x & 7) == 0 && x >= 0 && y >= 0 && (smem_u32(smem_dst) & 1023u) == 0u, status, 0xE00000u | (x & 0xffff)))

@@ -21,6 +21,7 @@ ERR_DEVICE_CHECK = -6
 FLAG_ACCUM_DW = 1
 FLAG_DETERMINISTIC = 2
 FLAG_KV_SAVED = 4
+FLAG_FUSED_BWD = 8
 
 # LAGA_DEBUG=1 selects the checked build of the same kernels (liblaga_debug.so): every TMA issue and global
 # store verifies its index arithmetic first and reports LAGA_ERR_DEVICE_CHECK instead of a bad access.
@@ -49,7 +50,8 @@ SIGNATURES = {
 }
 BUILTIN_SCRATCH_MAX_TOKEN_HEADS = 32768   # S * h limit of laga_fwd_builtin_scratch (16 MiB of bf16 KV)
 KERNELS = {"up_project": 0, "attn_fwd": 1, "bwd_delta": 2, "attn_bwd_dkv": 3, "attn_bwd_dq": 4,
-           "dkpe_reduce": 5, "dckv_gemm": 6, "dw_gemm": 7, "q_absorb": 8, "attn_absorbed": 9, "v_project": 10}
+           "dkpe_reduce": 5, "dckv_gemm": 6, "dw_gemm": 7, "q_absorb": 8, "attn_absorbed": 9, "v_project": 10,
+           "attn_bwd_fused": 11, "dq_convert": 12}
 
 
 class LagaError(RuntimeError):

@@ -55,7 +55,8 @@ def run_case(S, h, causal):
     tensors = make_inputs(sh, 900 + S + h)
     q, c_kv, k_pe, w, dout = (t.cuda() for t in tensors)
     bf, f32 = torch.bfloat16, torch.float32
-    ws_sizes = [laga.fwd_workspace_bytes(S, h), laga.bwd_workspace_bytes(S, h), laga.absorbed_fwd_workspace_bytes(S, h)]
+    ws_sizes = [laga.fwd_workspace_bytes(S, h), laga.bwd_workspace_bytes(S, h), laga.absorbed_fwd_workspace_bytes(S, h),
+                laga.bwd_workspace_bytes(S, h, flags=laga.FLAG_FUSED_BWD)]
     arena = Arena(sum(ws_sizes) + 16 * S * h * 192 * 4 + 64 * GUARD + 512 * h * 256 * 4 + (1 << 20))
     out = arena.take(S * h * 128 * 2, bf, (S, h, 128))
     lse = arena.take(S * h * 4, f32, (S, h))
@@ -65,17 +66,25 @@ def run_case(S, h, causal):
     dw = arena.take(512 * h * 256 * 4, f32, (512, h * 256))
     out_a = arena.take(S * h * 128 * 2, bf, (S, h, 128))
     lse_a = arena.take(S * h * 4, f32, (S, h))
-    ws_f, ws_b, ws_a = (arena.take(n) for n in ws_sizes)
+    dq_1 = arena.take(S * h * 192 * 2, bf, (S, h, 192))
+    dc_kv_1 = arena.take(S * 512 * 2, bf, (S, 512))
+    dk_pe_1 = arena.take(S * 64 * 2, bf, (S, 64))
+    dw_1 = arena.take(512 * h * 256 * 4, f32, (512, h * 256))
+    ws_f, ws_b, ws_a, ws_1 = (arena.take(n) for n in ws_sizes)
     laga.fwd(q, c_kv, k_pe, w, causal=causal, out=out, lse=lse, workspace=ws_f)
     laga.check_status(ws_f, where="laga_fwd")
     laga.bwd(q, c_kv, k_pe, w, out, lse, dout, causal=causal, dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw_kv_b=dw, workspace=ws_b)
     laga.check_status(ws_b, where="laga_bwd")
+    laga.bwd(q, c_kv, k_pe, w, out, lse, dout, causal=causal, dq=dq_1, dc_kv=dc_kv_1, dk_pe=dk_pe_1, dw_kv_b=dw_1,
+             workspace=ws_1, flags=laga.FLAG_FUSED_BWD)
+    laga.check_status(ws_1, where="laga_bwd (one-pass backward)")
     laga.absorbed_fwd(q, c_kv, k_pe, w, causal=causal, out=out_a, lse=lse_a, workspace=ws_a)
     laga.check_status(ws_a, where="laga_absorbed_fwd")
     torch.cuda.synchronize()
     assert arena.guards_intact(), f"a guard band was overwritten (S={S}, h={h})"
     ref = oracle.bwd(*tensors, sh.d_v, sh.softmax_scale, causal=causal, kv_round_bf16=True, return_fwd=True)
-    for name, got in (("out", out), ("dq", dq), ("dc_kv", dc_kv), ("dk_pe", dk_pe), ("dw", dw), ("out", out_a)):
+    for name, got in (("out", out), ("dq", dq), ("dc_kv", dc_kv), ("dk_pe", dk_pe), ("dw", dw), ("out", out_a),
+                      ("dq", dq_1), ("dc_kv", dc_kv_1), ("dk_pe", dk_pe_1), ("dw", dw_1)):
         err = rel_l2(got, ref[name])
         assert err <= 5e-3, (name, err)
     assert float((lse.double().cpu() - ref["lse"]).abs().max()) <= 1e-3

@@ -66,6 +66,10 @@ def test_workspace_sizes(laga):
     assert bwd >= 1024 + 2 * kv_bytes              # recomputed KV and dKV, both bf16
     assert bwd <= 1024 + 2 * kv_bytes + S * h * 2 * 4 + S * 64 * 4 + 8192
     assert laga.bwd_workspace_bytes(S, h, flags=laga.FLAG_DETERMINISTIC) >= bwd + S * h * 64 * 4
+    # the one-pass backward adds an fp32 dQ accumulator for a window of heads, at most 64 MB of it
+    fused = laga.bwd_workspace_bytes(S, h, flags=laga.FLAG_FUSED_BWD)
+    assert bwd + S * 192 * 4 <= fused <= bwd + (64 << 20) + 1024
+    assert laga.bwd_workspace_bytes(512, 2, flags=laga.FLAG_FUSED_BWD) == laga.bwd_workspace_bytes(512, 2) + 512 * 2 * 192 * 4
     assert laga.fwd_workspace_bytes(300, 3) % 1024 == 0 and laga.bwd_workspace_bytes(300, 3) % 1024 == 0
     # unsupported geometry or empty problem: 0
     assert laga.fwd_workspace_bytes(128, 2, d_c=256) == 0
@@ -103,7 +107,8 @@ def test_argument_validation_happens_before_any_device_work(laga):
                             a["d_rope"], a["d_v"], 0.07, 1, dq, good, good, good, good, ws_bytes, flags, None)
 
     assert bwd(dq=None) == laga.ERR_INVALID_ARG
-    assert bwd(flags=8) == laga.ERR_INVALID_ARG     # 1, 2 and 4 are defined
+    assert bwd(flags=16) == laga.ERR_INVALID_ARG    # 1, 2, 4 and 8 are defined
+    assert bwd(flags=laga.FLAG_FUSED_BWD | laga.FLAG_DETERMINISTIC) == laga.ERR_INVALID_ARG
     assert bwd(d_v=64) == laga.ERR_UNSUPPORTED
     assert bwd(ws_bytes=4096) == laga.ERR_WORKSPACE_TOO_SMALL
     assert lib.laga_up_project(None, good, 128, 2, 512, 128, 128, good, good, None) == laga.ERR_INVALID_ARG

@@ -27,7 +27,7 @@ def nan_like(shape, dtype):
     return torch.full(shape, float("nan"), dtype=dtype, device="cuda")
 
 
-def run_gpu(laga, tensors, causal, backward=True):
+def run_gpu(laga, tensors, causal, backward=True, bwd_flags=0):
     """Every output starts as NaN: a tile the kernels fail to write cannot pass on stale memory."""
     q, c_kv, k_pe, w, dout = (t.cuda() if t is not None else None for t in tensors)
     S, h = q.shape[0], q.shape[1]
@@ -40,7 +40,7 @@ def run_gpu(laga, tensors, causal, backward=True):
                                              dq=nan_like(tuple(q.shape), torch.bfloat16),
                                              dc_kv=nan_like(tuple(c_kv.shape), torch.bfloat16),
                                              dk_pe=nan_like(tuple(k_pe.shape), torch.bfloat16),
-                                             dw_kv_b=nan_like(tuple(w.shape), torch.float32))
+                                             dw_kv_b=nan_like(tuple(w.shape), torch.float32), flags=bwd_flags)
         laga.check_status(ws2, where="laga_bwd")
         res.update(dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw=dw)
     return {k: v.cpu() for k, v in res.items()}
@@ -89,6 +89,57 @@ def test_forward_backward_elementwise(laga, oracle, S, h, causal):
         if S >= 64:
             check_row_bands("out", g["out"], r["out"])
             check_row_bands("dq", g["dq"], r["dq"])
+
+
+FUSED_CASES = [(512, 2, True), (300, 3, True), (300, 3, False), (1, 1, True), (129, 2, True), (1024, 4, True),
+               (700, 1, True), (2048, 5, True)]
+
+
+@pytest.mark.parametrize("S,h,causal", FUSED_CASES)
+def test_one_pass_backward_elementwise(laga, oracle, S, h, causal):
+    """LAGA_FLAG_FUSED_BWD: the CTA-pair backward that computes every score tile once, against the oracle
+    with the same tolerances as the default path (its dQ is summed over key tiles in fp32 before the one
+    rounding to bf16, the same arithmetic as the TMEM accumulation of the default path up to order)."""
+    sh = LagaShape(S=S, h=h)
+    tensors = make_inputs(sh, 7000 + S + h)
+    g = run_gpu(laga, tensors, causal, bwd_flags=laga.FLAG_FUSED_BWD)
+    q, c_kv, k_pe, w, dout = tensors
+    r = oracle.bwd(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, causal=causal, kv_round_bf16=True, return_fwd=True)
+    if S > 1:
+        check_tensor("dq", g["dq"], r["dq"])
+        check_tensor("dk_pe", g["dk_pe"], r["dk_pe"])
+    else:
+        assert max_abs(g["dq"], r["dq"]) <= 1e-5 and max_abs(g["dk_pe"], r["dk_pe"]) <= 1e-5
+    check_tensor("dc_kv", g["dc_kv"], r["dc_kv"])
+    check_dw(g["dw"], r["dw"])
+    if S >= 64:
+        check_row_bands("dq", g["dq"], r["dq"])
+
+
+def test_one_pass_backward_at_the_headline_size_agrees_with_the_default_path(laga):
+    """At S = 16384, h = 16 the one-pass backward runs four launches over windows of four heads (its fp32 dQ
+    accumulator is capped at 64 MB).  The default path is compared with the oracle at this size elsewhere; here
+    the two GPU paths are compared with each other on every element: dK / dV, hence dc_kv and dW, come from the
+    same products in the same order (equal up to the atomics' order in dW), dQ differs by fp32 summation order."""
+    sh = CONFIGS["c2"]
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in make_inputs(sh, CONFIG_SEEDS["c2"]))
+    out, lse, ws = laga.fwd(q, c_kv, k_pe, w)
+    laga.check_status(ws)
+    assert laga.bwd_workspace_bytes(sh.S, sh.h, flags=laga.FLAG_FUSED_BWD) - laga.bwd_workspace_bytes(sh.S, sh.h) == sh.S * 4 * 192 * 4
+    res = {}
+    for name, flags in (("default", 0), ("one_pass", laga.FLAG_FUSED_BWD)):
+        dq, dc, dk, dw, ws2 = laga.bwd(q, c_kv, k_pe, w, out, lse, dout, dq=nan_like(tuple(q.shape), torch.bfloat16),
+                                       dc_kv=nan_like(tuple(c_kv.shape), torch.bfloat16), flags=flags)
+        laga.check_status(ws2, where=name)
+        res[name] = (dq, dc, dk, dw)
+        del ws2
+    a, b = res["one_pass"], res["default"]
+    assert not torch.isnan(a[0].float()).any() and not torch.isnan(a[1].float()).any()
+    assert float((a[0].float() - b[0].float()).norm() / b[0].float().norm()) < 1e-3          # dq
+    assert float((a[0].float() - b[0].float()).abs().max()) <= 2e-2 * max(1.0, float(b[0].float().pow(2).mean().sqrt()))
+    assert torch.equal(a[1], b[1])                                                            # dc_kv
+    assert float((a[2].float() - b[2].float()).norm() / b[2].float().norm()) < 1e-3          # dk_pe (atomics)
+    assert float((a[3] - b[3]).norm() / b[3].norm()) < 1e-5                                   # dw (atomics)
 
 
 def test_row_zero_and_head_shard_invariance(laga):
@@ -329,7 +380,7 @@ def test_kv_saved_flag_reuses_the_forwards_up_projection(laga):
     for a, b in zip(saved, recomputed):
         assert torch.equal(a, b)
     with pytest.raises(laga.LagaError):
-        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, flags=8)               # unknown flag bit
+        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, flags=16)              # unknown flag bit
 
 
 def test_long_ragged_sequence_sampled(laga, oracle):
