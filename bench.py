@@ -285,11 +285,99 @@ def run_c4(args):
     print(json.dumps(line), flush=True)
 
 
+PACKED_MIXES = {
+    # 16384 tokens of a 16-head shard each, packed in different ways (lengths in tokens)
+    "1x16384": [16384],
+    "4x4096": [4096] * 4,
+    "ragged_8": [8192, 4096, 2048, 1024, 512, 256, 128, 128],
+    "64x256": [256] * 64,
+}
+
+
+def run_packed(args):
+    """Batches and variable-length sequences (laga_fwd_varlen / laga_bwd_varlen): the same 16384 tokens of a
+    16-head shard packed as one sequence, as a batch of four, as a ragged mix and as 64 short sequences.  Each
+    mix is timed through one packed call per direction and, for comparison, as a loop of single-sequence calls
+    over the same rows.  FLOPs are algorithmic: causal pairs inside each sequence plus the token-wise GEMMs."""
+    from paper_2607_17644_b200 import laga
+    laga.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    sh = CONFIGS["c2"]
+    q, c_kv, k_pe, w, dout = (t.to(dev) for t in make_inputs(sh, CONFIG_SEEDS["c2"]))
+    out = torch.empty(sh.S, sh.h, sh.d_v, dtype=torch.bfloat16, device=dev)
+    lse = torch.empty(sh.S, sh.h, dtype=torch.float32, device=dev)
+    dq, dc_kv, dk_pe = torch.empty_like(q), torch.empty_like(c_kv), torch.empty_like(k_pe)
+    dw = torch.empty(sh.d_c, sh.n_cols, dtype=torch.float32, device=dev)
+    K, W = args.steps, max(args.warmup, 3)
+
+    def timed(fn):
+        for _ in range(W):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(K):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / K
+
+    results = {}
+    for name, lengths in PACKED_MIXES.items():
+        cu = [0]
+        for n in lengths:
+            cu.append(cu[-1] + n)
+        pairs = sum(n * (n + 1) // 2 for n in lengths)
+        total = 2 * sh.h * pairs * (sh.d_qk + sh.d_v) + 2 * sh.h * pairs * (3 * sh.d_qk + 2 * sh.d_v) \
+            + 3 * 2 * sh.S * sh.d_c * sh.n_cols
+        ws_f = laga.alloc_workspace(laga.fwd_varlen_workspace_bytes(sh.S, len(lengths), sh.h), dev)
+        ws_b = laga.alloc_workspace(laga.bwd_varlen_workspace_bytes(sh.S, len(lengths), sh.h), dev)
+
+        def packed_step():
+            laga.fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_f, cu_seqlens=cu)
+            laga.bwd(q, c_kv, k_pe, w, out, lse, dout, dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw_kv_b=dw, workspace=ws_b,
+                     cu_seqlens=cu)
+
+        packed_ms = timed(packed_step)
+        laga.check_status(ws_f, where=f"{name} laga_fwd_varlen")
+        laga.check_status(ws_b, where=f"{name} laga_bwd_varlen")
+        n_max = max(lengths)
+        ws_f1 = laga.alloc_workspace(laga.fwd_workspace_bytes(n_max, sh.h), dev)
+        ws_b1 = laga.alloc_workspace(laga.bwd_workspace_bytes(n_max, sh.h), dev)
+        dw1 = torch.empty_like(dw)
+
+        def loop_step():
+            for i, (a, b) in enumerate(zip(cu[:-1], cu[1:])):
+                laga.fwd(q[a:b], c_kv[a:b], k_pe[a:b], w, out=out[a:b], lse=lse[a:b], workspace=ws_f1)
+                laga.bwd(q[a:b], c_kv[a:b], k_pe[a:b], w, out[a:b], lse[a:b], dout[a:b], dq=dq[a:b], dc_kv=dc_kv[a:b],
+                         dk_pe=dk_pe[a:b], dw_kv_b=dw1, workspace=ws_b1, flags=laga.FLAG_ACCUM_DW if i else 0)
+
+        loop_ms = timed(loop_step)
+        laga.check_status(ws_b1, where=f"{name} loop of laga_bwd")
+        results[name] = {"sequences": len(lengths), "longest": n_max, "algorithmic_flops": total,
+                         "packed_ms": packed_ms, "packed_tflops": total / (packed_ms * 1e-3) / 1e12,
+                         "one_call_per_sequence_ms": loop_ms, "one_call_per_sequence_tflops": total / (loop_ms * 1e-3) / 1e12,
+                         "launches_packed": 11, "launches_looped": 11 * len(lengths)}
+        del ws_f, ws_b, ws_f1, ws_b1
+    head = results["4x4096"]
+    line = {"metric": "packed_batch_fwd_bwd_tflops", "value": head["packed_tflops"], "unit": UNIT, "n_gpus": 1, "steps": K,
+            "warmup": W, "ms_per_step": head["packed_ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "packed: 16384 tokens of a 16-head DeepSeek-V3 shard as a batch of 4 x 4096 (headline of "
+                                   "this line) and three other packings; causal within each sequence",
+                       "l2_policy": "inputs and workspaces larger than L2"},
+            "mixes": results, "gpu_launches": 11 * K}
+    print(json.dumps(line), flush=True)
+
+
 def run_cuda(args):
     from paper_2607_17644_b200 import laga
     laga.lib()
     if args.workload == "c4":
         return run_c4(args)
+    if args.workload == "packed":
+        return run_packed(args)
     world, rank, local_rank = dist_setup(args.gpus)
     dev = torch.device("cuda", torch.cuda.current_device())
     sh = CONFIGS[args.workload]
@@ -715,9 +803,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing and parity leg")
-    ap.add_argument("--workload", choices=sorted(CONFIGS), default=WORKLOAD,
+    ap.add_argument("--workload", choices=sorted(CONFIGS) + ["packed"], default=WORKLOAD,
                     help="benchmark configuration (default c2, the headline; c4 = the absorbed form beside the LAGA "
-                         "forward on c2's inputs; others are for profiling)")
+                         "forward on c2's inputs; packed = batches / variable-length sequences through the varlen "
+                         "entry points; others are for profiling)")
     ap.add_argument("--compare-eager", action="store_true",
                     help="also time the explicit and absorbed forms in eager PyTorch (N=1; tens of GB at c2)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=16384,

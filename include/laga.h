@@ -120,6 +120,39 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
              void* workspace, size_t workspace_bytes, unsigned flags, void* stream);
 
 /*
+ * Batches and variable-length sequences (Algorithm 1 steps 4-5 and Section 5.2 applied per sequence).
+ *
+ * n_seqs sequences are PACKED along the token axis: q [S_total, h, 192], c_kv [S_total, d_c], k_pe [S_total, d_rope]
+ * and every output in the same row order, sequence k occupying rows cu_seqlens[k] .. cu_seqlens[k+1]-1.
+ * cu_seqlens is a HOST array of n_seqs + 1 non-decreasing integers with cu_seqlens[0] = 0 and
+ * cu_seqlens[n_seqs] = S_total (a batch of B equal sequences of length L is {0, L, 2L, ...}; empty sequences are
+ * allowed).  Attention (and its causal mask) is confined to each sequence; the projections of step 4 and of
+ * Section 5.2 are token-wise and run once over all the packed tokens; dw_kv_b sums over all sequences, dk_pe
+ * over the shard's heads as in laga_bwd.  Everything else -- layouts, dtypes, flags, errors, ownership -- is as
+ * for laga_fwd / laga_bwd, with these differences:
+ *   - the workspace is sized by the _varlen_ queries below (they need n_seqs, not the lengths); LAGA_FLAG_KV_SAVED
+ *     pairs laga_fwd_varlen with laga_bwd_varlen on the same workspace, cu_seqlens included;
+ *   - the call copies a small table (32 bytes per 128-token tile) from host memory into the workspace, which
+ *     makes it synchronise with the stream's earlier work and unsuitable for CUDA-graph capture;
+ *   - LAGA_FLAG_FUSED_BWD is not available (LAGA_ERR_INVALID_ARG; its workspace query returns 0).
+ * A malformed cu_seqlens (not starting at 0, decreasing, not ending at S_total, or no token at all) is
+ * LAGA_ERR_INVALID_ARG before anything is enqueued.  All sequences' tiles are handed to the persistent kernels
+ * in one launch each, longest first.
+ */
+size_t laga_fwd_varlen_workspace_bytes(int S_total, int n_seqs, int h, int d_c, int d_nope, int d_rope, int d_v);
+size_t laga_bwd_varlen_workspace_bytes(int S_total, int n_seqs, int h, int d_c, int d_nope, int d_rope, int d_v,
+                                       unsigned flags);
+int laga_fwd_varlen(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const int* cu_seqlens,
+                    int n_seqs, int S_total, int h, int d_c, int d_nope, int d_rope, int d_v, float softmax_scale,
+                    int causal, void* out, float* lse, void* workspace, size_t workspace_bytes, unsigned flags,
+                    void* stream);
+int laga_bwd_varlen(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
+                    const float* lse, const void* dout, const int* cu_seqlens, int n_seqs, int S_total, int h,
+                    int d_c, int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* dq, void* dc_kv,
+                    void* dk_pe, float* dw_kv_b, void* workspace, size_t workspace_bytes, unsigned flags,
+                    void* stream);
+
+/*
  * Step entry points (the same kernels laga_fwd / laga_bwd launch, callable on their own).
  *
  * laga_up_project: Algorithm 1 step 4.   kv bf16 [S, h*(d_nope+d_v)] = c_kv . w_kv_b  (fp32 accumulate).

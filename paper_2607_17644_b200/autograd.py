@@ -17,10 +17,10 @@ from . import laga
 
 class _LagaAttention(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, q, c_kv, k_pe, w_kv_b, causal, softmax_scale, dw_fp32_out):
-        out, lse, _ = laga.fwd(q, c_kv, k_pe, w_kv_b, softmax_scale=softmax_scale, causal=causal)
+    def forward(ctx, q, c_kv, k_pe, w_kv_b, causal, softmax_scale, dw_fp32_out, cu_seqlens):
+        out, lse, _ = laga.fwd(q, c_kv, k_pe, w_kv_b, softmax_scale=softmax_scale, causal=causal, cu_seqlens=cu_seqlens)
         ctx.save_for_backward(q, c_kv, k_pe, w_kv_b, out, lse)
-        ctx.causal, ctx.softmax_scale, ctx.dw_fp32_out = causal, softmax_scale, dw_fp32_out
+        ctx.causal, ctx.softmax_scale, ctx.dw_fp32_out, ctx.cu_seqlens = causal, softmax_scale, dw_fp32_out, cu_seqlens
         ctx.mark_non_differentiable(lse)
         return out, lse
 
@@ -29,12 +29,17 @@ class _LagaAttention(torch.autograd.Function):
         q, c_kv, k_pe, w_kv_b, out, lse = ctx.saved_tensors
         acc = ctx.dw_fp32_out
         dq, dc_kv, dk_pe, dw, _ = laga.bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout.contiguous(), softmax_scale=ctx.softmax_scale,
-                                           causal=ctx.causal, dw_kv_b=acc, flags=laga.FLAG_ACCUM_DW if acc is not None else 0)
-        return dq, dc_kv, dk_pe, (None if acc is not None else dw.to(w_kv_b.dtype)), None, None, None
+                                           causal=ctx.causal, dw_kv_b=acc, flags=laga.FLAG_ACCUM_DW if acc is not None else 0,
+                                           cu_seqlens=ctx.cu_seqlens)
+        return dq, dc_kv, dk_pe, (None if acc is not None else dw.to(w_kv_b.dtype)), None, None, None, None
 
 
-def laga_attention(q, c_kv, k_pe, w_kv_b, causal=True, softmax_scale=None, dw_fp32_out=None, return_lse=False):
+def laga_attention(q, c_kv, k_pe, w_kv_b, causal=True, softmax_scale=None, dw_fp32_out=None, return_lse=False,
+                   cu_seqlens=None):
     """out[S,h,d_v] (and LSE) of one SP rank's head shard after the latent all-gather; differentiable in q, c_kv,
-    k_pe and w_kv_b.  Inputs are contiguous bf16 CUDA tensors with the shapes of ``laga.fwd``."""
-    out, lse = _LagaAttention.apply(q, c_kv, k_pe, w_kv_b, bool(causal), softmax_scale, dw_fp32_out)
+    k_pe and w_kv_b.  Inputs are contiguous bf16 CUDA tensors with the shapes of ``laga.fwd``.  With
+    ``cu_seqlens`` (n_seqs + 1 host integers) the rows are packed sequences and attention stays inside each."""
+    cu = None if cu_seqlens is None else tuple(int(v) for v in (cu_seqlens.tolist() if isinstance(cu_seqlens, torch.Tensor)
+                                                                  else cu_seqlens))
+    out, lse = _LagaAttention.apply(q, c_kv, k_pe, w_kv_b, bool(causal), softmax_scale, dw_fp32_out, cu)
     return (out, lse) if return_lse else out

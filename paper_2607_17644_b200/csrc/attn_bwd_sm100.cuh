@@ -38,24 +38,41 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gmem_sr
 // ---- delta and transposed softmax statistics ---------------------------------------------------
 // delta[s,i] = sum_d dO[s,i,d] O[s,i,d].  Written head-major and padded: stat_l2[i][s] = LSE*log2(e),
 // stat_delta[i][s] = delta for s < S; for S <= s < S_pad the entries are (+inf, 0) so that query rows
-// past the end of the sequence produce P = 0.
+// past the end of the sequence produce P = 0.  (S here counts the rows of out / dout / lse; S_pad the
+// padded positions, which for packed sequences exceed it by each sequence's own padding.)
 // Eight lanes per (row, head): each lane reads 16 channels of O and dO as two 16-byte loads apiece.
 __global__ void __launch_bounds__(256)
 bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
                  const float* __restrict__ lse, int S, int h, int S_pad, float* __restrict__ stat_l2,
-                 float* __restrict__ stat_delta, float4* __restrict__ zero_begin, size_t zero_count) {
+                 float* __restrict__ stat_delta, float4* __restrict__ zero_begin, size_t zero_count,
+                 const int2* __restrict__ seqs, int n_seqs) {
     // Also clears the fp32 buffer the dK/dV kernel accumulates the rope-column key gradients into
     // (zero_count float4 elements): one launch less than a separate memset.
     for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < zero_count;
          z += static_cast<size_t>(gridDim.x) * blockDim.x)
         zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;   // (row, head) pair
+    const long long item = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 3;   // (padded row, head) pair
     const int sub = threadIdx.x & 7;
     const bool live = item < static_cast<long long>(S_pad) * h;
     const int s = live ? static_cast<int>(item / h) : 0, i = live ? static_cast<int>(item % h) : 0;
+    // Packed sequences (seqs != nullptr): entry k is (first row, first padded position) of sequence k, entry
+    // n_seqs closes the list; every sequence is padded to a multiple of 128 positions of its own.  Padded
+    // position s belongs to the last sequence whose padded start is <= s.
+    int row = s;
+    bool valid = s < S;
+    if (seqs != nullptr) {
+        int lo = 0, hi = n_seqs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (seqs[mid].y <= s) lo = mid; else hi = mid - 1;
+        }
+        const int local = s - seqs[lo].y;
+        row = seqs[lo].x + local;
+        valid = row < seqs[lo + 1].x;
+    }
     float acc = 0.f;
-    if (live && s < S) {
-        const size_t base = (static_cast<size_t>(s) * h + i) * 128 + sub * 16;
+    if (live && valid) {
+        const size_t base = (static_cast<size_t>(row) * h + i) * 128 + sub * 16;
         const uint4 a0 = *reinterpret_cast<const uint4*>(out + base), a1 = *reinterpret_cast<const uint4*>(out + base + 8);
         const uint4 b0 = *reinterpret_cast<const uint4*>(dout + base), b1 = *reinterpret_cast<const uint4*>(dout + base + 8);
         const uint32_t aw[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
@@ -71,8 +88,7 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __r
 #pragma unroll
     for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (live && sub == 0) {
-        const bool valid = s < S;
-        stat_l2[static_cast<size_t>(i) * S_pad + s] = valid ? lse[static_cast<size_t>(s) * h + i] * 1.4426950408889634f : INFINITY;
+        stat_l2[static_cast<size_t>(i) * S_pad + s] = valid ? lse[static_cast<size_t>(row) * h + i] * 1.4426950408889634f : INFINITY;
         stat_delta[static_cast<size_t>(i) * S_pad + s] = valid ? acc : 0.f;
     }
 }
@@ -174,7 +190,6 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_q128 = (args.S + 127) / 128;
 
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1); mbar_init(kv_empty, 1);
@@ -204,12 +219,15 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     const uint32_t tmem_y = tmem_base + 128;
     const uint32_t tmem_dk = tmem_base + 192;
     const uint32_t tmem_dv = tmem_base + 384;
-    auto item_geometry = [&](int item, int& t0, int& head, int& j_begin, int& n_iter) {
-        int k_tile;
-        decode_item(args.sched, item, k_tile, head);
-        t0 = k_tile * 128;
-        j_begin = kCausal ? k_tile : 0;
-        n_iter = n_q128 - j_begin;             // >= 1 because t0 < S
+    // Indices are relative to the item's sequence (see SeqTile); `seq` carries its first row, its length
+    // and its start in the padded statistics arrays.
+    auto item_geometry = [&](int item, int& t0, int& head, int& j_begin, int& n_iter, SeqTile& seq) {
+        int rank;
+        decode_item(args.sched, item, rank, head);
+        seq = seq_tile(args.sched, rank, args.S, false);   // key tile 0 has the most queries
+        t0 = seq.tile * 128;
+        j_begin = kCausal ? seq.tile : 0;
+        n_iter = (seq.seq_len + 127) / 128 - j_begin;      // >= 1 because t0 < seq_len
     };
 
     if (abort_flag->value != 0u) {
@@ -223,16 +241,18 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
                 int t0, head, j_begin, n_iter;
-                item_geometry(item, t0, head, j_begin, n_iter);
+                SeqTile seq;
+                item_geometry(item, t0, head, j_begin, n_iter, seq);
+                const int row_base = seq.seq_start;
                 ok = mbar_wait(kv_empty, (n & 1u) ^ 1u, abort_flag, args.status, 0x41);
                 if (!ok) break;
                 mbar_arrive_expect_tx(kv_full, 5 * L::kSlab);
                 armed.arm(kv_full, n & 1u);
-                tma_load_2d_chk(args.status, smem + L::kK, &tmap_kv, kv_full, head * 256, t0);
-                tma_load_2d_chk(args.status, smem + L::kK + L::kSlab, &tmap_kv, kv_full, head * 256 + 64, t0);
-                tma_load_2d_chk(args.status, smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, t0);
-                tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, t0);
-                tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, kv_full, head * 256 + 192, t0);
+                tma_load_2d_chk(args.status, smem + L::kK, &tmap_kv, kv_full, head * 256, row_base + t0);
+                tma_load_2d_chk(args.status, smem + L::kK + L::kSlab, &tmap_kv, kv_full, head * 256 + 64, row_base + t0);
+                tma_load_2d_chk(args.status, smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, row_base + t0);
+                tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, row_base + t0);
+                tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, kv_full, head * 256 + 192, row_base + t0);
                 for (int j = 0; j < n_iter; ++j, ++T) {
                     const uint32_t sq = T % L::kQStages;
                     const int q0 = (j_begin + j) * 128;
@@ -242,16 +262,16 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     armed.arm(&q_full[sq], (T / L::kQStages) & 1u);
                     uint8_t* dst_q = smem + L::kQ + sq * 3 * L::kSlab;
                     for (int c = 0; c < 3; ++c)
-                        tma_load_2d_chk(args.status, dst_q + c * L::kSlab, &tmap_q, &q_full[sq], head * 192 + c * 64, q0);
+                        tma_load_2d_chk(args.status, dst_q + c * L::kSlab, &tmap_q, &q_full[sq], head * 192 + c * 64, row_base + q0);
                     float* stat = reinterpret_cast<float*>(smem + L::kStat + sq * 1024);
-                    bulk_load_1d(stat, args.stat_l2 + static_cast<size_t>(head) * args.S_pad + q0, 512, &q_full[sq]);
-                    bulk_load_1d(stat + 128, args.stat_delta + static_cast<size_t>(head) * args.S_pad + q0, 512, &q_full[sq]);
+                    bulk_load_1d(stat, args.stat_l2 + static_cast<size_t>(head) * args.S_pad + seq.pad_start + q0, 512, &q_full[sq]);
+                    bulk_load_1d(stat + 128, args.stat_delta + static_cast<size_t>(head) * args.S_pad + seq.pad_start + q0, 512, &q_full[sq]);
                     ok = mbar_wait(do_empty, (T & 1u) ^ 1u, abort_flag, args.status, 0x42);
                     if (!ok) break;
                     mbar_arrive_expect_tx(do_full, 2 * L::kSlab);
                     armed.arm(do_full, T & 1u);
                     for (int c = 0; c < 2; ++c)
-                        tma_load_2d_chk(args.status, smem + L::kDo + c * L::kSlab, &tmap_do, do_full, head * 128 + c * 64, q0);
+                        tma_load_2d_chk(args.status, smem + L::kDo + c * L::kSlab, &tmap_do, do_full, head * 128 + c * 64, row_base + q0);
                 }
             }
             if (abort_flag->value != 0u) armed.quiesce();
@@ -295,7 +315,8 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
                 int t0, head, j_begin, n_iter;
-                item_geometry(item, t0, head, j_begin, n_iter);
+                SeqTile seq;
+                item_geometry(item, t0, head, j_begin, n_iter, seq);
                 ok = mbar_wait(kv_full, n & 1u, abort_flag, args.status, 0x54);
                 if (ok) ok = issue_st(T0, T0 == 0);
                 if (ok) ok = issue_dp(T0);
@@ -359,8 +380,10 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             }
             if (item < 0) break;
             int t0, head, j_begin, n_iter;
-            item_geometry(item, t0, head, j_begin, n_iter);
-            const int t_idx = t0 + row;
+            SeqTile seq;
+            item_geometry(item, t0, head, j_begin, n_iter, seq);
+            const int t_idx = t0 + row;                       // key index within the sequence
+            const int t_row = seq.seq_start + t_idx;          // its row in the packed tensors
             for (int j = 0; j < n_iter; ++j) {
                 const uint32_t T = T0 + j;
                 const uint32_t ph = T & 1u;
@@ -440,9 +463,9 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             ok = mbar_wait_warp(acc_full, n & 1u, abort_flag, args.status, 0x64);
             if (!ok) break;
             tc_fence_after_sync();
-            const bool valid = t_idx < args.S;
-            __nv_bfloat16* dkv_row = args.dkv + static_cast<size_t>(t_idx) * args.h * 256 + head * 256;
-            float* dkr_row = args.dkpe_acc + static_cast<size_t>(t_idx) * 64;
+            const bool valid = t_idx < seq.seq_len;
+            __nv_bfloat16* dkv_row = args.dkv + static_cast<size_t>(t_row) * args.h * 256 + head * 256;
+            float* dkr_row = args.dkpe_acc + static_cast<size_t>(t_row) * 64;
             // 10 chunks of 32 columns: dK nope (0..3), dK rope (4..5), dV (6..9; dV follows dK in TMEM).
             // Group 0 drains chunks 0..4, group 1 chunks 5..9.
 #pragma unroll 1
@@ -460,7 +483,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                                                __uint_as_float(r[v * 4 + 2]) * args.scale, __uint_as_float(r[v * 4 + 3]) * args.scale);
                         if (args.dk_rope_per_head != nullptr)
                             reinterpret_cast<float4*>(args.dk_rope_per_head +
-                                                      (static_cast<size_t>(head) * args.S + t_idx) * 64 + (c - 4) * 32)[v] = w;
+                                                      (static_cast<size_t>(head) * args.S + t_row) * 64 + (c - 4) * 32)[v] = w;
                         else
                             atomicAdd(reinterpret_cast<float4*>(dkr_row + (c - 4) * 32) + v, w);
                     }
@@ -549,7 +572,6 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_q_tiles = (args.S + 127) / 128;
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1); mbar_init(q_empty, 1);
@@ -579,12 +601,14 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     const uint32_t tmem_dp = tmem_base + 128;
     const uint32_t tmem_do = tmem_base + 256;
     const uint32_t tmem_dq = tmem_base + 320;
-    auto item_geometry = [&](int item, int& q0, int& head, int& n_iter) {
+    // Indices are relative to the item's sequence (see SeqTile); `seq` carries its first row, its length
+    // and its start in the padded statistics arrays.
+    auto item_geometry = [&](int item, int& q0, int& head, int& n_iter, SeqTile& seq) {
         int rank;
         decode_item(args.sched, item, rank, head);
-        const int q_tile = n_q_tiles - 1 - rank;               // longest rows first
-        q0 = q_tile * 128;
-        n_iter = kCausal ? q_tile + 1 : n_q_tiles;
+        seq = seq_tile(args.sched, rank, args.S, true);        // longest rows first
+        q0 = seq.tile * 128;
+        n_iter = kCausal ? seq.tile + 1 : (seq.seq_len + 127) / 128;
     };
 
     if (abort_flag->value != 0u) {
@@ -594,39 +618,41 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             uint32_t T0 = 0;
             bool ok = true;
             ArmedBarriers armed(bars);
-            auto load_k = [&](uint32_t T, int j, int head) -> bool {
+            auto load_k = [&](uint32_t T, int j, int head) -> bool {   // j: first row of the key tile in the packed tensors
                 const uint32_t st = T % kDqKStages;
                 if (!mbar_wait(&k_empty[st], ((T / kDqKStages) & 1u) ^ 1u, abort_flag, args.status, 0x70)) return false;
                 mbar_arrive_expect_tx(&k_full[st], 3 * L::kSlab);
                 armed.arm(&k_full[st], (T / kDqKStages) & 1u);
                 uint8_t* sk = smem + L::kK + st * 3 * L::kSlab;
-                tma_load_2d_chk(args.status, sk, &tmap_kv, &k_full[st], head * 256, j * 128);
-                tma_load_2d_chk(args.status, sk + L::kSlab, &tmap_kv, &k_full[st], head * 256 + 64, j * 128);
-                tma_load_2d_chk(args.status, sk + 2 * L::kSlab, &tmap_kpe, &k_full[st], 0, j * 128);
+                tma_load_2d_chk(args.status, sk, &tmap_kv, &k_full[st], head * 256, j);
+                tma_load_2d_chk(args.status, sk + L::kSlab, &tmap_kv, &k_full[st], head * 256 + 64, j);
+                tma_load_2d_chk(args.status, sk + 2 * L::kSlab, &tmap_kpe, &k_full[st], 0, j);
                 return true;
             };
             for (uint32_t n = 0; ok; ++n) {
                 const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
                 int q0, head, n_iter;
-                item_geometry(item, q0, head, n_iter);
+                SeqTile seq;
+                item_geometry(item, q0, head, n_iter, seq);
+                const int row_base = seq.seq_start;
                 ok = mbar_wait(q_empty, (n & 1u) ^ 1u, abort_flag, args.status, 0x72);
                 if (!ok) break;
                 mbar_arrive_expect_tx(q_full, 3 * L::kSlab);
                 armed.arm(q_full, n & 1u);
                 for (int c = 0; c < 3; ++c)
-                    tma_load_2d_chk(args.status, smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, q0);
-                ok = load_k(T0, 0, head);
+                    tma_load_2d_chk(args.status, smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, row_base + q0);
+                ok = load_k(T0, row_base, head);
                 for (int j = 0; j < n_iter && ok; ++j) {
                     const uint32_t T = T0 + j;
-                    if (j + 1 < n_iter) ok = load_k(T + 1, j + 1, head);
+                    if (j + 1 < n_iter) ok = load_k(T + 1, row_base + (j + 1) * 128, head);
                     if (!ok) break;
                     ok = mbar_wait(v_empty, (T & 1u) ^ 1u, abort_flag, args.status, 0x71);
                     if (!ok) break;
                     mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
                     armed.arm(v_full, T & 1u);
-                    tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, v_full, head * 256 + 128, j * 128);
-                    tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, j * 128);
+                    tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, v_full, head * 256 + 128, row_base + j * 128);
+                    tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, row_base + j * 128);
                 }
                 T0 += static_cast<uint32_t>(n_iter);
             }
@@ -669,7 +695,8 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
                 int q0, head, n_iter;
-                item_geometry(item, q0, head, n_iter);
+                SeqTile seq;
+                item_geometry(item, q0, head, n_iter, seq);
                 ok = mbar_wait(q_full, n & 1u, abort_flag, args.status, 0x81);
                 if (ok) ok = issue_s(T0);
                 if (ok && n_iter == 1) mma_commit(q_empty);
@@ -714,10 +741,10 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             return it;
         };
         // dQ of a finished item: six 32-column chunks, three per group
-        auto drain = [&](uint32_t n_done, int s_idx, int head) -> bool {
+        // (s_idx: the row in the packed tensors; valid: it lies inside its sequence)
+        auto drain = [&](uint32_t n_done, int s_idx, bool valid, int head) -> bool {
             if (!mbar_wait_warp(acc_full, n_done & 1u, abort_flag, args.status, 0x92)) return false;
             tc_fence_after_sync();
-            const bool valid = s_idx < args.S;
             __nv_bfloat16* dst = args.dq + (static_cast<size_t>(s_idx) * args.h + head) * 192;
 #pragma unroll 1
             for (int c = g * 3; c < g * 3 + 3; ++c) {
@@ -746,16 +773,20 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         bool ok = true;
         int item = read_item(0, ok);
         int prev_s_idx = 0, prev_head = 0;
+        bool prev_valid = false;
         for (uint32_t n = 0; ok && item >= 0; ++n) {
             int q0, head, n_iter;
-            item_geometry(item, q0, head, n_iter);
-            const int s_idx = q0 + row;
-            const bool valid = s_idx < args.S;
+            SeqTile seq;
+            item_geometry(item, q0, head, n_iter, seq);
+            const int S_seq = seq.seq_len;
+            const int s_idx = q0 + row;                       // query index within the sequence
+            const int s_row = seq.seq_start + s_idx;          // its row in the packed tensors
+            const bool valid = s_idx < S_seq;
             {   // this thread's dO row, channels [64g, 64g+64), as 32 packed words into TMEM (the previous item's
                 // last dP MMA has completed: this group waited for it before writing its last dS)
                 uint32_t w[32];
                 if (valid) {
-                    const uint4* src = reinterpret_cast<const uint4*>(args.dout + (static_cast<size_t>(s_idx) * args.h + head) * 128 + g * 64);
+                    const uint4* src = reinterpret_cast<const uint4*>(args.dout + (static_cast<size_t>(s_row) * args.h + head) * 128 + g * 64);
 #pragma unroll
                     for (int v = 0; v < 8; ++v) {
                         const uint4 x = src[v];
@@ -772,9 +803,9 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 mbar_arrive(do_ready);
             }
             // Rows past the end of the sequence get LSE = +inf so that their P is exactly zero.
-            const float l2 = valid ? args.lse[static_cast<size_t>(s_idx) * args.h + head] * 1.4426950408889634f : INFINITY;
-            const float delta = valid ? args.stat_delta[static_cast<size_t>(head) * args.S_pad + s_idx] : 0.f;
-            if (n > 0) ok = drain(n - 1, prev_s_idx, prev_head);
+            const float l2 = valid ? args.lse[static_cast<size_t>(s_row) * args.h + head] * 1.4426950408889634f : INFINITY;
+            const float delta = valid ? args.stat_delta[static_cast<size_t>(head) * args.S_pad + seq.pad_start + s_idx] : 0.f;
+            if (n > 0) ok = drain(n - 1, prev_s_idx, prev_valid, prev_head);
             for (int j = 0; j < n_iter && ok; ++j) {
                 const uint32_t T = T0 + j;
                 ok = mbar_wait_warp(s_full, T & 1u, abort_flag, args.status, 0x90);
@@ -787,14 +818,14 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 tc_fence_before_sync();
                 mbar_arrive(s_read);
                 const int tk0 = j * 128 + g * 64;
-                const bool edge = (kCausal && tk0 + 63 > q0) || (tk0 + 64 > args.S);
+                const bool edge = (kCausal && tk0 + 63 > q0) || (tk0 + 64 > S_seq);
                 float p[64];
 #pragma unroll
                 for (int c = 0; c < 64; ++c) {
                     float v = fast_exp2(fmaf(__uint_as_float(sv[c]), args.scale_log2, -l2));
                     if (edge) {
                         const int t = tk0 + c;
-                        if ((kCausal && t > s_idx) || t >= args.S) v = 0.f;
+                        if ((kCausal && t > s_idx) || t >= S_seq) v = 0.f;
                     }
                     p[c] = v;
                 }
@@ -816,10 +847,11 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             }
             if (!ok) break;
             T0 += static_cast<uint32_t>(n_iter);
-            prev_s_idx = s_idx;
+            prev_s_idx = s_row;
+            prev_valid = valid;
             prev_head = head;
             item = read_item(n + 1, ok);
-            if (ok && item < 0) ok = drain(n, prev_s_idx, prev_head);
+            if (ok && item < 0) ok = drain(n, prev_s_idx, prev_valid, prev_head);
         }
     }
     tc_fence_before_sync();

@@ -105,7 +105,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     float* lsum = reinterpret_cast<float*>(smem + L::kLsum);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_q_tiles = (args.S + 127) / 128;
 
     if (threadIdx.x == 0) {
         mbar_init(q_ready, 128);
@@ -137,11 +136,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base + 3 * BK;       // [0,288) three S tiles | [288,416) O | [416,512) Q as packed bf16
     const uint32_t tmem_q = tmem_o + 128;
-    auto item_geometry = [&](int item, int& q0, int& head, int& n_kv) {
+    // q0 and every key index are relative to the item's sequence; row_base is the sequence's first row in the
+    // packed tensors and S_seq its length (0 and S for a single sequence).
+    auto item_geometry = [&](int item, int& q0, int& head, int& n_kv, int& row_base, int& S_seq) {
         int rank;
         decode_item(args.sched, item, rank, head);
-        q0 = (n_q_tiles - 1 - rank) * 128;                              // longest rows first
-        const int n_keys = kCausal ? min(q0 + 128, args.S) : args.S;    // keys any row of this tile attends to
+        const SeqTile st = seq_tile(args.sched, rank, args.S, true);    // longest rows first
+        q0 = st.tile * 128;
+        row_base = st.seq_start;
+        S_seq = st.seq_len;
+        const int n_keys = kCausal ? min(q0 + 128, S_seq) : S_seq;      // keys any row of this tile attends to
         n_kv = (n_keys + BK - 1) / BK;
     };
 
@@ -157,8 +161,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             for (uint32_t n = 0; ok; ++n) {
                 const int item = ring_publish(ring, args.sched, n, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
-                int q0, head, n_kv;
-                item_geometry(item, q0, head, n_kv);
+                int q0, head, n_kv, row_base, S_seq;
+                item_geometry(item, q0, head, n_kv, row_base, S_seq);
                 for (int j = 0; j < n_kv; ++j, ++T) {
                     const uint32_t s = T % kFwdStages;
                     ok = mbar_wait(&k_empty[s], ((T / kFwdStages) & 1u) ^ 1u, abort_flag, args.status, 0x10);
@@ -166,9 +170,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     uint8_t* dk = smem + L::kK + s * 3 * L::kSlab;
                     mbar_arrive_expect_tx(&k_full[s], 3 * L::kSlab);
                     armed.arm(&k_full[s], (T / kFwdStages) & 1u);
-                    tma_load_2d_chk(args.status, dk, &tmap_kv, &k_full[s], head * 256, j * BK);
-                    tma_load_2d_chk(args.status, dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, j * BK);
-                    tma_load_2d_chk(args.status, dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, j * BK);
+                    tma_load_2d_chk(args.status, dk, &tmap_kv, &k_full[s], head * 256, row_base + j * BK);
+                    tma_load_2d_chk(args.status, dk + L::kSlab, &tmap_kv, &k_full[s], head * 256 + 64, row_base + j * BK);
+                    tma_load_2d_chk(args.status, dk + 2 * L::kSlab, &tmap_kpe, &k_full[s], 0, row_base + j * BK);
                 }
             }
             if (abort_flag->value != 0u) armed.quiesce();
@@ -181,8 +185,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             for (uint32_t n = 0; ok; ++n) {
                 const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
-                int q0, head, n_kv;
-                item_geometry(item, q0, head, n_kv);
+                int q0, head, n_kv, row_base, S_seq;
+                item_geometry(item, q0, head, n_kv, row_base, S_seq);
                 for (int j = 0; j < n_kv; ++j, ++T) {
                     const uint32_t s = T % kFwdStages;
                     ok = mbar_wait(&v_empty[s], ((T / kFwdStages) & 1u) ^ 1u, abort_flag, args.status, 0x11);
@@ -190,8 +194,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     uint8_t* dv = smem + L::kV + s * 2 * L::kSlab;
                     mbar_arrive_expect_tx(&v_full[s], 2 * L::kSlab);
                     armed.arm(&v_full[s], (T / kFwdStages) & 1u);
-                    tma_load_2d_chk(args.status, dv, &tmap_kv, &v_full[s], head * 256 + 128, j * BK);
-                    tma_load_2d_chk(args.status, dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, j * BK);
+                    tma_load_2d_chk(args.status, dv, &tmap_kv, &v_full[s], head * 256 + 128, row_base + j * BK);
+                    tma_load_2d_chk(args.status, dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, row_base + j * BK);
                 }
             }
             if (abort_flag->value != 0u) armed.quiesce();
@@ -220,8 +224,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             for (uint32_t n = 0; ok; ++n) {
                 const int item = ring_read(ring, n, true, abort_flag, args.status, ok);
                 if (!ok || item < 0) break;
-                int q0, head, n_kv;
-                item_geometry(item, q0, head, n_kv);
+                int q0, head, n_kv, row_base, S_seq;
+                item_geometry(item, q0, head, n_kv, row_base, S_seq);
                 ok = mbar_wait(q_ready, n & 1u, abort_flag, args.status, 0x22);
                 for (int j = 0; j < 3 && j < n_kv && ok; ++j) {
                     const uint32_t T = T0 + j;
@@ -278,10 +282,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             return it;
         };
         // O of a finished item (all of its MMAs are known complete): each group drains half of the columns
-        auto drain = [&](int sq_idx, int head, float m_fin, float l_run) {
+        // (sq_idx: the row in the packed tensors; valid: it lies inside its sequence)
+        auto drain = [&](int sq_idx, bool valid, int head, float m_fin, float l_run) {
             tc_fence_after_sync();
             const float inv_l = 1.0f / l_run;
-            const bool valid = sq_idx < args.S;
             __nv_bfloat16* dst = args.out + (static_cast<size_t>(sq_idx) * args.h + head) * 128;
 #pragma unroll 1
             for (int c = 2 * g; c < 2 * g + 2; ++c) {
@@ -311,15 +315,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
         bool ok = true;
         int item = read_item(0, ok);
         int prev_sq_idx = 0, prev_head = 0;
+        bool prev_valid = false;
         float prev_m_fin = 0.f, prev_l_run = 1.f;
         for (uint32_t n = 0; ok && item >= 0; ++n) {
-            int q0, head, n_kv;
-            item_geometry(item, q0, head, n_kv);
-            const int sq_idx = q0 + row;              // global query index
+            int q0, head, n_kv, row_base, S_seq;
+            item_geometry(item, q0, head, n_kv, row_base, S_seq);
+            const int sq_idx = q0 + row;              // query index within the sequence
             if (g == 0) {   // this thread's query row (192 bf16 = 96 packed words) goes to TMEM once, as the A operand of S
                             // (the previous item's MMAs, which read the old tile, are known complete)
-                const bool q_valid = sq_idx < args.S;
-                const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(sq_idx) * args.h + head) * 192);
+                const bool q_valid = sq_idx < S_seq;
+                const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(row_base + sq_idx) * args.h + head) * 192);
 #pragma unroll 1
                 for (int c = 0; c < 3; ++c) {
                     uint32_t w[32];
@@ -335,7 +340,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 tc_fence_before_sync();
                 mbar_arrive(q_ready);
             }
-            if (n > 0) drain(prev_sq_idx, prev_head, prev_m_fin, prev_l_run);
+            if (n > 0) drain(prev_sq_idx, prev_valid, prev_head, prev_m_fin, prev_l_run);
             float m_mine = -INFINITY;                     // reference max (scaled, log2 domain) l_part refers to
             float l_part = 0.f;                           // this group's part of the row sum
             for (int j = 0; j < n_kv; ++j) {
@@ -352,11 +357,11 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 tmem_ld_wait();
 
                 const int t_last = j * BK + BK - 1;
-                if ((kCausal && t_last > q0) || t_last >= args.S) {   // the causal edge can cross two tiles
+                if ((kCausal && t_last > q0) || t_last >= S_seq) {   // the causal edge can cross two tiles
 #pragma unroll
                     for (int c = 0; c < BK; ++c) {
                         const int t = j * BK + c;
-                        if ((kCausal && t > sq_idx) || t >= args.S) sv[c] = __float_as_uint(-INFINITY);
+                        if ((kCausal && t > sq_idx) || t >= S_seq) sv[c] = __float_as_uint(-INFINITY);
                     }
                 }
                 // eight independent chains (three-input max: two elements per instruction)
@@ -440,13 +445,14 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             if (!ok) break;
             prev_l_run = lsum_n[row] + lsum_n[128 + row];
             prev_m_fin = m_fin;
-            prev_sq_idx = sq_idx;
+            prev_sq_idx = row_base + sq_idx;
+            prev_valid = sq_idx < S_seq;
             prev_head = head;
             ok = mbar_wait_warp(all_done, n & 1u, abort_flag, args.status, 0x32);
             if (!ok) break;
             T0 += static_cast<uint32_t>(n_kv);
             item = read_item(n + 1, ok);
-            if (ok && item < 0) drain(prev_sq_idx, prev_head, prev_m_fin, prev_l_run);
+            if (ok && item < 0) drain(prev_sq_idx, prev_valid, prev_head, prev_m_fin, prev_l_run);
         }
     }
     tc_fence_before_sync();

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
+#include <cstring>
 #include <initializer_list>
 #include <mutex>
 #include <vector>
@@ -263,12 +265,12 @@ struct ScopedKernelEvents {
 // How many of the h heads the persistent attention kernels sweep position by position instead of head by
 // head (see work_sched.cuh): as many as keep the swept heads' streamed operands (640 bytes per token and
 // head: K_nope, V and the rope band on one side, Q and dO on the other) within half of the 126 MB L2.
-WorkSchedule make_schedule(int n_tiles, int S, int h, unsigned* counter) {
+WorkSchedule make_schedule(int n_tiles, int S, int h, unsigned* counter, const int4* tiles = nullptr) {
     const long long per_head = static_cast<long long>(S) * 640;
     long long banded = (64ll << 20) / (per_head > 0 ? per_head : 1);
     if (banded < 1) banded = 1;
     if (banded > h) banded = h;
-    return WorkSchedule{n_tiles, h, static_cast<int>(banded), n_tiles * h, counter};
+    return WorkSchedule{n_tiles, h, static_cast<int>(banded), n_tiles * h, counter, tiles};
 }
 
 // ---- Algorithm 1 step 4: KV[S, N] = c_kv[S, d_c] . W[d_c, N] ------------------------------------
@@ -340,18 +342,85 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool d
     return launch_status();
 }
 
+// ---- packed variable-length sequences ---------------------------------------------------------------
+// Host-side plan of one call over packed sequences: every sequence's 128-row tiles in the two orders the
+// kernels want (longest work first) and the sequences' starts in the packed tensors and in the padded
+// statistics arrays.  `image` is what gets copied to the device, in one piece:
+//     int4 q_tiles[n_tiles] | int4 k_tiles[n_tiles] | int2 seqs[n_seqs + 1]
+struct SeqPlan {
+    int n_seqs = 0, S_total = 0, n_tiles = 0;
+    std::vector<int4> image;
+    size_t q_tiles_offset() const { return 0; }
+    size_t k_tiles_offset() const { return static_cast<size_t>(n_tiles) * sizeof(int4); }
+    size_t seqs_offset() const { return 2 * static_cast<size_t>(n_tiles) * sizeof(int4); }
+};
+// Upper bounds that depend only on (S_total, n_seqs), so that the workspace can be sized without the lengths.
+int varlen_s_pad(int S_total, int n_seqs) { return (S_total + 127 * n_seqs + 127) / 128 * 128; }
+int varlen_max_tiles(int S_total, int n_seqs) { return S_total / 128 + n_seqs; }
+size_t varlen_table_bytes(int S_total, int n_seqs) {
+    return align_up(2 * static_cast<size_t>(varlen_max_tiles(S_total, n_seqs)) * sizeof(int4) +
+                        (static_cast<size_t>(n_seqs) + 2) / 2 * sizeof(int4),
+                    1024);
+}
+
+// cu_seqlens: n_seqs + 1 non-decreasing host integers, cu[0] = 0, cu[n_seqs] = S_total.  Empty sequences are
+// allowed and contribute nothing.
+bool build_seq_plan(const int* cu, int n_seqs, int S_total, bool causal, SeqPlan* plan) {
+    if (cu[0] != 0 || cu[n_seqs] != S_total) return false;
+    struct Entry { int4 t; int work; };
+    std::vector<Entry> q_order, k_order;
+    std::vector<int2> seqs(static_cast<size_t>(n_seqs) + 1);
+    int pad = 0;
+    for (int k = 0; k < n_seqs; ++k) {
+        const int len = cu[k + 1] - cu[k];
+        if (len < 0) return false;
+        seqs[k] = make_int2(cu[k], pad);
+        const int tiles = (len + 127) / 128;
+        for (int t = 0; t < tiles; ++t) {
+            const int4 e = make_int4(cu[k], len, t, pad);
+            q_order.push_back({e, causal ? t + 1 : tiles});        // a query tile attends to the key tiles before it
+            k_order.push_back({e, causal ? tiles - t : tiles});    // a key tile is attended by the query tiles after it
+        }
+        pad += tiles * 128;
+    }
+    seqs[n_seqs] = make_int2(S_total, pad);
+    auto by_work = [](const Entry& a, const Entry& b) { return a.work > b.work; };
+    std::stable_sort(q_order.begin(), q_order.end(), by_work);
+    std::stable_sort(k_order.begin(), k_order.end(), by_work);
+    plan->n_seqs = n_seqs;
+    plan->S_total = S_total;
+    plan->n_tiles = static_cast<int>(q_order.size());
+    plan->image.assign(2 * q_order.size() + (seqs.size() + 1) / 2, make_int4(0, 0, 0, 0));
+    for (size_t i = 0; i < q_order.size(); ++i) {
+        plan->image[i] = q_order[i].t;
+        plan->image[q_order.size() + i] = k_order[i].t;
+    }
+    std::memcpy(plan->image.data() + 2 * q_order.size(), seqs.data(), seqs.size() * sizeof(int2));
+    return plan->n_tiles > 0;
+}
+
+// Copies the plan into the workspace.  The source is pageable host memory: the runtime stages it before the
+// call returns (so the plan may be freed afterwards), at the price of a stream synchronisation inside the call.
+int upload_seq_plan(const SeqPlan& plan, void* tables, cudaStream_t stream) {
+    return cudaMemcpyAsync(tables, plan.image.data(), plan.image.size() * sizeof(int4), cudaMemcpyHostToDevice, stream) ==
+                   cudaSuccess
+               ? LAGA_OK
+               : LAGA_ERR_CUDA;
+}
+
 // ---- Algorithm 1 step 5 -------------------------------------------------------------------------
 int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int h, float softmax_scale,
-                    int causal, void* out, float* lse, unsigned* status, cudaStream_t stream) {
+                    int causal, void* out, float* lse, unsigned* status, cudaStream_t stream,
+                    const int4* q_tiles = nullptr, int n_seq_tiles = 0) {
     using L = AttnFwdSmem;
     const int N = h * (kDn + kDv);
     CUtensorMap tkv, tpe;   // boxes of 64 columns x one key tile of rows
     if (!cached_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, kFwdKeys)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, kFwdKeys)) return LAGA_ERR_CUDA;
-    const int n_tiles = (S + 127) / 128;
+    const int n_tiles = q_tiles ? n_seq_tiles : (S + 127) / 128;
     AttnFwdArgs a{S, h, softmax_scale * 1.4426950408889634f, reinterpret_cast<const __nv_bfloat16*>(q),
                   reinterpret_cast<__nv_bfloat16*>(out), lse, status,
-                  make_schedule(n_tiles, S, h, slot_counter(status, kSlotFwd)), slot_probe(status, kSlotFwd)};
+                  make_schedule(n_tiles, S, h, slot_counter(status, kSlotFwd), q_tiles), slot_probe(status, kSlotFwd)};
     dim3 grid(persistent_grid(n_tiles * h), 1, 1);
     ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream);
     if (causal) attn_fwd_sm100_kernel<true><<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a);
@@ -361,7 +430,7 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
 
 // ---- Section 5.2: backward of step 5 ------------------------------------------------------------
 struct BwdWorkspace {
-    size_t kv, dkv, stat_l2, stat_delta, dkpe_acc, dk_rope_per_head, dq_acc, total;
+    size_t kv, dkv, stat_l2, stat_delta, dkpe_acc, dk_rope_per_head, dq_acc, tables, total;
     int S_pad;
     int head_window;      // heads per launch of the fused backward; 0 = the two-kernel backward
 };
@@ -382,10 +451,11 @@ int fused_head_window(int S, int h) {
     return (h + launches - 1) / launches;
 }
 
-BwdWorkspace bwd_workspace_layout(int S, int h, bool deterministic, bool fused) {
+// n_seqs = 0: one sequence of S tokens; otherwise S tokens in n_seqs packed sequences (tables at the end).
+BwdWorkspace bwd_workspace_layout(int S, int h, bool deterministic, bool fused, int n_seqs = 0) {
     BwdWorkspace w;
     const size_t kv_bytes = align_up(static_cast<size_t>(S) * h * (kDn + kDv) * 2, 1024);
-    w.S_pad = (S + 127) / 128 * 128;
+    w.S_pad = n_seqs > 0 ? varlen_s_pad(S, n_seqs) : (S + 127) / 128 * 128;
     const size_t stat_bytes = align_up(static_cast<size_t>(h) * w.S_pad * sizeof(float), 1024);
     w.kv = kStatusBytes;
     w.dkv = w.kv + kv_bytes;
@@ -396,14 +466,17 @@ BwdWorkspace bwd_workspace_layout(int S, int h, bool deterministic, bool fused) 
     w.dq_acc = w.dk_rope_per_head +
                (deterministic ? align_up(static_cast<size_t>(h) * S * kDr * sizeof(float), 1024) : 0);
     w.head_window = fused ? fused_head_window(S, h) : 0;
-    w.total = w.dq_acc + align_up(static_cast<size_t>(S) * w.head_window * (kDn + kDr) * sizeof(float), 1024);
+    w.tables = w.dq_acc + align_up(static_cast<size_t>(S) * w.head_window * (kDn + kDr) * sizeof(float), 1024);
+    w.total = w.tables + (n_seqs > 0 ? varlen_table_bytes(S, n_seqs) : 0);
     return w;
 }
 
 int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void* out, const float* lse,
                     const void* dout, int S, int h, float softmax_scale, int causal, void* dq, void* dkv,
                     void* dk_pe, float* stat_l2, float* stat_delta, float* dkpe_acc, float* dk_rope_per_head, int S_pad,
-                    float* dq_acc, int head_window, unsigned* status, cudaStream_t stream) {
+                    float* dq_acc, int head_window, unsigned* status, cudaStream_t stream,
+                    const int4* q_tiles = nullptr, const int4* k_tiles = nullptr, const int2* seqs = nullptr,
+                    int n_seqs = 0, int n_seq_tiles = 0) {
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
     {   // delta and the transposed, padded softmax statistics; clears the rope-gradient accumulator on the way
@@ -413,7 +486,7 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         bwd_delta_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(out),
                                                      reinterpret_cast<const __nv_bfloat16*>(dout), lse, S, h, S_pad,
                                                      stat_l2, stat_delta, reinterpret_cast<float4*>(dkpe_acc),
-                                                     static_cast<size_t>(S) * kDr / 4);
+                                                     static_cast<size_t>(S) * kDr / 4, seqs, n_seqs);
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     }
     const uint64_t q_row = static_cast<uint64_t>(h) * 192, do_row = static_cast<uint64_t>(h) * 128;
@@ -422,7 +495,7 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         !cached_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, 128) ||
         !cached_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, 128))
         return LAGA_ERR_CUDA;
-    const int n_tiles = (S + 127) / 128;
+    const int n_tiles = q_tiles ? n_seq_tiles : (S + 127) / 128;
     if (head_window > 0) {
         // One pass over the score tiles on CTA pairs, a window of heads per launch; dQ goes through dq_acc.
         if (cudaMemsetAsync(dq_acc, 0, static_cast<size_t>(S) * head_window * (kDn + kDr) * sizeof(float), stream) != cudaSuccess)
@@ -453,10 +526,10 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         dim3 grid(persistent_grid(n_tiles * h), 1, 1);
         AttnBwdDkvArgs a{S, h, S_pad, scale_log2, softmax_scale, stat_l2, stat_delta,
                          reinterpret_cast<__nv_bfloat16*>(dkv), dkpe_acc, dk_rope_per_head, status,
-                         make_schedule(n_tiles, S, h, slot_counter(status, kSlotDkv)), slot_probe(status, kSlotDkv)};
+                         make_schedule(n_tiles, S, h, slot_counter(status, kSlotDkv), k_tiles), slot_probe(status, kSlotDkv)};
         AttnBwdDqArgs b{S, h, scale_log2, softmax_scale, lse, stat_delta, S_pad,
                         reinterpret_cast<const __nv_bfloat16*>(dout), reinterpret_cast<__nv_bfloat16*>(dq), status,
-                        make_schedule(n_tiles, S, h, slot_counter(status, kSlotDq)), slot_probe(status, kSlotDq)};
+                        make_schedule(n_tiles, S, h, slot_counter(status, kSlotDq), q_tiles), slot_probe(status, kSlotDq)};
         {
             ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream);
             if (causal) attn_bwd_dkv_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
@@ -628,9 +701,10 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
     return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st);
 }
 
-int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
-             int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out, float* lse,
-             void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+// laga_fwd and laga_fwd_varlen: cu_seqlens == nullptr means one sequence of S tokens.
+static int fwd_impl(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const int* cu_seqlens, int n_seqs,
+                    int S, int h, int d_c, int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out,
+                    float* lse, void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
     if (!q || !c_kv || !k_pe || !w_kv_b || !out || !lse || !workspace || S < 1 || h < 1)
         return LAGA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(c_kv) || !aligned16(k_pe) || !aligned16(w_kv_b) || !aligned16(out) ||
@@ -638,23 +712,66 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
         return LAGA_ERR_INVALID_ARG;
     if (flags != 0 || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
     if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
-    if (workspace_bytes < laga_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v))
+    const size_t kv_end = laga_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v);
+    SeqPlan plan;
+    if (cu_seqlens != nullptr) {
+        if (n_seqs < 1 || !build_seq_plan(cu_seqlens, n_seqs, S, causal != 0, &plan)) return LAGA_ERR_INVALID_ARG;
+        if (workspace_bytes < kv_end + varlen_table_bytes(S, n_seqs)) return LAGA_ERR_WORKSPACE_TOO_SMALL;
+    } else if (workspace_bytes < kv_end) {
         return LAGA_ERR_WORKSPACE_TOO_SMALL;
+    }
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
     if ((rc = check_pointers({q, c_kv, k_pe, w_kv_b, out, lse, workspace})) != LAGA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned* status = static_cast<unsigned*>(workspace);
-    void* kv = static_cast<uint8_t*>(workspace) + kStatusBytes;
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    void* kv = base + kStatusBytes;
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
+    const int4* q_tiles = nullptr;
+    if (cu_seqlens != nullptr) {
+        if ((rc = upload_seq_plan(plan, base + kv_end, st)) != LAGA_OK) return rc;
+        q_tiles = reinterpret_cast<const int4*>(base + kv_end + plan.q_tiles_offset());
+    }
+    // step 4 is token-wise: one GEMM over all the packed tokens
     if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
-    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st);
+    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st, q_tiles, plan.n_tiles);
 }
 
-int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
-             const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
-             float softmax_scale, int causal, void* dq, void* dc_kv, void* dk_pe, float* dw_kv_b, void* workspace,
-             size_t workspace_bytes, unsigned flags, void* stream) {
+int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
+             int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* out, float* lse,
+             void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+    return fwd_impl(q, c_kv, k_pe, w_kv_b, nullptr, 0, S, h, d_c, d_nope, d_rope, d_v, softmax_scale, causal, out, lse,
+                    workspace, workspace_bytes, flags, stream);
+}
+
+size_t laga_fwd_varlen_workspace_bytes(int S_total, int n_seqs, int h, int d_c, int d_nope, int d_rope, int d_v) {
+    const size_t base = laga_fwd_workspace_bytes(S_total, h, d_c, d_nope, d_rope, d_v);
+    if (base == 0 || n_seqs < 1) return 0;
+    return base + varlen_table_bytes(S_total, n_seqs);
+}
+
+size_t laga_bwd_varlen_workspace_bytes(int S_total, int n_seqs, int h, int d_c, int d_nope, int d_rope, int d_v,
+                                       unsigned flags) {
+    if (S_total < 1 || h < 1 || n_seqs < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
+    if (flags & LAGA_FLAG_FUSED_BWD) return 0;
+    return bwd_workspace_layout(S_total, h, (flags & LAGA_FLAG_DETERMINISTIC) != 0, false, n_seqs).total;
+}
+
+int laga_fwd_varlen(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const int* cu_seqlens,
+                    int n_seqs, int S_total, int h, int d_c, int d_nope, int d_rope, int d_v, float softmax_scale,
+                    int causal, void* out, float* lse, void* workspace, size_t workspace_bytes, unsigned flags,
+                    void* stream) {
+    if (!cu_seqlens) return LAGA_ERR_INVALID_ARG;
+    return fwd_impl(q, c_kv, k_pe, w_kv_b, cu_seqlens, n_seqs, S_total, h, d_c, d_nope, d_rope, d_v, softmax_scale, causal,
+                    out, lse, workspace, workspace_bytes, flags, stream);
+}
+
+// laga_bwd and laga_bwd_varlen: cu_seqlens == nullptr means one sequence of S tokens.
+static int bwd_impl(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out, const float* lse,
+                    const void* dout, const int* cu_seqlens, int n_seqs, int S, int h, int d_c, int d_nope, int d_rope,
+                    int d_v, float softmax_scale, int causal, void* dq, void* dc_kv, void* dk_pe, float* dw_kv_b,
+                    void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
     if (!q || !c_kv || !k_pe || !w_kv_b || !out || !lse || !dout || !dq || !dc_kv || !dk_pe || !dw_kv_b ||
         !workspace || S < 1 || h < 1)
         return LAGA_ERR_INVALID_ARG;
@@ -669,7 +786,11 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
     const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
     const bool fused = (flags & LAGA_FLAG_FUSED_BWD) != 0;
     if (fused && deterministic) return LAGA_ERR_INVALID_ARG;   // the fused kernel's dQ and dk_pe sums are order dependent
-    const BwdWorkspace w = bwd_workspace_layout(S, h, deterministic, fused);
+    if (fused && cu_seqlens != nullptr) return LAGA_ERR_INVALID_ARG;   // the one-pass kernel takes one sequence
+    SeqPlan plan;
+    if (cu_seqlens != nullptr && (n_seqs < 1 || !build_seq_plan(cu_seqlens, n_seqs, S, causal != 0, &plan)))
+        return LAGA_ERR_INVALID_ARG;
+    const BwdWorkspace w = bwd_workspace_layout(S, h, deterministic, fused, cu_seqlens ? n_seqs : 0);
     if (workspace_bytes < w.total) return LAGA_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();
     if (rc != LAGA_OK) return rc;
@@ -682,6 +803,14 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
     void* dkv = base + w.dkv;
     const int N = h * (kDn + kDv);
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
+    const int4 *q_tiles = nullptr, *k_tiles = nullptr;
+    const int2* seqs = nullptr;
+    if (cu_seqlens != nullptr) {
+        if ((rc = upload_seq_plan(plan, base + w.tables, st)) != LAGA_OK) return rc;
+        q_tiles = reinterpret_cast<const int4*>(base + w.tables + plan.q_tiles_offset());
+        k_tiles = reinterpret_cast<const int4*>(base + w.tables + plan.k_tiles_offset());
+        seqs = reinterpret_cast<const int2*>(base + w.tables + plan.seqs_offset());
+    }
     // K_nope / V are recomputed from the latent (the forward keeps only out and lse) unless the caller
     // vouches that the forward's copy is still in this workspace: both layouts put it right after the status.
     if (!(flags & LAGA_FLAG_KV_SAVED) && (rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
@@ -689,12 +818,31 @@ int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
                               reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
                               reinterpret_cast<float*>(base + w.dkpe_acc),
                               deterministic ? reinterpret_cast<float*>(base + w.dk_rope_per_head) : nullptr, w.S_pad,
-                              reinterpret_cast<float*>(base + w.dq_acc), w.head_window, status, st)) != LAGA_OK)
+                              reinterpret_cast<float*>(base + w.dq_acc), w.head_window, status, st, q_tiles, k_tiles, seqs,
+                              plan.n_seqs, plan.n_tiles)) != LAGA_OK)
         return rc;
+    // the two GEMMs of Section 5.2 are token-wise: one launch each over all the packed tokens
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,
                           accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st)) != LAGA_OK)
         return rc;
     return launch_dw(c_kv, dkv, S, N, dw_kv_b, deterministic, status, st);
+}
+
+int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
+             const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
+             float softmax_scale, int causal, void* dq, void* dc_kv, void* dk_pe, float* dw_kv_b, void* workspace,
+             size_t workspace_bytes, unsigned flags, void* stream) {
+    return bwd_impl(q, c_kv, k_pe, w_kv_b, out, lse, dout, nullptr, 0, S, h, d_c, d_nope, d_rope, d_v, softmax_scale, causal,
+                    dq, dc_kv, dk_pe, dw_kv_b, workspace, workspace_bytes, flags, stream);
+}
+
+int laga_bwd_varlen(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
+                    const float* lse, const void* dout, const int* cu_seqlens, int n_seqs, int S_total, int h, int d_c,
+                    int d_nope, int d_rope, int d_v, float softmax_scale, int causal, void* dq, void* dc_kv, void* dk_pe,
+                    float* dw_kv_b, void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+    if (!cu_seqlens) return LAGA_ERR_INVALID_ARG;
+    return bwd_impl(q, c_kv, k_pe, w_kv_b, out, lse, dout, cu_seqlens, n_seqs, S_total, h, d_c, d_nope, d_rope, d_v,
+                    softmax_scale, causal, dq, dc_kv, dk_pe, dw_kv_b, workspace, workspace_bytes, flags, stream);
 }
 
 // ---- forward without caller-provided scratch ----------------------------------------------------

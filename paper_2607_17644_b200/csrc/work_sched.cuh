@@ -18,7 +18,26 @@ struct WorkSchedule {
     int banded_heads;     // 1 <= banded_heads <= h
     int total_items;      // n_tiles * h
     unsigned int* counter;   // global, zero when the kernel starts
+    const int4* tiles;    // packed sequences: one entry per tile rank (below); nullptr = one sequence of S tokens
 };
+
+// Packed variable-length sequences.  The tokens of all sequences are stacked along the row axis; a tile never
+// spans two sequences.  The host lists every sequence's tiles, longest work first, as
+// (seq_start, seq_len, tile index within the sequence, start of the sequence in the padded statistics arrays);
+// rank r of the schedule is entry r.  Rows a tile reads past its sequence's end belong to the next sequence
+// (or are TMA zero fill at the very end): the kernels mask them by the sequence length exactly as they mask
+// the rows past S for a single sequence.
+struct SeqTile {
+    int seq_start;   // first row of the sequence in the packed tensors
+    int seq_len;
+    int tile;        // tile index within the sequence
+    int pad_start;   // first entry of the sequence in the per-head statistics arrays (a multiple of 128)
+};
+__device__ __forceinline__ SeqTile seq_tile(const WorkSchedule& ws, int rank, int S, bool longest_is_last) {
+    if (ws.tiles == nullptr) return SeqTile{0, S, longest_is_last ? ws.n_tiles - 1 - rank : rank, 0};
+    const int4 t = __ldg(ws.tiles + rank);
+    return SeqTile{t.x, t.y, t.z, t.w};
+}
 
 // item -> (rank of the tile within its head, longest first; head)
 __device__ __forceinline__ void decode_item(const WorkSchedule& ws, int item, int& rank, int& head) {

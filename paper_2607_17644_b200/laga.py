@@ -38,6 +38,10 @@ SIGNATURES = {
     "laga_bwd_workspace_bytes": (_sz, [_ci] * 6 + [_cu]),
     "laga_fwd": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
     "laga_bwd": (_ci, [_vp] * 7 + [_ci] * 6 + [_cf, _ci] + [_vp] * 4 + [_vp, _sz, _cu, _vp]),
+    "laga_fwd_varlen_workspace_bytes": (_sz, [_ci] * 7),
+    "laga_bwd_varlen_workspace_bytes": (_sz, [_ci] * 7 + [_cu]),
+    "laga_fwd_varlen": (_ci, [_vp] * 4 + [ctypes.POINTER(_ci)] + [_ci] * 7 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
+    "laga_bwd_varlen": (_ci, [_vp] * 7 + [ctypes.POINTER(_ci)] + [_ci] * 7 + [_cf, _ci] + [_vp] * 4 + [_vp, _sz, _cu, _vp]),
     "laga_absorbed_fwd_workspace_bytes": (_sz, [_ci] * 6),
     "laga_absorbed_fwd": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
     "laga_up_project": (_ci, [_vp, _vp] + [_ci] * 5 + [_vp, _vp, _vp]),
@@ -139,6 +143,22 @@ def bwd_workspace_bytes(S, h, d_c=512, d_nope=128, d_rope=64, d_v=128, flags=0) 
     return int(lib().laga_bwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v, flags))
 
 
+def fwd_varlen_workspace_bytes(S_total, n_seqs, h, d_c=512, d_nope=128, d_rope=64, d_v=128) -> int:
+    return int(lib().laga_fwd_varlen_workspace_bytes(S_total, n_seqs, h, d_c, d_nope, d_rope, d_v))
+
+
+def bwd_varlen_workspace_bytes(S_total, n_seqs, h, d_c=512, d_nope=128, d_rope=64, d_v=128, flags=0) -> int:
+    return int(lib().laga_bwd_varlen_workspace_bytes(S_total, n_seqs, h, d_c, d_nope, d_rope, d_v, flags))
+
+
+def _cu_seqlens(cu_seqlens):
+    """The host array laga_*_varlen takes: n_seqs + 1 C ints from a list or a CPU tensor."""
+    values = [int(v) for v in (cu_seqlens.tolist() if isinstance(cu_seqlens, torch.Tensor) else cu_seqlens)]
+    if len(values) < 2:
+        raise ValueError("cu_seqlens needs at least two entries (one sequence)")
+    return (ctypes.c_int * len(values))(*values), len(values) - 1
+
+
 def alloc_workspace(n_bytes: int, device="cuda") -> torch.Tensor:
     """A 1024-byte aligned byte buffer (torch's caching allocator aligns to at least 512; over-allocate)."""
     buf = torch.empty(n_bytes + 1024, dtype=torch.uint8, device=device)
@@ -147,8 +167,9 @@ def alloc_workspace(n_bytes: int, device="cuda") -> torch.Tensor:
 
 
 def fwd(q, c_kv, k_pe, w_kv_b, d_v=128, softmax_scale=None, causal=True, out=None, lse=None, workspace=None,
-        stream=None):
-    """laga_fwd: returns (out bf16 [S,h,d_v], lse fp32 [S,h], workspace).  Enqueues only."""
+        stream=None, cu_seqlens=None):
+    """laga_fwd: returns (out bf16 [S,h,d_v], lse fp32 [S,h], workspace).  Enqueues only.
+    With cu_seqlens (list or CPU tensor, n_seqs + 1 entries): laga_fwd_varlen over packed sequences."""
     S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
     dev = same_device(q, c_kv, k_pe, w_kv_b, out, lse, workspace)
     if softmax_scale is None:
@@ -159,16 +180,23 @@ def fwd(q, c_kv, k_pe, w_kv_b, d_v=128, softmax_scale=None, causal=True, out=Non
         lse = torch.empty(S, h, dtype=torch.float32, device=dev)
     _dev(out, torch.bfloat16, (S, h, d_v), "out")
     _dev(lse, torch.float32, (S, h), "lse")
-    need = fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v)
+    cu, n_seqs = _cu_seqlens(cu_seqlens) if cu_seqlens is not None else (None, 0)
+    need = (fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v) if cu is None else
+            fwd_varlen_workspace_bytes(S, n_seqs, h, d_c, d_nope, d_rope, d_v))
     if need == 0:
         raise LagaError(ERR_UNSUPPORTED, "laga_fwd_workspace_bytes")
     if workspace is None:
         workspace = alloc_workspace(need, dev)
     with _on(dev):
-        rc = lib().laga_fwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope, d_v,
-                            float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse), _ptr(workspace),
-                            workspace.numel(), 0, _stream(stream, dev))
-    _check(rc, "laga_fwd")
+        if cu is None:
+            rc = lib().laga_fwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), S, h, d_c, d_nope, d_rope, d_v,
+                                float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse), _ptr(workspace),
+                                workspace.numel(), 0, _stream(stream, dev))
+        else:
+            rc = lib().laga_fwd_varlen(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), cu, n_seqs, S, h, d_c, d_nope,
+                                       d_rope, d_v, float(softmax_scale), int(bool(causal)), _ptr(out), _ptr(lse),
+                                       _ptr(workspace), workspace.numel(), 0, _stream(stream, dev))
+    _check(rc, "laga_fwd" if cu is None else "laga_fwd_varlen")
     return out, lse, workspace
 
 
@@ -227,8 +255,9 @@ def fwd_builtin_scratch(q, c_kv, k_pe, w_kv_b, out, lse, d_v=128, softmax_scale=
 
 
 def bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout, d_v=128, softmax_scale=None, causal=True, dq=None, dc_kv=None,
-        dk_pe=None, dw_kv_b=None, workspace=None, flags=0, stream=None):
-    """laga_bwd: returns (dq, dc_kv, dk_pe, dw_kv_b, workspace).  Enqueues only."""
+        dk_pe=None, dw_kv_b=None, workspace=None, flags=0, stream=None, cu_seqlens=None):
+    """laga_bwd: returns (dq, dc_kv, dk_pe, dw_kv_b, workspace).  Enqueues only.
+    With cu_seqlens (list or CPU tensor, n_seqs + 1 entries): laga_bwd_varlen over packed sequences."""
     S, h, d_c, d_nope, d_rope = _geometry(q, c_kv, k_pe, w_kv_b, d_v)
     dev = same_device(q, c_kv, k_pe, w_kv_b, out, lse, dout, dq, dc_kv, dk_pe, dw_kv_b, workspace)
     if softmax_scale is None:
@@ -244,17 +273,25 @@ def bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout, d_v=128, softmax_scale=None, caus
             raise ValueError("LAGA_FLAG_ACCUM_DW needs an existing dw_kv_b to add into")
         dw_kv_b = torch.empty(w_kv_b.shape, dtype=torch.float32, device=dev)
     _dev(dw_kv_b, torch.float32, w_kv_b.shape, "dw_kv_b")
-    need = bwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v, flags)
+    cu, n_seqs = _cu_seqlens(cu_seqlens) if cu_seqlens is not None else (None, 0)
+    need = (bwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v, flags) if cu is None else
+            bwd_varlen_workspace_bytes(S, n_seqs, h, d_c, d_nope, d_rope, d_v, flags))
     if need == 0:
         raise LagaError(ERR_UNSUPPORTED, "laga_bwd_workspace_bytes")
     if workspace is None:
         workspace = alloc_workspace(need, dev)
     with _on(dev):
-        rc = lib().laga_bwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), _ptr(out), _ptr(lse), _ptr(dout), S, h,
-                            d_c, d_nope, d_rope, d_v, float(softmax_scale), int(bool(causal)), _ptr(dq), _ptr(dc_kv),
-                            _ptr(dk_pe), _ptr(dw_kv_b), _ptr(workspace), workspace.numel(), flags,
-                            _stream(stream, dev))
-    _check(rc, "laga_bwd")
+        if cu is None:
+            rc = lib().laga_bwd(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), _ptr(out), _ptr(lse), _ptr(dout), S, h,
+                                d_c, d_nope, d_rope, d_v, float(softmax_scale), int(bool(causal)), _ptr(dq), _ptr(dc_kv),
+                                _ptr(dk_pe), _ptr(dw_kv_b), _ptr(workspace), workspace.numel(), flags,
+                                _stream(stream, dev))
+        else:
+            rc = lib().laga_bwd_varlen(_ptr(q), _ptr(c_kv), _ptr(k_pe), _ptr(w_kv_b), _ptr(out), _ptr(lse), _ptr(dout),
+                                       cu, n_seqs, S, h, d_c, d_nope, d_rope, d_v, float(softmax_scale),
+                                       int(bool(causal)), _ptr(dq), _ptr(dc_kv), _ptr(dk_pe), _ptr(dw_kv_b),
+                                       _ptr(workspace), workspace.numel(), flags, _stream(stream, dev))
+    _check(rc, "laga_bwd" if cu is None else "laga_bwd_varlen")
     return dq, dc_kv, dk_pe, dw_kv_b, workspace
 
 

@@ -116,6 +116,39 @@ def test_argument_validation_happens_before_any_device_work(laga):
     assert lib.laga_query_status(None, None, None) == laga.ERR_INVALID_ARG
 
 
+def test_varlen_entry_points_validate_cu_seqlens_before_any_device_work(laga):
+    lib = laga.lib()
+    p = ctypes.c_void_p
+    good = p(1024)
+
+    def cu(*v):
+        return (ctypes.c_int * len(v))(*v)
+
+    def fwd(cu_seqlens, n_seqs, S_total=256, ws_bytes=1 << 40):
+        return lib.laga_fwd_varlen(good, good, good, good, cu_seqlens, n_seqs, S_total, 2, 512, 128, 64, 128, 0.07, 1,
+                                   good, good, good, ws_bytes, 0, None)
+
+    def bwd(cu_seqlens, n_seqs, S_total=256, flags=0, ws_bytes=1 << 40):
+        return lib.laga_bwd_varlen(good, good, good, good, good, good, good, cu_seqlens, n_seqs, S_total, 2, 512, 128,
+                                   64, 128, 0.07, 1, good, good, good, good, good, ws_bytes, flags, None)
+
+    for call in (fwd, bwd):
+        assert call(None, 2) == laga.ERR_INVALID_ARG
+        assert call(cu(0, 100, 256), 0) == laga.ERR_INVALID_ARG          # no sequence
+        assert call(cu(1, 100, 256), 2) == laga.ERR_INVALID_ARG          # does not start at 0
+        assert call(cu(0, 100, 255), 2) == laga.ERR_INVALID_ARG          # does not end at S_total
+        assert call(cu(0, 200, 100, 256), 3) == laga.ERR_INVALID_ARG     # decreasing
+        assert call(cu(0, 100, 256), 2, ws_bytes=4096) == laga.ERR_WORKSPACE_TOO_SMALL
+    assert bwd(cu(0, 100, 256), 2, flags=laga.FLAG_FUSED_BWD) == laga.ERR_INVALID_ARG
+    # sizes: the single-sequence figure plus the tile tables, whatever the lengths are
+    S, n, h = 5000, 7, 4
+    assert laga.fwd_varlen_workspace_bytes(S, n, h) >= laga.fwd_workspace_bytes(S, h) + 32 * (S // 128 + n)
+    assert laga.fwd_varlen_workspace_bytes(S, n, h) <= laga.fwd_workspace_bytes(S, h) + 32 * (S // 128 + n) + 8 * n + 2048
+    assert laga.bwd_varlen_workspace_bytes(S, n, h) >= laga.bwd_workspace_bytes(S, h) + 2 * h * 127 * n * 4
+    assert laga.bwd_varlen_workspace_bytes(S, n, h, flags=laga.FLAG_FUSED_BWD) == 0
+    assert laga.fwd_varlen_workspace_bytes(S, 0, h) == 0 and laga.bwd_varlen_workspace_bytes(S, 0, h) == 0
+
+
 def test_binding_rejects_cpu_tensors(laga):
     import torch
     q = torch.zeros(128, 2, 192, dtype=torch.bfloat16)
