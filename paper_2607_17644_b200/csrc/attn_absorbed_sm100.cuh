@@ -93,13 +93,15 @@ attn_absorbed_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_qabs, co
         tma_prefetch_desc(&tmap_qabs); tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_ckv); tma_prefetch_desc(&tmap_kpe);
         if ((smem_u32(smem) & 1023u) != 0u) {   // the swizzled operand slabs need a 1024-byte aligned base
             abort_flag->value = 1;
-            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD3u);
         }
     }
     if (warp == 5) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    grid_launch_dependents();
+    grid_dependency_wait();          // global memory from here on
+    if (threadIdx.x == 0 && abort_flag->value != 0u) atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD3u);   // set-up found the shared memory misaligned
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_s = tmem_base + 256;
     const uint32_t tmem_q = tmem_base + 384;

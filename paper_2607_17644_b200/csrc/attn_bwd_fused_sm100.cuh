@@ -138,15 +138,17 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
         if ((smem_u32(smem) & 1023u) != 0u) {   // the swizzled operand slabs need a 1024-byte aligned base
             abort_flag->value = 1;
-            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD2u);
         }
     }
-    clock_probe_begin(args.clock_probe);
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     cluster_sync();                      // the peer's barriers are initialised before anything arrives on them
     tc_fence_after_sync();
+    grid_launch_dependents();
+    grid_dependency_wait();              // global memory from here on
+    if (threadIdx.x == 0 && abort_flag->value != 0u) atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD2u);   // set-up found the shared memory misaligned
+    clock_probe_begin(args.clock_probe);
     const uint32_t tmem_base = *tmem_slot;
 
     auto tile_at = [&](int n) -> FusedTile {
@@ -614,6 +616,8 @@ attn_bwd_fused_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
 __global__ void __launch_bounds__(256)
 bwd_dq_convert_kernel(float* __restrict__ dq_acc, int S, int h, int head_begin, int head_count, float scale,
                       __nv_bfloat16* __restrict__ dq) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const size_t idx = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 8;   // 8 channels per thread
     const size_t row_elems = static_cast<size_t>(head_count) * 192;
     if (idx >= static_cast<size_t>(S) * row_elems) return;

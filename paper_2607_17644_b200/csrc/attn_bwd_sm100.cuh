@@ -46,6 +46,8 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __r
                  const float* __restrict__ lse, int S, int h, int S_pad, float* __restrict__ stat_l2,
                  float* __restrict__ stat_delta, float4* __restrict__ zero_begin, size_t zero_count,
                  const int2* __restrict__ seqs, int n_seqs) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     // Also clears the fp32 buffer the dK/dV kernel accumulates the rope-column key gradients into
     // (zero_count float4 elements): one launch less than a separate memset.
     for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < zero_count;
@@ -98,6 +100,8 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __r
 // head's columns into an fp32 accumulator with atomics; this kernel rounds the sums to bf16.
 __global__ void __launch_bounds__(256)
 bwd_dkpe_convert_kernel(const float* __restrict__ dkpe_acc, int S, __nv_bfloat16* __restrict__ dk_pe) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const size_t idx = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
     if (idx >= static_cast<size_t>(S) * 64) return;
     const float4 v = *reinterpret_cast<const float4*>(dkpe_acc + idx);
@@ -110,6 +114,8 @@ bwd_dkpe_convert_kernel(const float* __restrict__ dkpe_acc, int S, __nv_bfloat16
 // Deterministic alternative to the atomics: sum the per-head buffers in head order.
 __global__ void __launch_bounds__(256)
 bwd_dkpe_reduce_kernel(const float* __restrict__ dk_rope, int S, int h, __nv_bfloat16* __restrict__ dk_pe) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const size_t n = static_cast<size_t>(S) * 64;
     if (idx >= n) return;
@@ -206,14 +212,16 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
         if ((smem_u32(smem) & 1023u) != 0u) {   // the swizzled operand slabs need a 1024-byte aligned base
             abort_flag->value = 1;
-            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD0u);
         }
     }
-    clock_probe_begin(args.clock_probe);
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    grid_launch_dependents();
+    grid_dependency_wait();          // set-up above overlaps the previous kernel's tail; global memory from here on
+    if (threadIdx.x == 0 && abort_flag->value != 0u) atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD0u);   // set-up found the shared memory misaligned
+    clock_probe_begin(args.clock_probe);
     const uint32_t tmem_base = *tmem_slot;
     // columns: [0,128) X | [128,192) Y | [192,384) dK | [384,512) dV
     const uint32_t tmem_y = tmem_base + 128;
@@ -587,14 +595,16 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
         if ((smem_u32(smem) & 1023u) != 0u) {
             abort_flag->value = 1;
-            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD1u);
         }
     }
-    clock_probe_begin(args.clock_probe);
     if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    grid_launch_dependents();
+    grid_dependency_wait();          // set-up above overlaps the previous kernel's tail; global memory from here on
+    if (threadIdx.x == 0 && abort_flag->value != 0u) atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD1u);   // set-up found the shared memory misaligned
+    clock_probe_begin(args.clock_probe);
     const uint32_t tmem_base = *tmem_slot;
     // columns: [0,128) S | [128,256) dP, then dS as bf16 (keys 0..63 in [128,160), 64..127 in [192,224)) |
     //          [256,320) dO as bf16 | [320,512) dQ

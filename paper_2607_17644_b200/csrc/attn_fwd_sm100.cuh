@@ -125,14 +125,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
         tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
         if ((smem_u32(smem) & 1023u) != 0u) {   // the swizzled operand slabs need a 1024-byte aligned base
             abort_flag->value = 1;
-            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD2u);
         }
     }
-    clock_probe_begin(args.clock_probe);
     if (warp == 9) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    grid_launch_dependents();
+    grid_dependency_wait();          // set-up above overlaps the previous kernel's tail; global memory from here on
+    if (threadIdx.x == 0 && abort_flag->value != 0u) atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD2u);   // set-up found the shared memory misaligned
+    clock_probe_begin(args.clock_probe);
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base + 3 * BK;       // [0,288) three S tiles | [288,416) O | [416,512) Q as packed bf16
     const uint32_t tmem_q = tmem_o + 128;

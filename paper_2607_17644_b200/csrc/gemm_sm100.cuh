@@ -78,12 +78,14 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tma_prefetch_desc(&tmap_b);
     }
     if (warp == 1) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
-    for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < args.zero_count;
-         z += static_cast<size_t>(gridDim.x) * blockDim.x)
-        args.zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    grid_launch_dependents();
+    grid_dependency_wait();          // global memory from here on
+    for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < args.zero_count;
+         z += static_cast<size_t>(gridDim.x) * blockDim.x)
+        args.zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
     const uint32_t tmem_base = *tmem_slot;
 
     auto k_range = [&](int split, int& kt_begin, int& n_kt) {
@@ -280,17 +282,19 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         tma_prefetch_desc(&tmap_b);
         if ((smem_u32(smem) & 1023u) != 0u) {
             abort_flag->value = 1;
-            atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD4u);
         }
     }
     if (warp == 1) { tmem_alloc_pair(tmem_slot, kTmemCols); tmem_relinquish_pair(); }
-    for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < args.zero_count;
-         z += static_cast<size_t>(gridDim.x) * blockDim.x)
-        args.zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
     tc_fence_before_sync();
     __syncthreads();
     cluster_sync();            // the peer's barriers exist before anything can arrive on them
     tc_fence_after_sync();
+    grid_launch_dependents();
+    grid_dependency_wait();    // global memory from here on
+    if (threadIdx.x == 0 && abort_flag->value != 0u) atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD4u);   // set-up found the shared memory misaligned
+    for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < args.zero_count;
+         z += static_cast<size_t>(gridDim.x) * blockDim.x)
+        args.zero_begin[z] = make_float4(0.f, 0.f, 0.f, 0.f);
     const uint32_t tmem_base = *tmem_slot;
     const bool run = abort_flag->value == 0u;   // (the layout is the same in both CTAs: they agree)
 

@@ -109,6 +109,7 @@ void init_device(DeviceInfo* info, int dev) {
     using G = GemmPairSmem<256, kGemmStages>;
     bool ok = allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, false, true, EPI_BF16>, G::kTotalBytes) &&
               allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, false, false, EPI_BF16>, G::kTotalBytes) &&
+              allow_smem(gemm_pair_sm100_kernel<128, kGemmStages, false, false, EPI_BF16>, GemmPairSmem<128, kGemmStages>::kTotalBytes) &&
               allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, true, true, EPI_ATOMIC_F32>, G::kTotalBytes) &&
               allow_smem(gemm_sm100_kernel<128, 4, false, true, EPI_BF16>, GemmSmem<128, 4>::kTotalBytes) &&
               allow_smem(attn_absorbed_fwd_sm100_kernel<true>, AttnAbsorbedSmem::kTotalBytes) &&
@@ -236,6 +237,29 @@ bool cached_tmap_bf16(CUtensorMap* map, const void* base, uint64_t inner_elems, 
     return true;
 }
 
+// ---- launches ----------------------------------------------------------------------------------------
+// Every kernel is launched through here.  `overlap` asks for programmatic dependent launch: the kernel may be
+// scheduled while the kernel enqueued just before it on the stream is still running, and runs its set-up
+// there; its threads then wait (griddepcontrol.wait, which every kernel of the library executes first thing
+// after set-up) until that kernel has completed.  Only launches that directly follow another launch of the
+// same entry point ask for it: the first kernel after a memset, a copy or the caller's own work is launched
+// the ordinary way.
+template <typename... Params, typename... Args>
+void launch_kernel(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem_bytes, cudaStream_t stream, bool overlap,
+                   Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = overlap ? &attr : nullptr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);   // the caller reads cudaGetLastError
+}
+
 // ---- measurement aid (laga_profile_kernel) ---------------------------------------------------------
 // Caller-provided CUDA events recorded around launches of one kernel, cycling through the registered pairs.
 struct ProfileSlot {
@@ -275,7 +299,7 @@ WorkSchedule make_schedule(int n_tiles, int S, int h, unsigned* counter, const i
 
 // ---- Algorithm 1 step 4: KV[S, N] = c_kv[S, d_c] . W[d_c, N] ------------------------------------
 int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, bool overlap = false) {
     constexpr int BN = 256, STAGES = kGemmStages;
     auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
     using L = GemmPairSmem<BN, STAGES>;
@@ -286,7 +310,7 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
     if (!cached_tmap_bf16(&tc, kv, N, S, static_cast<uint64_t>(N) * 2, 32)) return LAGA_ERR_CUDA;
     GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status, nullptr, 0, 1, 0, 0, 0};
     dim3 grid(pair_grid((N / BN) * ((S + 255) / 256)), 1, 1);
-    { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, tc, a); }
+    { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); launch_kernel(kernel, grid, dim3(192), L::kTotalBytes, stream, overlap, ta, tb, tc, a); }
     return launch_status();
 }
 
@@ -294,9 +318,10 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
 // dc_kv[S, d_c] = dKV[S, N] . W^T          (A = dKV K-major, B = W rows d_c / inner N: K-major)
 // `clear` (optional) is an fp32 buffer of clear_floats elements this launch zeroes on its way in: the dW
 // GEMM that follows accumulates into it with atomics.
-int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float* clear, size_t clear_floats,
-                unsigned* status, cudaStream_t stream) {
-    constexpr int BN = 256, STAGES = kGemmStages;
+template <int BN>
+int launch_dckv_bn(const void* dkv, const void* w, int S, int N, void* dc_kv, float* clear, size_t clear_floats,
+                   unsigned* status, cudaStream_t stream, bool overlap) {
+    constexpr int STAGES = kGemmStages;
     auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
     using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
@@ -306,39 +331,53 @@ int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float
     if (!cached_tmap_bf16(&tc, dc_kv, kDc, S, kDc * 2, 32)) return LAGA_ERR_CUDA;
     GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status, reinterpret_cast<float4*>(clear), clear_floats / 4, 1, 0, 0, 0};
     dim3 grid(pair_grid((kDc / BN) * ((S + 255) / 256)), 1, 1);
-    { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, tc, a); }
+    { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); launch_kernel(kernel, grid, dim3(192), L::kTotalBytes, stream, overlap, ta, tb, tc, a); }
     return launch_status();
+}
+int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float* clear, size_t clear_floats,
+                unsigned* status, cudaStream_t stream, bool overlap = false) {
+    // The output is only d_c = 512 columns wide: with 256-column tiles a short sequence leaves most CTA pairs
+    // without a tile (S = 4096: 32 tiles for 74 pairs).  Narrower tiles double the count at the price of
+    // reading the dKV rows once more from L2.
+    const int tiles_256 = (kDc / 256) * ((S + 255) / 256);
+    if (tiles_256 < sm_count() / 2)
+        return launch_dckv_bn<128>(dkv, w, S, N, dc_kv, clear, clear_floats, status, stream, overlap);
+    return launch_dckv_bn<256>(dkv, w, S, N, dc_kv, clear, clear_floats, status, stream, overlap);
 }
 
 // dW[d_c, N] += c_kv^T . dKV   (both operands read with the token index as K: MN-major), split over
 // the sequence with fp32 atomic accumulation into a buffer the caller of this function has cleared
 // (launch_dckv does it) or wants added to.
 int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool deterministic,
-              unsigned* status, cudaStream_t stream) {
+              unsigned* status, cudaStream_t stream, bool overlap = false) {
     constexpr int BN = 256, STAGES = kGemmStages;
     auto kernel = gemm_pair_sm100_kernel<BN, STAGES, true, true, EPI_ATOMIC_F32>;
     using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 64)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tb, dkv, N, S, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;
-    // Split the sequence so that tiles x splits fills whole waves of the persistent grid: the smallest
-    // split count (fewest atomics) whose last wave is at least 90 % full, else the best found.
+    // Split the sequence to fill the persistent grid, but every split adds one fp32 atomic pass over the whole
+    // [d_c, N] output.  Measured on B200: the atomics of one pass move at about 4.2 TB/s and the tiles run at
+    // about 1.3 PFLOP/s times the fill of the last wave, so pick the split count that minimises
+    //     flops / (1.3e15 * fill(s)) + s * output bytes / 4.2e12
+    // (S = 4096, h = 16: 2 splits, 25 us, where filling the grid to 97 % with 9 splits took 39 us).
     const int tiles = (kDc / 256) * (N / BN);
     const int k_tiles = (S + 63) / 64;
     const int sms = sm_count() / 2;       // CTA pairs
     int splits = 1;
-    double best = 0.0;
+    double best = 1e30;
+    const double flops = 2.0 * S * kDc * N, out_bytes = static_cast<double>(kDc) * N * sizeof(float);
     for (int s = 1; s <= 16 && s <= k_tiles && !deterministic; ++s) {   // one split: one add per element
         const int total = tiles * s;
-        const double eff = static_cast<double>(total) / (static_cast<double>((total + sms - 1) / sms) * sms);
-        if (eff > best + 1e-9) { best = eff; splits = s; }
-        if (eff >= 0.9) { splits = s; break; }
+        const double fill = static_cast<double>(total) / (static_cast<double>((total + sms - 1) / sms) * sms);
+        const double cost = flops / (1.3e15 * fill) + s * out_bytes / 4.2e12;
+        if (cost < best) { best = cost; splits = s; }
     }
     const int per_split = (k_tiles + splits - 1) / splits;
     splits = (k_tiles + per_split - 1) / per_split;
     GemmArgs a{kDc, N, S, per_split, splits, dw, N, status, nullptr, 0, 1, 0, 0, 0};
     dim3 grid(pair_grid(tiles * splits), 1, 1);
-    { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); kernel<<<grid, 192, L::kTotalBytes, stream>>>(ta, tb, ta, a); }   // (fp32 atomic epilogue: the output map is unused)
+    { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); launch_kernel(kernel, grid, dim3(192), L::kTotalBytes, stream, overlap, ta, tb, ta, a); }   // (fp32 atomic epilogue: the output map is unused)
     return launch_status();
 }
 
@@ -411,7 +450,7 @@ int upload_seq_plan(const SeqPlan& plan, void* tables, cudaStream_t stream) {
 // ---- Algorithm 1 step 5 -------------------------------------------------------------------------
 int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int h, float softmax_scale,
                     int causal, void* out, float* lse, unsigned* status, cudaStream_t stream,
-                    const int4* q_tiles = nullptr, int n_seq_tiles = 0) {
+                    const int4* q_tiles = nullptr, int n_seq_tiles = 0, bool overlap = false) {
     using L = AttnFwdSmem;
     const int N = h * (kDn + kDv);
     CUtensorMap tkv, tpe;   // boxes of 64 columns x one key tile of rows
@@ -423,8 +462,8 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
                   make_schedule(n_tiles, S, h, slot_counter(status, kSlotFwd), q_tiles), slot_probe(status, kSlotFwd)};
     dim3 grid(persistent_grid(n_tiles * h), 1, 1);
     ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream);
-    if (causal) attn_fwd_sm100_kernel<true><<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a);
-    else attn_fwd_sm100_kernel<false><<<grid, kFwdThreads, L::kTotalBytes, stream>>>(tkv, tpe, a);
+    launch_kernel(causal ? attn_fwd_sm100_kernel<true> : attn_fwd_sm100_kernel<false>, grid, dim3(kFwdThreads), L::kTotalBytes,
+                  stream, overlap, tkv, tpe, a);
     return launch_status();
 }
 
@@ -476,17 +515,16 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
                     void* dk_pe, float* stat_l2, float* stat_delta, float* dkpe_acc, float* dk_rope_per_head, int S_pad,
                     float* dq_acc, int head_window, unsigned* status, cudaStream_t stream,
                     const int4* q_tiles = nullptr, const int4* k_tiles = nullptr, const int2* seqs = nullptr,
-                    int n_seqs = 0, int n_seq_tiles = 0) {
+                    int n_seqs = 0, int n_seq_tiles = 0, bool overlap = false) {
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
     {   // delta and the transposed, padded softmax statistics; clears the rope-gradient accumulator on the way
         const long long items = static_cast<long long>(S_pad) * h;   // eight lanes per (row, head)
         const unsigned blocks = static_cast<unsigned>((items * 8 + 255) / 256);
         ScopedKernelEvents ev(LAGA_KERNEL_BWD_DELTA, stream);
-        bwd_delta_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(out),
-                                                     reinterpret_cast<const __nv_bfloat16*>(dout), lse, S, h, S_pad,
-                                                     stat_l2, stat_delta, reinterpret_cast<float4*>(dkpe_acc),
-                                                     static_cast<size_t>(S) * kDr / 4, seqs, n_seqs);
+        launch_kernel(bwd_delta_kernel, dim3(blocks), dim3(256), 0, stream, overlap, reinterpret_cast<const __nv_bfloat16*>(out),
+                      reinterpret_cast<const __nv_bfloat16*>(dout), lse, S, h, S_pad, stat_l2, stat_delta,
+                      reinterpret_cast<float4*>(dkpe_acc), static_cast<size_t>(S) * kDr / 4, seqs, n_seqs);
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
     }
     const uint64_t q_row = static_cast<uint64_t>(h) * 192, do_row = static_cast<uint64_t>(h) * 128;
@@ -532,14 +570,14 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
                         make_schedule(n_tiles, S, h, slot_counter(status, kSlotDq), q_tiles), slot_probe(status, kSlotDq)};
         {
             ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream);
-            if (causal) attn_bwd_dkv_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
-            else attn_bwd_dkv_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDkvSmem::kTotalBytes, stream>>>(tq, tdo, tkv, tpe, a);
+            launch_kernel(causal ? attn_bwd_dkv_sm100_kernel<true> : attn_bwd_dkv_sm100_kernel<false>, grid, dim3(kBwdThreads),
+                          AttnBwdDkvSmem::kTotalBytes, stream, true, tq, tdo, tkv, tpe, a);
         }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
         {
             ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream);
-            if (causal) attn_bwd_dq_sm100_kernel<true><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
-            else attn_bwd_dq_sm100_kernel<false><<<grid, kBwdThreads, AttnBwdDqSmem::kTotalBytes, stream>>>(tq, tkv, tpe, b);
+            launch_kernel(causal ? attn_bwd_dq_sm100_kernel<true> : attn_bwd_dq_sm100_kernel<false>, grid, dim3(kBwdThreads),
+                          AttnBwdDqSmem::kTotalBytes, stream, true, tq, tkv, tpe, b);
         }
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
@@ -547,12 +585,12 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         ScopedKernelEvents ev(LAGA_KERNEL_DKPE_REDUCE, stream);
         if (dk_rope_per_head != nullptr) {
             const size_t n = static_cast<size_t>(S) * kDr;
-            bwd_dkpe_reduce_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
-                dk_rope_per_head, S, h, reinterpret_cast<__nv_bfloat16*>(dk_pe));
+            launch_kernel(bwd_dkpe_reduce_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream, true,
+                          dk_rope_per_head, S, h, reinterpret_cast<__nv_bfloat16*>(dk_pe));
         } else {
             const size_t n = static_cast<size_t>(S) * kDr / 4;
-            bwd_dkpe_convert_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(
-                dkpe_acc, S, reinterpret_cast<__nv_bfloat16*>(dk_pe));
+            launch_kernel(bwd_dkpe_convert_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream, true,
+                          dkpe_acc, S, reinterpret_cast<__nv_bfloat16*>(dk_pe));
         }
     }
     return launch_status();
@@ -735,7 +773,7 @@ static int fwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
     }
     // step 4 is token-wise: one GEMM over all the packed tokens
     if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
-    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st, q_tiles, plan.n_tiles);
+    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st, q_tiles, plan.n_tiles, true);
 }
 
 int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, int S, int h, int d_c,
@@ -819,13 +857,13 @@ static int bwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
                               reinterpret_cast<float*>(base + w.dkpe_acc),
                               deterministic ? reinterpret_cast<float*>(base + w.dk_rope_per_head) : nullptr, w.S_pad,
                               reinterpret_cast<float*>(base + w.dq_acc), w.head_window, status, st, q_tiles, k_tiles, seqs,
-                              plan.n_seqs, plan.n_tiles)) != LAGA_OK)
+                              plan.n_seqs, plan.n_tiles, /*overlap=*/!(flags & LAGA_FLAG_KV_SAVED))) != LAGA_OK)
         return rc;
     // the two GEMMs of Section 5.2 are token-wise: one launch each over all the packed tokens
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,
-                          accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st)) != LAGA_OK)
+                          accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st, true)) != LAGA_OK)
         return rc;
-    return launch_dw(c_kv, dkv, S, N, dw_kv_b, deterministic, status, st);
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, deterministic, status, st, true);
 }
 
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
@@ -898,7 +936,7 @@ int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, 
     // reads them.
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
     if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
-    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st);
+    return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st, nullptr, 0, true);
 }
 
 size_t laga_absorbed_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v) {

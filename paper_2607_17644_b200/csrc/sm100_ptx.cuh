@@ -155,6 +155,17 @@ struct ArmedBarriers {
 };
 
 // ------------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  A kernel launched with the programmatic-stream-serialization attribute may
+// start while the kernel before it in the stream is still running: its CTAs take SMs as they free up and run
+// their set-up (barrier init, TMEM allocation, descriptor prefetch), then every thread waits here until the
+// preceding grid has completed and its memory is visible.  NOTHING global may be read or written before the
+// wait.  Every kernel of the library executes both calls, so completion is transitive along a chain of
+// launches; without the launch attribute they return at once.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------------
 // TMA (tiled bulk tensor copies global -> shared, completion on an mbarrier)
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
