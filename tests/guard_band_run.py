@@ -91,10 +91,53 @@ def run_case(S, h, causal):
     assert float((lse_a.double().cpu() - ref["lse"]).abs().max()) <= 5e-3
 
 
+def run_packed_case(lengths, h, causal):
+    """The packed variable-length entry points between guard bands, against the oracle sequence by sequence."""
+    cu = [0]
+    for n in lengths:
+        cu.append(cu[-1] + n)
+    S = cu[-1]
+    sh = LagaShape(S=S, h=h)
+    tensors = make_inputs(sh, 950 + S + h)
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in tensors)
+    bf, f32 = torch.bfloat16, torch.float32
+    ws_sizes = [laga.fwd_varlen_workspace_bytes(S, len(lengths), h), laga.bwd_varlen_workspace_bytes(S, len(lengths), h)]
+    arena = Arena(sum(ws_sizes) + 8 * S * h * 192 * 4 + 32 * GUARD + 512 * h * 256 * 4 + (1 << 20))
+    out = arena.take(S * h * 128 * 2, bf, (S, h, 128))
+    lse = arena.take(S * h * 4, f32, (S, h))
+    dq = arena.take(S * h * 192 * 2, bf, (S, h, 192))
+    dc_kv = arena.take(S * 512 * 2, bf, (S, 512))
+    dk_pe = arena.take(S * 64 * 2, bf, (S, 64))
+    dw = arena.take(512 * h * 256 * 4, f32, (512, h * 256))
+    ws_f, ws_b = (arena.take(n) for n in ws_sizes)
+    laga.fwd(q, c_kv, k_pe, w, causal=causal, out=out, lse=lse, workspace=ws_f, cu_seqlens=cu)
+    laga.check_status(ws_f, where="laga_fwd_varlen")
+    laga.bwd(q, c_kv, k_pe, w, out, lse, dout, causal=causal, dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw_kv_b=dw, workspace=ws_b,
+             cu_seqlens=cu)
+    laga.check_status(ws_b, where="laga_bwd_varlen")
+    torch.cuda.synchronize()
+    assert arena.guards_intact(), f"a guard band was overwritten (packed {lengths}, h={h})"
+    dw_ref = torch.zeros(512, h * 256, dtype=torch.float64)
+    for a, b in zip(cu[:-1], cu[1:]):
+        if a == b:
+            continue
+        tq, tc, tk, tw, tdo = tensors
+        ref = oracle.bwd(tq[a:b], tc[a:b], tk[a:b], tw, tdo[a:b], sh.d_v, sh.softmax_scale, causal=causal,
+                         kv_round_bf16=True, return_fwd=True)
+        dw_ref += ref["dw"]
+        if b - a > 1:
+            for name, got in (("out", out), ("dq", dq), ("dc_kv", dc_kv), ("dk_pe", dk_pe)):
+                assert rel_l2(got[a:b], ref[name]) <= 5e-3, (name, a, b)
+        assert float((lse[a:b].double().cpu() - ref["lse"]).abs().max()) <= 1e-3
+    assert rel_l2(dw, dw_ref) <= 5e-3
+
+
 if __name__ == "__main__":
     laga.lib()
     expect_debug = os.environ.get("LAGA_DEBUG", "0") not in ("", "0")
     assert laga.DEBUG == expect_debug and laga.LIB_PATH.endswith("liblaga_debug.so" if expect_debug else "liblaga.so")
     for S, h, causal in ((300, 3, True), (1024, 4, True), (129, 2, False), (1, 1, True), (2500, 1, True)):
         run_case(S, h, causal)
+    for lengths, h, causal in (([300, 1, 140], 2, True), ([129, 0, 700], 1, False)):
+        run_packed_case(lengths, h, causal)
     print("GUARD_BANDS_OK", "checked build" if expect_debug else "normal build")
