@@ -363,6 +363,34 @@ def test_deterministic_flag_gives_bitwise_repeatable_gradients(laga, oracle):
     assert (dw2 - runs[0][3]).abs().max() <= 1e-4 * runs[0][3].abs().max()
 
 
+def test_back_to_back_calls_repeat_bit_for_bit(laga):
+    """The kernels of an entry point are chained by programmatic dependent launch: each starts its set-up while
+    the one before it drains and must not touch global memory before that one has completed.  Forty forward +
+    backward steps enqueued back to back on one stream, reusing the same workspaces and outputs, with ordered
+    reductions: a kernel that ran ahead of its producer (or overwrote what its predecessor still reads) would
+    show up as a step that differs from the first."""
+    sh = LagaShape(S=1536, h=4)
+    q, c_kv, k_pe, w, dout = (t.cuda() for t in make_inputs(sh, 77))
+    det = laga.FLAG_DETERMINISTIC
+    ws_f = laga.alloc_workspace(laga.fwd_workspace_bytes(sh.S, sh.h))
+    ws_b = laga.alloc_workspace(laga.bwd_workspace_bytes(sh.S, sh.h, flags=det))
+    out, lse = nan_like((sh.S, sh.h, 128), torch.bfloat16), nan_like((sh.S, sh.h), torch.float32)
+    grads = [nan_like(tuple(q.shape), torch.bfloat16), nan_like(tuple(c_kv.shape), torch.bfloat16),
+             nan_like(tuple(k_pe.shape), torch.bfloat16), nan_like(tuple(w.shape), torch.float32)]
+    snapshots = []
+    for _ in range(40):
+        laga.fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_f)
+        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, dq=grads[0], dc_kv=grads[1], dk_pe=grads[2], dw_kv_b=grads[3],
+                 workspace=ws_b, flags=det)
+        snapshots.append([t.clone() for t in (out, lse, *grads)])       # stream-ordered copies, no host sync
+    laga.check_status(ws_f)
+    laga.check_status(ws_b)
+    for step in snapshots[1:]:
+        for a, b in zip(snapshots[0], step):
+            assert torch.equal(a, b)
+    assert not any(torch.isnan(t.float()).any() for t in snapshots[0])
+
+
 def test_kv_saved_flag_reuses_the_forwards_up_projection(laga):
     """With LAGA_FLAG_KV_SAVED the backward reads K_nope/V where the forward left them in the shared
     workspace; with the deterministic flag on both sides the two backwards must agree bit for bit."""
