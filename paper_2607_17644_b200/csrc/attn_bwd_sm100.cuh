@@ -1,26 +1,30 @@
 // Backward of Algorithm 1 step 5 (Section 5.2: the chain rule through the softmax attention) for
-// the DeepSeek-V3 head geometry, as two tcgen05 kernels that recompute P from the saved LSE:
+// the DeepSeek-V3 head geometry, as two persistent tcgen05 kernels that recompute P from the saved LSE:
 //
-//   attn_bwd_dkv  one CTA per (128-key tile, head), sweeping the 64-row query tiles that attend to it:
-//                 S^T = K Q^T, dP^T = V dO^T, P^T = exp(scale S^T - LSE), dS^T = P^T (dP^T - delta),
-//                 dV += P^T dO, dK += dS^T Q  (dK 192 wide: 128 nope columns + 64 rope columns).
-//                 TMEM lanes are keys, so LSE and delta are per-column vectors staged in shared memory.
-//   attn_bwd_dq   one CTA per (128-query tile, head), sweeping 128-key tiles:
+//   attn_bwd_dkv  one (128-key tile, head) item at a time per CTA, sweeping the 128-row query tiles that
+//                 attend to it: S^T = K Q^T, dP^T = V dO^T, P^T = exp(scale S^T - LSE),
+//                 dS^T = P^T (dP^T - delta), dV += P^T dO, dK += dS^T Q (dK 192 wide: 128 nope columns +
+//                 64 rope columns).  TMEM lanes are keys, so LSE and delta are per-column vectors staged
+//                 in shared memory.
+//   attn_bwd_dq   one (128-query tile, head) item at a time per CTA, sweeping 128-key tiles:
 //                 S = Q K^T, dP = dO V^T, dS = P (dP - delta), dQ += dS K.  TMEM lanes are queries.
 //
 // Both read K_nope / V from the recomputed bf16 up-projection KV[S, h*256] and the shared rope band
-// from k_pe[S, 64]; both keep every accumulator in TMEM and never materialise S x S.
+// from k_pe[S, 64]; both keep every accumulator in TMEM and never materialise S x S.  With packed
+// variable-length sequences (work_sched.cuh: SeqTile) an item is a tile of one sequence and every index
+// below is relative to that sequence.
 //
 // Roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 and 6..9 two consumer
-// warpgroups (every thread owns one TMEM lane).  P^T / dS^T (dkv) and dS (dq) never touch shared
-// memory: the consumers write them back to TMEM as packed bf16 and the accumulating MMAs read their
-// A operand from there.  Scratch columns are reused by an MMA that the same thread issues after the
-// MMAs that read them; the tensor pipe runs one thread's MMAs in order, so that reuse needs no barrier.
-//   dkv: dK (192) + dV (128) leave 192 TMEM columns, so query tiles are 64 rows and the two groups
-//        take alternate tiles (scratch 2 x 64 columns + P^T 2 x 32): one group's exponentials overlap
-//        the other's MMAs.  A 64-wide N costs 48 cycles per MMA against 32 ideal.
-//   dq:  128-key tiles, all MMAs 128 wide; the two groups take 64 key columns each.  dO (the A
-//        operand of dP) lives in TMEM, which frees shared memory for a third K stage.
+// warpgroups (every thread owns one TMEM lane; the groups split a tile's 128 columns).  P^T / dS^T (dkv)
+// and dS (dq) never touch shared memory: the consumers write them back to TMEM as packed bf16 and the
+// accumulating MMAs read their A operand from there.  Scratch columns are reused by an MMA that the same
+// thread issues after the MMAs that read them; the tensor pipe runs one thread's MMAs in order, so that
+// reuse needs no barrier.
+//   dkv: dK (192) + dV (128) leave 192 TMEM columns: X (128, fp32: S^T then dP^T) and Y (64, bf16: P^T then
+//        dS^T) for ONE 128-wide tile, so that every MMA is at least 128 wide (a 64-wide N costs 48 cycles
+//        per MMA against 32 ideal and re-reads its A tile for half the work).
+//   dq:  128-key tiles, all MMAs 128 wide.  dO (the A operand of dP) lives in TMEM, which frees shared
+//        memory for a third K stage.
 #pragma once
 #include "attn_fwd_sm100.cuh"
 #include "sm100_ptx.cuh"
