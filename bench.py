@@ -371,11 +371,80 @@ def run_packed(args):
     print(json.dumps(line), flush=True)
 
 
+LINEAR_SHAPES = {
+    # name: (K, N) for M = 16384 tokens and a 16-head shard of DeepSeek-V3 (hidden 7168, q_lora 1536)
+    "W_kv_a (step 1: hidden -> latent + rope key)": (7168, 576),
+    "W_q_b (step 1: low-rank query -> 16 heads x 192)": (1536, 3072),
+    "W_kv_b (step 4: latent -> 16 heads x 256)": (512, 4096),
+    "W_o (step 7: 16 heads x 128 -> hidden)": (2048, 7168),
+}
+
+
+def run_linear(args):
+    """The dense projections around the path (Algorithm 1 steps 1, 4 and 7) through laga_linear /
+    laga_linear_backward on 16384 tokens, with the same products through torch.matmul (cuBLAS) beside them."""
+    from paper_2607_17644_b200 import laga
+    laga.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    M, K_steps, W = 16384, args.steps, max(args.warmup, 3)
+    g = torch.Generator().manual_seed(1234)
+
+    def timed(fn):
+        for _ in range(W):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(K_steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / K_steps
+
+    rows = {}
+    for name, (K, N) in LINEAR_SHAPES.items():
+        x = torch.randn(M, K, generator=g).to(torch.bfloat16).to(dev)
+        w = (torch.randn(K, N, generator=g) * K ** -0.5).to(torch.bfloat16).to(dev)
+        dy = torch.randn(M, N, generator=g).to(torch.bfloat16).to(dev)
+        y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+        dx = torch.empty(M, K, dtype=torch.bfloat16, device=dev)
+        dw = torch.empty(K, N, dtype=torch.float32, device=dev)
+        st = torch.zeros(1, dtype=torch.int32, device=dev)
+        fwd_ms = timed(lambda: laga.linear(x, w, y=y, status_word=st))
+        bwd_ms = timed(lambda: laga.linear_backward(dy, x, w, dx=dx, dw=dw, status_word=st))
+        assert laga.query_status(st)[0] == laga.OK
+        lib_fwd_ms = timed(lambda: torch.matmul(x, w, out=y))
+        wt = w.t().contiguous()
+
+        def lib_bwd():
+            torch.matmul(dy, wt, out=dx)
+            torch.matmul(x.t(), dy)
+
+        lib_bwd_ms = timed(lib_bwd)
+        fl = 2.0 * M * K * N
+        rows[name] = {"K": K, "N": N, "fwd_ms": fwd_ms, "fwd_tflops": fl / (fwd_ms * 1e-3) / 1e12,
+                      "bwd_ms": bwd_ms, "bwd_tflops": 2 * fl / (bwd_ms * 1e-3) / 1e12,
+                      "torch_matmul_fwd_ms": lib_fwd_ms, "torch_matmul_bwd_ms": lib_bwd_ms}
+        del x, w, dy, y, dx, dw, wt
+    head = rows["W_o (step 7: 16 heads x 128 -> hidden)"]
+    line = {"metric": "linear_projection_fwd_tflops", "value": head["fwd_tflops"], "unit": UNIT, "n_gpus": 1, "steps": K_steps,
+            "warmup": W, "ms_per_step": head["fwd_ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "linear: the dense projections of Algorithm 1 steps 1, 4 and 7 at 16384 tokens, 16-head shard "
+                                   "(headline of this line: W_o forward)",
+                       "l2_policy": "operands larger than L2 except W"},
+            "shapes": rows, "gpu_launches": K_steps}
+    print(json.dumps(line), flush=True)
+
+
 def run_cuda(args):
     from paper_2607_17644_b200 import laga
     laga.lib()
     if args.workload == "c4":
         return run_c4(args)
+    if args.workload == "linear":
+        return run_linear(args)
     if args.workload == "packed":
         return run_packed(args)
     world, rank, local_rank = dist_setup(args.gpus)
@@ -819,10 +888,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing and parity leg")
-    ap.add_argument("--workload", choices=sorted(CONFIGS) + ["packed"], default=WORKLOAD,
+    ap.add_argument("--workload", choices=sorted(CONFIGS) + ["packed", "linear"], default=WORKLOAD,
                     help="benchmark configuration (default c2, the headline; c4 = the absorbed form beside the LAGA "
                          "forward on c2's inputs; packed = batches / variable-length sequences through the varlen "
-                         "entry points; others are for profiling)")
+                         "entry points; linear = the dense projections of steps 1, 4 and 7; others are for profiling)")
     ap.add_argument("--compare-eager", action="store_true",
                     help="also time the explicit and absorbed forms in eager PyTorch (N=1; tens of GB at c2)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=16384,

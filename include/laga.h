@@ -153,6 +153,22 @@ int laga_bwd_varlen(const void* q, const void* c_kv, const void* k_pe, const voi
                     void* stream);
 
 /*
+ * The dense projections around the path (Algorithm 1 steps 1 and 7: W_q, W_kv_a, W_o), on the same CTA-pair
+ * tcgen05 GEMM that runs step 4.  All bf16, row-major, device pointers; fp32 accumulation.
+ *
+ * laga_linear:           y bf16 [M, N] = x [M, K] . w [K, N]
+ * laga_linear_backward:  dx bf16 [M, K] = dy [M, N] . w^T          written
+ *                        dw fp32 [K, N] (+)= x^T . dy               overwritten, or added to with LAGA_FLAG_ACCUM_DW;
+ *                        LAGA_FLAG_DETERMINISTIC as for laga_bwd (no split over M, one addition per element)
+ * M >= 1 is arbitrary; K and N must be multiples of 8 (row pitches of 16 bytes), anything else is
+ * LAGA_ERR_INVALID_ARG.  N and K need not be multiples of the 256-column tiles (576 works).
+ * status_word: one device word (4 bytes, 4-byte aligned), cleared by the call; read it with laga_query_status.
+ */
+int laga_linear(const void* x, const void* w, int M, int K, int N, void* y, void* status_word, void* stream);
+int laga_linear_backward(const void* dy, const void* x, const void* w, int M, int K, int N, void* dx, float* dw,
+                         unsigned flags, void* status_word, void* stream);
+
+/*
  * Step entry points (the same kernels laga_fwd / laga_bwd launch, callable on their own).
  *
  * laga_up_project: Algorithm 1 step 4.   kv bf16 [S, h*(d_nope+d_v)] = c_kv . w_kv_b  (fp32 accumulate).

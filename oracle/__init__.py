@@ -209,3 +209,18 @@ def bwd_keys(q, c_kv, k_pe, w_kv_b, dout, d_v, softmax_scale, keys, causal=True,
         raise RuntimeError(f"laga_oracle_bwd_keys failed with code {rc}")
     return {"dk": torch.from_numpy(dk), "dv": torch.from_numpy(dv), "dk_pe": torch.from_numpy(dkpe),
             "dc_kv": torch.from_numpy(dc)}
+
+
+# ---- the dense projections around the path (Algorithm 1 steps 1 and 7) ------------------------------
+# Their definition IS the matrix product, so the oracle is that product in float64 through the library
+# routine (torch.matmul on CPU tensors), nothing else.
+
+def linear(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
+    """y[M, N] = x[M, K] . w[K, N] in float64 (Algorithm 1 steps 1 and 7: W_q, W_kv_a, W_o)."""
+    return x.to(torch.float64) @ w.to(torch.float64)
+
+
+def linear_bwd(dy: torch.Tensor, x: torch.Tensor, w: torch.Tensor):
+    """Gradients of ``linear`` for an upstream dy[M, N]: dx[M, K] = dy . w^T and dw[K, N] = x^T . dy, float64."""
+    dy64 = dy.to(torch.float64)
+    return dy64 @ w.to(torch.float64).T, x.to(torch.float64).T @ dy64

@@ -20,7 +20,8 @@
 namespace laga {
 
 struct GemmArgs {
-    int M, N, K;          // problem size; M may be ragged, N % BN == 0, K tail is zero-filled by TMA
+    int M, N, K;          // problem size; M may be ragged; N % 8 == 0 (CTA-pair kernel: any such N; one-CTA kernel: N % BN == 0);
+                          // the K tail is zero-filled by TMA
     int k_tiles_per_split;
     int n_splits;         // split-K factor (1 unless EPI_ATOMIC_F32)
     void* C;              // bf16 [M, ldc] (EPI_BF16) or fp32 [M, ldc] (EPI_ATOMIC_F32)
@@ -265,7 +266,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_cta_rank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int tiles_n = args.N / BN;
+    const int tiles_n = (args.N + BN - 1) / BN;   // the last column tile may be ragged: loads past N are zero fill, stores are clipped
     const int tiles_m = (args.M + 255) / 256;
     const int tiles_per_batch = tiles_n * tiles_m * args.n_splits;
     const int total_tiles = tiles_per_batch * args.batches;
@@ -400,6 +401,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 if (EPI == EPI_BF16) {
 #pragma unroll 1
                     for (int c = 0; c < BN / 64; ++c, ++boxes) {
+                        if ((tb % tiles_n) * BN + c * 64 >= args.N) break;   // past the last column (ragged N); TMA clips a partial box
                         uint32_t r[64];
                         __syncwarp();
                         tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 64, r);
@@ -419,7 +421,7 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         }
                         fence_async_shared();
                         __syncwarp();
-                        if (lane == 0 && device_check(((n0 + c * 64) & 7) == 0 && n0 + c * 64 + 64 <= args.ldc, args.status, 0xE70000u | c)) {
+                        if (lane == 0 && device_check(((n0 + c * 64) & 7) == 0 && n0 + c * 64 < args.ldc, args.status, 0xE70000u | c)) {
                             tma_store_2d(&tmap_c, box, n0 + c * 64, m0 + quarter * 32);
                             tma_store_commit();
                         }
@@ -427,6 +429,8 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 } else {
 #pragma unroll 1
                     for (int c = 0; c < BN / 32; ++c) {
+                        const int col = (tb % tiles_n) * BN + c * 32;       // column within this batch's N
+                        if (col >= args.N) break;                           // ragged N: nothing beyond the last column
                         uint32_t r[32];
                         __syncwarp();
                         tmem_ld_x32(tmem_base + lane_addr + buf * BN + c * 32, r);
@@ -434,11 +438,12 @@ gemm_pair_sm100_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                         if (row < args.M) {
                             float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.C) +
                                                                     static_cast<size_t>(row) * args.ldc + n0 + c * 32);
-                            if (!device_check(aligned16_dev(dst) && n0 + c * 32 + 32 <= args.ldc, args.status, 0xE20000u | c)) continue;
+                            if (!device_check(aligned16_dev(dst) && n0 + c * 32 < args.ldc, args.status, 0xE20000u | c)) continue;
 #pragma unroll
                             for (int v = 0; v < 8; ++v)
-                                atomicAdd(dst + v, make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
-                                                               __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3])));
+                                if (col + v * 4 + 4 <= args.N)
+                                    atomicAdd(dst + v, make_float4(__uint_as_float(r[v * 4]), __uint_as_float(r[v * 4 + 1]),
+                                                                   __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3])));
                         }
                     }
                 }

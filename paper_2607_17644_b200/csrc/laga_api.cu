@@ -297,19 +297,20 @@ WorkSchedule make_schedule(int n_tiles, int S, int h, unsigned* counter, const i
     return WorkSchedule{n_tiles, h, static_cast<int>(banded), n_tiles * h, counter, tiles};
 }
 
-// ---- Algorithm 1 step 4: KV[S, N] = c_kv[S, d_c] . W[d_c, N] ------------------------------------
+// ---- y[M, N] = x[M, K] . W[K, N]: Algorithm 1 step 4 (KV = c_kv W, K = d_c) and the dense projections of
+// ---- steps 1 and 7 through laga_linear --------------------------------------------------------------
 int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
-                      cudaStream_t stream, bool overlap = false) {
+                      cudaStream_t stream, bool overlap = false, int K = kDc) {
     constexpr int BN = 256, STAGES = kGemmStages;
     auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
     using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
-    if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = d_c
-    if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;  // rows = d_c
+    if (!cached_tmap_bf16(&ta, c_kv, K, S, static_cast<uint64_t>(K) * 2, 128)) return LAGA_ERR_CUDA;     // rows = tokens, inner = K
+    if (!cached_tmap_bf16(&tb, w, N, K, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;        // rows = K
     CUtensorMap tc;                                                                    // output boxes of 64 columns x 32 rows
     if (!cached_tmap_bf16(&tc, kv, N, S, static_cast<uint64_t>(N) * 2, 32)) return LAGA_ERR_CUDA;
-    GemmArgs a{S, N, kDc, kDc / 64, 1, kv, N, status, nullptr, 0, 1, 0, 0, 0};
-    dim3 grid(pair_grid((N / BN) * ((S + 255) / 256)), 1, 1);
+    GemmArgs a{S, N, K, (K + 63) / 64, 1, kv, N, status, nullptr, 0, 1, 0, 0, 0};
+    dim3 grid(pair_grid(((N + BN - 1) / BN) * ((S + 255) / 256)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); launch_kernel(kernel, grid, dim3(192), L::kTotalBytes, stream, overlap, ta, tb, tc, a); }
     return launch_status();
 }
@@ -320,53 +321,54 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
 // GEMM that follows accumulates into it with atomics.
 template <int BN>
 int launch_dckv_bn(const void* dkv, const void* w, int S, int N, void* dc_kv, float* clear, size_t clear_floats,
-                   unsigned* status, cudaStream_t stream, bool overlap) {
+                   unsigned* status, cudaStream_t stream, bool overlap, int K) {
     constexpr int STAGES = kGemmStages;
     auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, false, EPI_BF16>;
     using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
     if (!cached_tmap_bf16(&ta, dkv, N, S, static_cast<uint64_t>(N) * 2, 128)) return LAGA_ERR_CUDA;
-    if (!cached_tmap_bf16(&tb, w, N, kDc, static_cast<uint64_t>(N) * 2, BN / 2)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&tb, w, N, K, static_cast<uint64_t>(N) * 2, BN / 2)) return LAGA_ERR_CUDA;
     CUtensorMap tc;
-    if (!cached_tmap_bf16(&tc, dc_kv, kDc, S, kDc * 2, 32)) return LAGA_ERR_CUDA;
-    GemmArgs a{S, kDc, N, (N + 63) / 64, 1, dc_kv, kDc, status, reinterpret_cast<float4*>(clear), clear_floats / 4, 1, 0, 0, 0};
-    dim3 grid(pair_grid((kDc / BN) * ((S + 255) / 256)), 1, 1);
+    if (!cached_tmap_bf16(&tc, dc_kv, K, S, static_cast<uint64_t>(K) * 2, 32)) return LAGA_ERR_CUDA;
+    GemmArgs a{S, K, N, (N + 63) / 64, 1, dc_kv, K, status, reinterpret_cast<float4*>(clear), clear_floats / 4, 1, 0, 0, 0};
+    dim3 grid(pair_grid(((K + BN - 1) / BN) * ((S + 255) / 256)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DCKV_GEMM, stream); launch_kernel(kernel, grid, dim3(192), L::kTotalBytes, stream, overlap, ta, tb, tc, a); }
     return launch_status();
 }
+// (K: the width of the output, d_c for the path itself)
 int launch_dckv(const void* dkv, const void* w, int S, int N, void* dc_kv, float* clear, size_t clear_floats,
-                unsigned* status, cudaStream_t stream, bool overlap = false) {
-    // The output is only d_c = 512 columns wide: with 256-column tiles a short sequence leaves most CTA pairs
-    // without a tile (S = 4096: 32 tiles for 74 pairs).  Narrower tiles double the count at the price of
-    // reading the dKV rows once more from L2.
-    const int tiles_256 = (kDc / 256) * ((S + 255) / 256);
+                unsigned* status, cudaStream_t stream, bool overlap = false, int K = kDc) {
+    // With 256-column tiles a short sequence leaves most CTA pairs without a tile when the output is narrow
+    // (d_c = 512, S = 4096: 32 tiles for 74 pairs).  Narrower tiles double the count at the price of reading the
+    // dKV rows once more from L2.
+    const int tiles_256 = ((K + 255) / 256) * ((S + 255) / 256);
     if (tiles_256 < sm_count() / 2)
-        return launch_dckv_bn<128>(dkv, w, S, N, dc_kv, clear, clear_floats, status, stream, overlap);
-    return launch_dckv_bn<256>(dkv, w, S, N, dc_kv, clear, clear_floats, status, stream, overlap);
+        return launch_dckv_bn<128>(dkv, w, S, N, dc_kv, clear, clear_floats, status, stream, overlap, K);
+    return launch_dckv_bn<256>(dkv, w, S, N, dc_kv, clear, clear_floats, status, stream, overlap, K);
 }
 
 // dW[d_c, N] += c_kv^T . dKV   (both operands read with the token index as K: MN-major), split over
 // the sequence with fp32 atomic accumulation into a buffer the caller of this function has cleared
 // (launch_dckv does it) or wants added to.
 int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool deterministic,
-              unsigned* status, cudaStream_t stream, bool overlap = false) {
+              unsigned* status, cudaStream_t stream, bool overlap = false, int K = kDc) {
     constexpr int BN = 256, STAGES = kGemmStages;
     auto kernel = gemm_pair_sm100_kernel<BN, STAGES, true, true, EPI_ATOMIC_F32>;
     using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
-    if (!cached_tmap_bf16(&ta, c_kv, kDc, S, kDc * 2, 64)) return LAGA_ERR_CUDA;
+    if (!cached_tmap_bf16(&ta, c_kv, K, S, static_cast<uint64_t>(K) * 2, 64)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tb, dkv, N, S, static_cast<uint64_t>(N) * 2, 64)) return LAGA_ERR_CUDA;
     // Split the sequence to fill the persistent grid, but every split adds one fp32 atomic pass over the whole
-    // [d_c, N] output.  Measured on B200: the atomics of one pass move at about 4.2 TB/s and the tiles run at
+    // [K, N] output.  Measured on B200: the atomics of one pass move at about 4.2 TB/s and the tiles run at
     // about 1.3 PFLOP/s times the fill of the last wave, so pick the split count that minimises
     //     flops / (1.3e15 * fill(s)) + s * output bytes / 4.2e12
     // (S = 4096, h = 16: 2 splits, 25 us, where filling the grid to 97 % with 9 splits took 39 us).
-    const int tiles = (kDc / 256) * (N / BN);
+    const int tiles = ((K + 255) / 256) * ((N + BN - 1) / BN);
     const int k_tiles = (S + 63) / 64;
     const int sms = sm_count() / 2;       // CTA pairs
     int splits = 1;
     double best = 1e30;
-    const double flops = 2.0 * S * kDc * N, out_bytes = static_cast<double>(kDc) * N * sizeof(float);
+    const double flops = 2.0 * S * K * N, out_bytes = static_cast<double>(K) * N * sizeof(float);
     for (int s = 1; s <= 16 && s <= k_tiles && !deterministic; ++s) {   // one split: one add per element
         const int total = tiles * s;
         const double fill = static_cast<double>(total) / (static_cast<double>((total + sms - 1) / sms) * sms);
@@ -375,7 +377,7 @@ int launch_dw(const void* c_kv, const void* dkv, int S, int N, float* dw, bool d
     }
     const int per_split = (k_tiles + splits - 1) / splits;
     splits = (k_tiles + per_split - 1) / per_split;
-    GemmArgs a{kDc, N, S, per_split, splits, dw, N, status, nullptr, 0, 1, 0, 0, 0};
+    GemmArgs a{K, N, S, per_split, splits, dw, N, status, nullptr, 0, 1, 0, 0, 0};
     dim3 grid(pair_grid(tiles * splits), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_DW_GEMM, stream); launch_kernel(kernel, grid, dim3(192), L::kTotalBytes, stream, overlap, ta, tb, ta, a); }   // (fp32 atomic epilogue: the output map is unused)
     return launch_status();
@@ -794,6 +796,36 @@ size_t laga_bwd_varlen_workspace_bytes(int S_total, int n_seqs, int h, int d_c, 
     if (S_total < 1 || h < 1 || n_seqs < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
     if (flags & LAGA_FLAG_FUSED_BWD) return 0;
     return bwd_workspace_layout(S_total, h, (flags & LAGA_FLAG_DETERMINISTIC) != 0, false, n_seqs).total;
+}
+
+int laga_linear(const void* x, const void* w, int M, int K, int N, void* y, void* status_word, void* stream) {
+    if (!x || !w || !y || !status_word || M < 1 || K < 8 || N < 8 || (K & 7) || (N & 7)) return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return LAGA_ERR_INVALID_ARG;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({x, w, y, status_word})) != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = zero_status_word(status_word, st)) != LAGA_OK) return rc;
+    return launch_up_project(x, w, M, N, y, static_cast<unsigned*>(status_word), st, false, K);
+}
+
+int laga_linear_backward(const void* dy, const void* x, const void* w, int M, int K, int N, void* dx, float* dw,
+                         unsigned flags, void* status_word, void* stream) {
+    if (!dy || !x || !w || !dx || !dw || !status_word || M < 1 || K < 8 || N < 8 || (K & 7) || (N & 7))
+        return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(dy) || !aligned16(x) || !aligned16(w) || !aligned16(dx) || !aligned16(dw)) return LAGA_ERR_INVALID_ARG;
+    if (flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC)) return LAGA_ERR_INVALID_ARG;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({dy, x, w, dx, dw, status_word})) != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned* status = static_cast<unsigned*>(status_word);
+    const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
+    if ((rc = zero_status_word(status_word, st)) != LAGA_OK) return rc;
+    if ((rc = launch_dckv(dy, w, M, N, dx, accumulate ? nullptr : dw, accumulate ? 0 : static_cast<size_t>(K) * N, status, st,
+                          false, K)) != LAGA_OK)
+        return rc;
+    return launch_dw(x, dy, M, N, dw, (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st, true, K);
 }
 
 int laga_fwd_varlen(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const int* cu_seqlens,

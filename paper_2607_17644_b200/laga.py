@@ -44,6 +44,8 @@ SIGNATURES = {
     "laga_bwd_varlen": (_ci, [_vp] * 7 + [ctypes.POINTER(_ci)] + [_ci] * 7 + [_cf, _ci] + [_vp] * 4 + [_vp, _sz, _cu, _vp]),
     "laga_absorbed_fwd_workspace_bytes": (_sz, [_ci] * 6),
     "laga_absorbed_fwd": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
+    "laga_linear": (_ci, [_vp, _vp, _ci, _ci, _ci, _vp, _vp, _vp]),
+    "laga_linear_backward": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp, _vp, _cu, _vp, _vp]),
     "laga_up_project": (_ci, [_vp, _vp] + [_ci] * 5 + [_vp, _vp, _vp]),
     "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
     "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
@@ -293,6 +295,45 @@ def bwd(q, c_kv, k_pe, w_kv_b, out, lse, dout, d_v=128, softmax_scale=None, caus
                                        _ptr(workspace), workspace.numel(), flags, _stream(stream, dev))
     _check(rc, "laga_bwd" if cu is None else "laga_bwd_varlen")
     return dq, dc_kv, dk_pe, dw_kv_b, workspace
+
+
+def linear(x, w, y=None, status_word=None, stream=None):
+    """laga_linear: y bf16 [M, N] = x [M, K] . w [K, N] (Algorithm 1 steps 1 and 7).  Returns (y, status_word)."""
+    M, K = x.shape
+    N = w.shape[1]
+    _dev(x, torch.bfloat16, (M, K), "x")
+    _dev(w, torch.bfloat16, (K, N), "w")
+    dev = same_device(x, w, y, status_word)
+    y = torch.empty(M, N, dtype=torch.bfloat16, device=dev) if y is None else _dev(y, torch.bfloat16, (M, N), "y")
+    if status_word is None:
+        status_word = torch.zeros(1, dtype=torch.int32, device=dev)
+    with _on(dev):
+        rc = lib().laga_linear(_ptr(x), _ptr(w), M, K, N, _ptr(y), _ptr(status_word), _stream(stream, dev))
+    _check(rc, "laga_linear")
+    return y, status_word
+
+
+def linear_backward(dy, x, w, dx=None, dw=None, flags=0, status_word=None, stream=None):
+    """laga_linear_backward: dx bf16 [M, K] = dy . w^T, dw fp32 [K, N] (+)= x^T . dy.  Returns (dx, dw, status_word)."""
+    M, K = x.shape
+    N = w.shape[1]
+    _dev(x, torch.bfloat16, (M, K), "x")
+    _dev(w, torch.bfloat16, (K, N), "w")
+    _dev(dy, torch.bfloat16, (M, N), "dy")
+    dev = same_device(dy, x, w, dx, dw, status_word)
+    dx = torch.empty(M, K, dtype=torch.bfloat16, device=dev) if dx is None else _dev(dx, torch.bfloat16, (M, K), "dx")
+    if dw is None:
+        if flags & FLAG_ACCUM_DW:
+            raise ValueError("LAGA_FLAG_ACCUM_DW needs an existing dw to add into")
+        dw = torch.empty(K, N, dtype=torch.float32, device=dev)
+    _dev(dw, torch.float32, (K, N), "dw")
+    if status_word is None:
+        status_word = torch.zeros(1, dtype=torch.int32, device=dev)
+    with _on(dev):
+        rc = lib().laga_linear_backward(_ptr(dy), _ptr(x), _ptr(w), M, K, N, _ptr(dx), _ptr(dw), flags, _ptr(status_word),
+                                        _stream(stream, dev))
+    _check(rc, "laga_linear_backward")
+    return dx, dw, status_word
 
 
 def up_project(c_kv, w_kv_b, h, d_nope=128, d_v=128, kv=None, status_word=None, stream=None):

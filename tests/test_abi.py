@@ -114,6 +114,11 @@ def test_argument_validation_happens_before_any_device_work(laga):
     assert lib.laga_up_project(None, good, 128, 2, 512, 128, 128, good, good, None) == laga.ERR_INVALID_ARG
     assert lib.laga_kv_backward(good, good, good, 128, 2, 512, 128, 128, good, good, 4, good, None) == laga.ERR_INVALID_ARG
     assert lib.laga_query_status(None, None, None) == laga.ERR_INVALID_ARG
+    assert lib.laga_linear(good, good, 128, 512, 260, good, good, None) == laga.ERR_INVALID_ARG      # N not a multiple of 8
+    assert lib.laga_linear(good, good, 128, 4, 256, good, good, None) == laga.ERR_INVALID_ARG        # K < 8
+    assert lib.laga_linear(good, None, 128, 512, 256, good, good, None) == laga.ERR_INVALID_ARG
+    assert lib.laga_linear_backward(good, good, good, 0, 512, 256, good, good, 0, good, None) == laga.ERR_INVALID_ARG
+    assert lib.laga_linear_backward(good, good, good, 8, 512, 256, good, good, 4, good, None) == laga.ERR_INVALID_ARG   # KV_SAVED means nothing here
 
 
 def test_varlen_entry_points_validate_cu_seqlens_before_any_device_work(laga):

@@ -336,3 +336,38 @@ def test_row_and_key_subsets_match_full_backward(oracle, causal):
     assert (k["dk"] - full["dk"][keys]).abs().max() < 1e-13 and (k["dv"] - full["dv"][keys]).abs().max() < 1e-13
     assert (k["dk_pe"] - full["dk_pe"][keys]).abs().max() < 1e-13
     assert (k["dc_kv"] - full["dc_kv"][keys]).abs().max() < 1e-12
+
+
+def test_linear_oracle_against_loops_closed_forms_and_autograd(oracle):
+    """The dense projections (Algorithm 1 steps 1 and 7).  The oracle calls a library matrix product, so it is
+    pinned by things that are not that call: an explicit triple loop on a tiny case (a transposed operand or a
+    swapped index fails it), closed forms (identity weight; all-ones weight = row sums), the bilinear trace
+    identity between the two gradients, and torch.autograd on an elementwise restatement."""
+    g = torch.Generator().manual_seed(31)
+    M, K, N = 5, 4, 3
+    x = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    w = torch.randn(K, N, generator=g).to(torch.bfloat16)
+    dy = torch.randn(M, N, generator=g).to(torch.bfloat16)
+    y = oracle.linear(x, w)
+    dx, dw = oracle.linear_bwd(dy, x, w)
+    xs, ws, dys = x.double().tolist(), w.double().tolist(), dy.double().tolist()
+    for m in range(M):
+        for n in range(N):
+            assert abs(float(y[m, n]) - sum(xs[m][k] * ws[k][n] for k in range(K))) < 1e-12
+        for k in range(K):
+            assert abs(float(dx[m, k]) - sum(dys[m][n] * ws[k][n] for n in range(N))) < 1e-12
+    for k in range(K):
+        for n in range(N):
+            assert abs(float(dw[k, n]) - sum(xs[m][k] * dys[m][n] for m in range(M))) < 1e-12
+    # closed forms
+    eye = torch.eye(K).to(torch.bfloat16)
+    assert torch.equal(oracle.linear(x, eye), x.double())
+    ones = torch.ones(K, 2).to(torch.bfloat16)
+    assert torch.allclose(oracle.linear(x, ones), x.double().sum(dim=1, keepdim=True).expand(M, 2), atol=1e-12)
+    # <dy, y> = <dx, x> = <dw, w>
+    t = float((dy.double() * y).sum())
+    assert abs(t - float((dx * x.double()).sum())) < 1e-10 and abs(t - float((dw * w.double()).sum())) < 1e-10
+    # autograd of sum_mn dy[m,n] * sum_k x[m,k] w[k,n], written with broadcasting (no matmul)
+    xa, wa = x.double().requires_grad_(True), w.double().requires_grad_(True)
+    ((xa[:, :, None] * wa[None, :, :]).sum(dim=1) * dy.double()).sum().backward()
+    assert torch.allclose(xa.grad, dx, atol=1e-12) and torch.allclose(wa.grad, dw, atol=1e-12)
