@@ -177,3 +177,23 @@ def test_autograd_wrapper_takes_packed_sequences(laga):
     assert torch.equal(leaves[0].grad, dq) and torch.equal(leaves[1].grad, dc_kv)
     assert float((leaves[2].grad.float() - dk_pe.float()).abs().max()) <= 2e-2 * max(1.0, float(dk_pe.float().abs().max()))
     assert float((leaves[3].grad.float() - dw).norm() / dw.norm()) < 1e-2      # bf16 copy of an fp32 gradient
+
+
+def test_random_packings(laga, oracle):
+    """Seeded random packings (two to six sequences of 1..700 tokens, one to three heads, either mask): the
+    longest-first tile order and the per-sequence padding change with every draw."""
+    rng = torch.Generator().manual_seed(4600)
+    for trial in range(6):
+        n_seqs = int(torch.randint(2, 7, (1,), generator=rng))
+        lengths = [int(torch.randint(1, 701, (1,), generator=rng)) for _ in range(n_seqs)]
+        h = int(torch.randint(1, 4, (1,), generator=rng))
+        causal = bool(torch.randint(0, 2, (1,), generator=rng))
+        cu = cu_of(lengths)
+        sh = LagaShape(S=cu[-1], h=h)
+        tensors = make_inputs(sh, 4600 + trial)
+        g = run_packed(laga, tensors, cu, causal)
+        r = oracle_packed(oracle, tensors, sh, cu, causal)
+        for name in ("out", "dq", "dk_pe", "dc_kv"):
+            check_tensor(f"{name} (lengths {lengths}, h={h}, causal={causal})", g[name], r[name])
+        assert max_abs(g["lse"], r["lse"]) <= TOL_LSE
+        check_dw(g["dw"], r["dw"])
