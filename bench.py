@@ -427,6 +427,25 @@ def run_linear(args):
                       "bwd_ms": bwd_ms, "bwd_tflops": 2 * fl / (bwd_ms * 1e-3) / 1e12,
                       "torch_matmul_fwd_ms": lib_fwd_ms, "torch_matmul_bwd_ms": lib_bwd_ms}
         del x, w, dy, y, dx, dw, wt
+    # LayerNorm of the latent (step 1): HBM-bound, reported against the measured copy bandwidth.  262144 tokens so
+    # that one tensor (268 MB) is larger than L2; the timed calls then really stream from and to HBM.
+    D, M_ln = 512, 262144
+    x = torch.randn(M_ln, D, generator=g).to(torch.bfloat16).to(dev)
+    gamma = (1 + 0.2 * torch.randn(D, generator=g)).to(torch.bfloat16).to(dev)
+    beta = (0.1 * torch.randn(D, generator=g)).to(torch.bfloat16).to(dev)
+    dy = torch.randn(M_ln, D, generator=g).to(torch.bfloat16).to(dev)
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    _, mean, rstd = laga.layernorm(x, gamma, beta, y=y)
+    ln_fwd_ms = timed(lambda: laga.layernorm(x, gamma, beta, y=y))
+    ln_bwd_ms = timed(lambda: laga.layernorm_backward(dy, x, gamma, mean, rstd, dx=dx))
+    peaks = measured_peaks()
+    fwd_bytes, bwd_bytes = 2 * M_ln * D * 2 + 2 * M_ln * 4, 3 * M_ln * D * 2 + 2 * M_ln * 4
+    layernorm = {"M": M_ln, "D": D, "fwd_ms": ln_fwd_ms, "fwd_bytes": fwd_bytes, "fwd_gbs": fwd_bytes / (ln_fwd_ms * 1e-3) / 1e9,
+                 "bwd_ms": ln_bwd_ms, "bwd_bytes": bwd_bytes, "bwd_gbs": bwd_bytes / (ln_bwd_ms * 1e-3) / 1e9,
+                 "hbm_peak_gbs": peaks["hbm_gbs"], "fwd_frac": fwd_bytes / (ln_fwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                 "bwd_frac": bwd_bytes / (ln_bwd_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                 "note": "algorithmic bytes: x in, y out (+ the two statistics) forward; dy and x in, dx out backward"}
+    del x, dy, y, dx
     head = rows["W_o (step 7: 16 heads x 128 -> hidden)"]
     line = {"metric": "linear_projection_fwd_tflops", "value": head["fwd_tflops"], "unit": UNIT, "n_gpus": 1, "steps": K_steps,
             "warmup": W, "ms_per_step": head["fwd_ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -434,7 +453,7 @@ def run_linear(args):
             "config": {"workload": "linear: the dense projections of Algorithm 1 steps 1, 4 and 7 at 16384 tokens, 16-head shard "
                                    "(headline of this line: W_o forward)",
                        "l2_policy": "operands larger than L2 except W"},
-            "shapes": rows, "gpu_launches": K_steps}
+            "shapes": rows, "layernorm_of_the_latent": layernorm, "gpu_launches": K_steps}
     print(json.dumps(line), flush=True)
 
 

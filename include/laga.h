@@ -169,6 +169,23 @@ int laga_linear_backward(const void* dy, const void* x, const void* w, int M, in
                          unsigned flags, void* status_word, void* stream);
 
 /*
+ * LayerNorm of the latent (Algorithm 1 step 1: latent <- LayerNorm(latent), between W_kv_a and the gather).
+ * The paper names the operation and nothing else; this is the usual definition over the last axis with
+ * biased variance, learnable scale and optional shift:
+ *   y[m, :] = (x[m, :] - mean_m) * rstd_m * gamma + beta,   rstd_m = 1 / sqrt(var_m + eps)
+ * x, y, dy, dx bf16 [M, D]; gamma, beta bf16 [D] (beta may be NULL: no shift); statistics and arithmetic fp32.
+ * laga_layernorm optionally writes mean and rstd (fp32 [M]; either may be NULL) -- the backward needs both.
+ * laga_layernorm_backward writes dx and OVERWRITES dgamma fp32 [D] and, if not NULL, dbeta fp32 [D] (sums over
+ * the M rows, added with fp32 atomics: low-order bits may vary from run to run).
+ * D must be a multiple of 8 and at most 1024 (the latent is 512 wide), eps >= 0; anything else is
+ * LAGA_ERR_INVALID_ARG.  HBM-bound kernels without bounded waits: no status word, errors are launch errors.
+ */
+int laga_layernorm(const void* x, const void* gamma, const void* beta, int M, int D, float eps, void* y, float* mean,
+                   float* rstd, void* stream);
+int laga_layernorm_backward(const void* dy, const void* x, const void* gamma, const float* mean, const float* rstd, int M,
+                            int D, void* dx, float* dgamma, float* dbeta, void* stream);
+
+/*
  * Step entry points (the same kernels laga_fwd / laga_bwd launch, callable on their own).
  *
  * laga_up_project: Algorithm 1 step 4.   kv bf16 [S, h*(d_nope+d_v)] = c_kv . w_kv_b  (fp32 accumulate).

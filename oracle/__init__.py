@@ -224,3 +224,44 @@ def linear_bwd(dy: torch.Tensor, x: torch.Tensor, w: torch.Tensor):
     """Gradients of ``linear`` for an upstream dy[M, N]: dx[M, K] = dy . w^T and dw[K, N] = x^T . dy, float64."""
     dy64 = dy.to(torch.float64)
     return dy64 @ w.to(torch.float64).T, x.to(torch.float64).T @ dy64
+
+
+# ---- LayerNorm of the latent (Algorithm 1 step 1) ---------------------------------------------------
+# The paper names the operation only; the definition written out here is the usual one: statistics over the
+# last axis, biased variance, scale gamma, optional shift beta.  float64 throughout, one row at a time.
+
+def layernorm(x: torch.Tensor, gamma: torch.Tensor, beta, eps: float):
+    """y = (x - mean) / sqrt(var + eps) * gamma + beta, row by row.  Returns (y, mean, rstd) in float64."""
+    x64, g64 = x.to(torch.float64), gamma.to(torch.float64)
+    b64 = torch.zeros_like(g64) if beta is None else beta.to(torch.float64)
+    M, D = x64.shape
+    y = torch.empty_like(x64)
+    mean = torch.empty(M, dtype=torch.float64)
+    rstd = torch.empty(M, dtype=torch.float64)
+    for m in range(M):
+        mu = x64[m].sum() / D
+        var = ((x64[m] - mu) ** 2).sum() / D
+        r = 1.0 / torch.sqrt(var + eps)
+        y[m] = (x64[m] - mu) * r * g64 + b64
+        mean[m], rstd[m] = mu, r
+    return y, mean, rstd
+
+
+def layernorm_bwd(dy: torch.Tensor, x: torch.Tensor, gamma: torch.Tensor, eps: float):
+    """Gradients of ``layernorm`` for an upstream dy: (dx [M, D], dgamma [D], dbeta [D]) in float64, from the chain
+    rule through mean and variance written out row by row."""
+    dy64, x64, g64 = dy.to(torch.float64), x.to(torch.float64), gamma.to(torch.float64)
+    M, D = x64.shape
+    dx = torch.empty_like(x64)
+    dgamma = torch.zeros(D, dtype=torch.float64)
+    dbeta = torch.zeros(D, dtype=torch.float64)
+    for m in range(M):
+        mu = x64[m].sum() / D
+        var = ((x64[m] - mu) ** 2).sum() / D
+        r = 1.0 / torch.sqrt(var + eps)
+        xhat = (x64[m] - mu) * r
+        g = dy64[m] * g64
+        dx[m] = r * (g - g.sum() / D - xhat * (g * xhat).sum() / D)
+        dgamma += dy64[m] * xhat
+        dbeta += dy64[m]
+    return dx, dgamma, dbeta

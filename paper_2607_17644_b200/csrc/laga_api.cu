@@ -17,6 +17,7 @@
 #include "attn_bwd_sm100.cuh"
 #include "attn_fwd_sm100.cuh"
 #include "gemm_sm100.cuh"
+#include "layernorm_sm100.cuh"
 
 namespace {
 
@@ -826,6 +827,51 @@ int laga_linear_backward(const void* dy, const void* x, const void* w, int M, in
                           false, K)) != LAGA_OK)
         return rc;
     return launch_dw(x, dy, M, N, dw, (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st, true, K);
+}
+
+int laga_layernorm(const void* x, const void* gamma, const void* beta, int M, int D, float eps, void* y, float* mean,
+                   float* rstd, void* stream) {
+    if (!x || !gamma || !y || M < 1 || D < 8 || (D & 7) || D > kLnMaxD || !(eps >= 0.f)) return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(gamma) || !aligned16(y) || (beta && !aligned16(beta))) return LAGA_ERR_INVALID_ARG;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({x, gamma, y})) != LAGA_OK) return rc;
+    if (beta && (rc = check_pointers({beta})) != LAGA_OK) return rc;
+    if (mean && (rc = check_pointers({mean})) != LAGA_OK) return rc;
+    if (rstd && (rc = check_pointers({rstd})) != LAGA_OK) return rc;
+    // one resident wave striding over the rows (four blocks of 256 threads fit an SM at D <= 512)
+    const int blocks_needed = (M + kLnWarps - 1) / kLnWarps, cap = sm_count() * 4;
+    const dim3 grid(blocks_needed < cap ? blocks_needed : cap), block(kLnWarps * 32);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto xs = static_cast<const __nv_bfloat16*>(x), gs = static_cast<const __nv_bfloat16*>(gamma), bs = static_cast<const __nv_bfloat16*>(beta);
+    auto ys = static_cast<__nv_bfloat16*>(y);
+    if (D <= 256) layernorm_fwd_kernel<1><<<grid, block, 0, st>>>(xs, gs, bs, M, D, eps, ys, mean, rstd);
+    else if (D <= 512) layernorm_fwd_kernel<2><<<grid, block, 0, st>>>(xs, gs, bs, M, D, eps, ys, mean, rstd);
+    else layernorm_fwd_kernel<4><<<grid, block, 0, st>>>(xs, gs, bs, M, D, eps, ys, mean, rstd);
+    return launch_status();
+}
+
+int laga_layernorm_backward(const void* dy, const void* x, const void* gamma, const float* mean, const float* rstd, int M,
+                            int D, void* dx, float* dgamma, float* dbeta, void* stream) {
+    if (!dy || !x || !gamma || !mean || !rstd || !dx || !dgamma || M < 1 || D < 8 || (D & 7) || D > kLnMaxD)
+        return LAGA_ERR_INVALID_ARG;
+    if (!aligned16(dy) || !aligned16(x) || !aligned16(gamma) || !aligned16(dx)) return LAGA_ERR_INVALID_ARG;
+    int rc = check_device();
+    if (rc != LAGA_OK) return rc;
+    if ((rc = check_pointers({dy, x, gamma, mean, rstd, dx, dgamma})) != LAGA_OK) return rc;
+    if (dbeta && (rc = check_pointers({dbeta})) != LAGA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(dgamma, 0, static_cast<size_t>(D) * sizeof(float), st) != cudaSuccess) return LAGA_ERR_CUDA;
+    if (dbeta && cudaMemsetAsync(dbeta, 0, static_cast<size_t>(D) * sizeof(float), st) != cudaSuccess) return LAGA_ERR_CUDA;
+    // one resident wave (two blocks per SM) strides over the rows: each block ends with D atomics per output
+    const int blocks_needed = (M + kLnWarps - 1) / kLnWarps, cap = sm_count() * 2;
+    const dim3 grid(blocks_needed < cap ? blocks_needed : cap), block(kLnWarps * 32);
+    auto dys = static_cast<const __nv_bfloat16*>(dy), xs = static_cast<const __nv_bfloat16*>(x), gs = static_cast<const __nv_bfloat16*>(gamma);
+    auto dxs = static_cast<__nv_bfloat16*>(dx);
+    if (D <= 256) layernorm_bwd_kernel<1><<<grid, block, 0, st>>>(dys, xs, gs, mean, rstd, M, D, dxs, dgamma, dbeta);
+    else if (D <= 512) layernorm_bwd_kernel<2><<<grid, block, 0, st>>>(dys, xs, gs, mean, rstd, M, D, dxs, dgamma, dbeta);
+    else layernorm_bwd_kernel<4><<<grid, block, 0, st>>>(dys, xs, gs, mean, rstd, M, D, dxs, dgamma, dbeta);
+    return launch_status();
 }
 
 int laga_fwd_varlen(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const int* cu_seqlens,

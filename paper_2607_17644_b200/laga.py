@@ -46,6 +46,8 @@ SIGNATURES = {
     "laga_absorbed_fwd": (_ci, [_vp] * 4 + [_ci] * 6 + [_cf, _ci, _vp, _vp, _vp, _sz, _cu, _vp]),
     "laga_linear": (_ci, [_vp, _vp, _ci, _ci, _ci, _vp, _vp, _vp]),
     "laga_linear_backward": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp, _vp, _cu, _vp, _vp]),
+    "laga_layernorm": (_ci, [_vp, _vp, _vp, _ci, _ci, _cf, _vp, _vp, _vp, _vp]),
+    "laga_layernorm_backward": (_ci, [_vp] * 5 + [_ci, _ci] + [_vp] * 4),
     "laga_up_project": (_ci, [_vp, _vp] + [_ci] * 5 + [_vp, _vp, _vp]),
     "laga_kv_backward": (_ci, [_vp] * 3 + [_ci] * 5 + [_vp, _vp, _cu, _vp, _vp]),
     "laga_query_status": (_ci, [_vp, _vp, ctypes.POINTER(_cu)]),
@@ -334,6 +336,43 @@ def linear_backward(dy, x, w, dx=None, dw=None, flags=0, status_word=None, strea
                                         _stream(stream, dev))
     _check(rc, "laga_linear_backward")
     return dx, dw, status_word
+
+
+def layernorm(x, gamma, beta=None, eps=1e-5, y=None, stream=None):
+    """laga_layernorm: returns (y bf16 [M, D], mean fp32 [M], rstd fp32 [M])."""
+    M, D = x.shape
+    _dev(x, torch.bfloat16, (M, D), "x")
+    _dev(gamma, torch.bfloat16, (D,), "gamma")
+    if beta is not None:
+        _dev(beta, torch.bfloat16, (D,), "beta")
+    dev = same_device(x, gamma, beta, y)
+    y = torch.empty_like(x) if y is None else _dev(y, torch.bfloat16, (M, D), "y")
+    mean = torch.empty(M, dtype=torch.float32, device=dev)
+    rstd = torch.empty(M, dtype=torch.float32, device=dev)
+    with _on(dev):
+        rc = lib().laga_layernorm(_ptr(x), _ptr(gamma), _ptr(beta) if beta is not None else None, M, D, float(eps), _ptr(y),
+                                  _ptr(mean), _ptr(rstd), _stream(stream, dev))
+    _check(rc, "laga_layernorm")
+    return y, mean, rstd
+
+
+def layernorm_backward(dy, x, gamma, mean, rstd, with_beta=True, dx=None, stream=None):
+    """laga_layernorm_backward: returns (dx bf16 [M, D], dgamma fp32 [D], dbeta fp32 [D] or None)."""
+    M, D = x.shape
+    _dev(x, torch.bfloat16, (M, D), "x")
+    _dev(dy, torch.bfloat16, (M, D), "dy")
+    _dev(gamma, torch.bfloat16, (D,), "gamma")
+    _dev(mean, torch.float32, (M,), "mean")
+    _dev(rstd, torch.float32, (M,), "rstd")
+    dev = same_device(dy, x, gamma, mean, rstd, dx)
+    dx = torch.empty_like(x) if dx is None else _dev(dx, torch.bfloat16, (M, D), "dx")
+    dgamma = torch.empty(D, dtype=torch.float32, device=dev)
+    dbeta = torch.empty(D, dtype=torch.float32, device=dev) if with_beta else None
+    with _on(dev):
+        rc = lib().laga_layernorm_backward(_ptr(dy), _ptr(x), _ptr(gamma), _ptr(mean), _ptr(rstd), M, D, _ptr(dx), _ptr(dgamma),
+                                           _ptr(dbeta) if dbeta is not None else None, _stream(stream, dev))
+    _check(rc, "laga_layernorm_backward")
+    return dx, dgamma, dbeta
 
 
 def up_project(c_kv, w_kv_b, h, d_nope=128, d_v=128, kv=None, status_word=None, stream=None):

@@ -371,3 +371,51 @@ def test_linear_oracle_against_loops_closed_forms_and_autograd(oracle):
     xa, wa = x.double().requires_grad_(True), w.double().requires_grad_(True)
     ((xa[:, :, None] * wa[None, :, :]).sum(dim=1) * dy.double()).sum().backward()
     assert torch.allclose(xa.grad, dx, atol=1e-12) and torch.allclose(wa.grad, dw, atol=1e-12)
+
+
+def test_layernorm_oracle_against_library_closed_forms_and_finite_differences(oracle):
+    """LayerNorm of the latent (Algorithm 1 step 1).  Pins: torch.nn.functional.layer_norm with float64 autograd
+    (a library routine the oracle does not call), closed forms (a constant row normalises to beta; a two-valued
+    row to +-gamma), invariance to a shift and -- with eps = 0 -- to a positive scale of the row, the identities
+    sum_c dx = 0 and sum_c dx * xhat = 0, and central finite differences."""
+    g = torch.Generator().manual_seed(41)
+    M, D, eps = 6, 16, 1e-5
+    x = (torch.randn(M, D, generator=g) * 2 + 0.5).to(torch.bfloat16)
+    gamma = (1 + 0.3 * torch.randn(D, generator=g)).to(torch.bfloat16)
+    beta = (0.2 * torch.randn(D, generator=g)).to(torch.bfloat16)
+    dy = torch.randn(M, D, generator=g).to(torch.bfloat16)
+    y, mean, rstd = oracle.layernorm(x, gamma, beta, eps)
+    dx, dgamma, dbeta = oracle.layernorm_bwd(dy, x, gamma, eps)
+    xa, ga, ba = x.double().requires_grad_(True), gamma.double().requires_grad_(True), beta.double().requires_grad_(True)
+    ya = torch.nn.functional.layer_norm(xa, (D,), ga, ba, eps)
+    assert torch.allclose(ya, y, atol=1e-12)
+    (ya * dy.double()).sum().backward()
+    assert torch.allclose(xa.grad, dx, atol=1e-11) and torch.allclose(ga.grad, dgamma, atol=1e-11)
+    assert torch.allclose(ba.grad, dbeta, atol=1e-12)
+    assert torch.allclose(mean, x.double().mean(dim=1), atol=1e-13)
+    assert torch.allclose(rstd, 1 / torch.sqrt(x.double().var(dim=1, unbiased=False) + eps), atol=1e-12)
+    # closed forms
+    const = torch.full((1, D), 3.0).to(torch.bfloat16)
+    assert torch.allclose(oracle.layernorm(const, gamma, beta, eps)[0], beta.double().expand(1, D), atol=1e-12)
+    two = torch.tensor([[1.0, -1.0] * (D // 2)]).to(torch.bfloat16)        # mean 0, variance 1
+    assert torch.allclose(oracle.layernorm(two, gamma, None, 0.0)[0], two.double() * gamma.double(), atol=1e-12)
+    # shift invariance; scale invariance without eps
+    assert torch.allclose(oracle.layernorm(x.double() + 7.0, gamma, beta, eps)[0], y, atol=1e-10)
+    assert torch.allclose(oracle.layernorm(x.double() * 4.0, gamma, beta, 0.0)[0], oracle.layernorm(x, gamma, beta, 0.0)[0], atol=1e-10)
+    # dx is orthogonal to the constant and to xhat (the two directions the normalisation removes), up to eps
+    xhat = (x.double() - mean[:, None]) * rstd[:, None]
+    assert float(dx.sum(dim=1).abs().max()) < 1e-10
+    assert float((dx * xhat).sum(dim=1).abs().max()) < 1e-3
+    # finite differences of L = sum(dy * y) in a few entries of x and gamma
+    def loss(xv, gv):
+        return float((oracle.layernorm(xv, gv, beta, eps)[0] * dy.double()).sum())
+    for (m, c) in [(0, 0), (3, 7), (5, 15)]:
+        h = 1e-5
+        xp, xm = x.double().clone(), x.double().clone()
+        xp[m, c] += h
+        xm[m, c] -= h
+        assert abs((loss(xp, gamma) - loss(xm, gamma)) / (2 * h) - float(dx[m, c])) < 1e-6
+        gp, gmn = gamma.double().clone(), gamma.double().clone()
+        gp[c] += h
+        gmn[c] -= h
+        assert abs((loss(x, gp) - loss(x, gmn)) / (2 * h) - float(dgamma[c])) < 1e-6
