@@ -10,7 +10,7 @@ absence is an error: there is no CPU or eager fallback.
 """
 from .inputs import CONFIGS, CONFIG_SEEDS, LagaShape, make_inputs  # noqa: F401
 
-__all__ = ["CONFIGS", "CONFIG_SEEDS", "LagaShape", "make_inputs", "laga", "laga_attention"]
+__all__ = ["CONFIGS", "CONFIG_SEEDS", "LagaShape", "make_inputs", "laga", "laga_attention", "LagaBlock"]
 
 
 def __getattr__(name):
@@ -19,4 +19,6 @@ def __getattr__(name):
         return importlib.import_module(".laga", __name__)
     if name == "laga_attention":          # the differentiable call (torch.autograd plumbing around laga.fwd / laga.bwd)
         return importlib.import_module(".autograd", __name__).laga_attention
+    if name == "LagaBlock":               # Algorithm 1 with one rank, every step on the library's kernels
+        return importlib.import_module(".block", __name__).LagaBlock
     raise AttributeError(name)
