@@ -682,7 +682,7 @@ int zero_status_word(void* status_word, cudaStream_t stream) {
 
 extern "C" {
 
-int laga_version(void) { return 200; }
+int laga_version(void) { return 210; }
 
 const char* laga_status_string(int status) {
     switch (status) {
