@@ -70,7 +70,7 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 // Persistent: one CTA per SM takes (query tile, head) items from the work counter.  The K, V and
 // score-tile rings and the alternation of the two softmax groups run on a tile count that continues
 // across items, so the producers prefetch the next item's first key tiles under the current item's
-// last ones; between items, group 0 puts the next query tile into TMEM before the finished O is
+// last ones; between items, the groups put the next query tile into TMEM before the finished O is
 // drained, so the next item's first score MMAs run under the drain.
 template <bool kCausal>
 __global__ void __launch_bounds__(kFwdThreads, 1)
@@ -80,7 +80,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     constexpr int BK = kFwdKeys;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
-    uint64_t* q_ready = bars + 0;    // warpgroup 0 has put the item's Q tile into TMEM
+    uint64_t* q_ready = bars + 0;    // both warpgroups have put their halves of the item's Q tile into TMEM
     uint64_t* k_full = bars + 1;     // [3]
     uint64_t* k_empty = bars + 4;    // [3]
     uint64_t* v_full = bars + 7;     // [3]
@@ -107,7 +107,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        mbar_init(q_ready, 128);
+        mbar_init(q_ready, 256);
         for (int s = 0; s < 3; ++s) {
             mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); mbar_init(&s_full[s], 1);
             mbar_init(&p_full[s], 128);
@@ -323,21 +323,23 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             int q0, head, n_kv, row_base, S_seq;
             item_geometry(item, q0, head, n_kv, row_base, S_seq);
             const int sq_idx = q0 + row;              // query index within the sequence
-            if (g == 0) {   // this thread's query row (192 bf16 = 96 packed words) goes to TMEM once, as the A operand of S
-                            // (the previous item's MMAs, which read the old tile, are known complete)
+            {   // The item's query tile goes to TMEM once, as the A operand of S (the previous item's MMAs, which read
+                // the old tile, are known complete).  Both groups own every TMEM lane (warps w and w + 4 address the same
+                // 32 lanes), so each takes half of the row: group g the 48 packed words [48g, 48g + 48).  A lane reads
+                // its own row and rows are kilobytes apart, so every 16-byte load is a round trip to L2 or HBM that
+                // touches 32 different lines per instruction: all of a thread's loads are issued before the first is
+                // used (three dependent rounds of eight cost 7.5 K clocks per item, one round far less).
                 const bool q_valid = sq_idx < S_seq;
-                const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(row_base + sq_idx) * args.h + head) * 192);
-#pragma unroll 1
-                for (int c = 0; c < 3; ++c) {
-                    uint32_t w[32];
+                const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(row_base + sq_idx) * args.h + head) * 192) + g * 12;
+                uint4 x[12];
 #pragma unroll
-                    for (int v = 0; v < 8; ++v) {
-                        const uint4 x = q_valid ? src[c * 8 + v] : make_uint4(0u, 0u, 0u, 0u);
-                        w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
-                    }
-                    __syncwarp();
-                    tmem_st_x32(tmem_q + lane_addr + c * 32, w);
-                }
+                for (int v = 0; v < 12; ++v) x[v] = q_valid ? src[v] : make_uint4(0u, 0u, 0u, 0u);
+                uint32_t w[48];
+#pragma unroll
+                for (int v = 0; v < 12; ++v) { w[v * 4] = x[v].x; w[v * 4 + 1] = x[v].y; w[v * 4 + 2] = x[v].z; w[v * 4 + 3] = x[v].w; }
+                __syncwarp();
+                tmem_st_x32(tmem_q + lane_addr + g * 48, w);
+                tmem_st_x16(tmem_q + lane_addr + g * 48 + 32, w + 32);
                 tmem_st_wait();
                 tc_fence_before_sync();
                 mbar_arrive(q_ready);
