@@ -478,6 +478,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             const bool valid = t_idx < seq.seq_len;
             __nv_bfloat16* dkv_row = args.dkv + static_cast<size_t>(t_row) * args.h * 256 + head * 256;
             float* dkr_row = args.dkpe_acc + static_cast<size_t>(t_row) * 64;
+            const bool wide = aligned32_dev(args.dkv);     // rows are h * 512 bytes: every chunk is 32-byte aligned if the base is
             // 10 chunks of 32 columns: dK nope (0..3), dK rope (4..5), dV (6..9; dV follows dK in TMEM).
             // Group 0 drains chunks 0..4, group 1 chunks 5..9.
 #pragma unroll 1
@@ -502,14 +503,16 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 } else {
                     const float mul = c < 4 ? args.scale : 1.0f;
                     __nv_bfloat16* dst = dkv_row + (c < 4 ? c * 32 : 128 + (c - 6) * 32);
+                    uint32_t w[16];
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]) * mul, __uint_as_float(r[v * 8 + 1]) * mul);
-                        w.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]) * mul, __uint_as_float(r[v * 8 + 3]) * mul);
-                        w.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]) * mul, __uint_as_float(r[v * 8 + 5]) * mul);
-                        w.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]) * mul, __uint_as_float(r[v * 8 + 7]) * mul);
-                        reinterpret_cast<uint4*>(dst)[v] = w;
+                    for (int v = 0; v < 16; ++v) w[v] = pack_bf16x2(__uint_as_float(r[2 * v]) * mul, __uint_as_float(r[2 * v + 1]) * mul);
+                    if (wide) {          // two 32-byte stores per 32-column chunk
+                        st_global_v8(dst, w);
+                        st_global_v8(dst + 16, w + 8);
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            reinterpret_cast<uint4*>(dst)[v] = make_uint4(w[v * 4], w[v * 4 + 1], w[v * 4 + 2], w[v * 4 + 3]);
                     }
                 }
             }
@@ -760,6 +763,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             if (!mbar_wait_warp(acc_full, n_done & 1u, abort_flag, args.status, 0x92)) return false;
             tc_fence_after_sync();
             __nv_bfloat16* dst = args.dq + (static_cast<size_t>(s_idx) * args.h + head) * 192;
+            const bool wide = aligned32_dev(args.dq);      // rows are 384 bytes: every chunk is 32-byte aligned if the base is
 #pragma unroll 1
             for (int c = g * 3; c < g * 3 + 3; ++c) {
                 uint32_t r[32];
@@ -768,14 +772,16 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 tmem_ld_wait();
                 if (!valid) continue;
                 if (!device_check(head < args.h && aligned16_dev(dst), args.status, 0xE50000u | c)) continue;
+                uint32_t w[16];
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    uint4 w;
-                    w.x = pack_bf16x2(__uint_as_float(r[v * 8 + 0]) * args.scale, __uint_as_float(r[v * 8 + 1]) * args.scale);
-                    w.y = pack_bf16x2(__uint_as_float(r[v * 8 + 2]) * args.scale, __uint_as_float(r[v * 8 + 3]) * args.scale);
-                    w.z = pack_bf16x2(__uint_as_float(r[v * 8 + 4]) * args.scale, __uint_as_float(r[v * 8 + 5]) * args.scale);
-                    w.w = pack_bf16x2(__uint_as_float(r[v * 8 + 6]) * args.scale, __uint_as_float(r[v * 8 + 7]) * args.scale);
-                    reinterpret_cast<uint4*>(dst + c * 32)[v] = w;
+                for (int v = 0; v < 16; ++v) w[v] = pack_bf16x2(__uint_as_float(r[2 * v]) * args.scale, __uint_as_float(r[2 * v + 1]) * args.scale);
+                if (wide) {          // two 32-byte stores per 32-column chunk
+                    st_global_v8(dst + c * 32, w);
+                    st_global_v8(dst + c * 32 + 16, w + 8);
+                } else {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v)
+                        reinterpret_cast<uint4*>(dst + c * 32)[v] = make_uint4(w[v * 4], w[v * 4 + 1], w[v * 4 + 2], w[v * 4 + 3]);
                 }
             }
             __syncwarp();
@@ -800,11 +806,17 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 // last dP MMA has completed: this group waited for it before writing its last dS)
                 uint32_t w[32];
                 if (valid) {
-                    const uint4* src = reinterpret_cast<const uint4*>(args.dout + (static_cast<size_t>(s_row) * args.h + head) * 128 + g * 64);
+                    const __nv_bfloat16* srcb = args.dout + (static_cast<size_t>(s_row) * args.h + head) * 128 + g * 64;
+                    if (aligned32_dev(args.dout)) {          // four 32-byte loads (rows are 256 bytes)
 #pragma unroll
-                    for (int v = 0; v < 8; ++v) {
-                        const uint4 x = src[v];
-                        w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
+                        for (int v = 0; v < 4; ++v) ld_global_v8(srcb + v * 16, w + v * 8);
+                    } else {
+                        const uint4* src = reinterpret_cast<const uint4*>(srcb);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            const uint4 x = src[v];
+                            w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
+                        }
                     }
                 } else {
 #pragma unroll

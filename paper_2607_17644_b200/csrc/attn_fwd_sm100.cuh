@@ -289,6 +289,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             tc_fence_after_sync();
             const float inv_l = 1.0f / l_run;
             __nv_bfloat16* dst = args.out + (static_cast<size_t>(sq_idx) * args.h + head) * 128;
+            const bool wide = aligned32_dev(args.out);
 #pragma unroll 1
             for (int c = 2 * g; c < 2 * g + 2; ++c) {
                 uint32_t o[32];
@@ -296,14 +297,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 tmem_ld_x32(tmem_o + lane_addr + c * 32, o);
                 tmem_ld_wait();
                 if (valid && device_check(aligned16_dev(dst) && head < args.h && sq_idx >= 0, args.status, 0xE30000u | c)) {
+                    uint32_t w[16];
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(o[v * 8 + 0]) * inv_l, __uint_as_float(o[v * 8 + 1]) * inv_l);
-                        w.y = pack_bf16x2(__uint_as_float(o[v * 8 + 2]) * inv_l, __uint_as_float(o[v * 8 + 3]) * inv_l);
-                        w.z = pack_bf16x2(__uint_as_float(o[v * 8 + 4]) * inv_l, __uint_as_float(o[v * 8 + 5]) * inv_l);
-                        w.w = pack_bf16x2(__uint_as_float(o[v * 8 + 6]) * inv_l, __uint_as_float(o[v * 8 + 7]) * inv_l);
-                        reinterpret_cast<uint4*>(dst + c * 32)[v] = w;
+                    for (int v = 0; v < 16; ++v) w[v] = pack_bf16x2(__uint_as_float(o[2 * v]) * inv_l, __uint_as_float(o[2 * v + 1]) * inv_l);
+                    if (wide) {          // two 32-byte stores per 32-column chunk (rows are 256 bytes)
+                        st_global_v8(dst + c * 32, w);
+                        st_global_v8(dst + c * 32 + 16, w + 8);
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            reinterpret_cast<uint4*>(dst + c * 32)[v] = make_uint4(w[v * 4], w[v * 4 + 1], w[v * 4 + 2], w[v * 4 + 3]);
                     }
                 }
             }
@@ -331,12 +334,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 // used (three dependent rounds of eight cost 7.5 K clocks per item, one round far less).
                 const bool q_valid = sq_idx < S_seq;
                 const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(row_base + sq_idx) * args.h + head) * 192) + g * 12;
-                uint4 x[12];
-#pragma unroll
-                for (int v = 0; v < 12; ++v) x[v] = q_valid ? src[v] : make_uint4(0u, 0u, 0u, 0u);
                 uint32_t w[48];
+                if (!q_valid) {
 #pragma unroll
-                for (int v = 0; v < 12; ++v) { w[v * 4] = x[v].x; w[v * 4 + 1] = x[v].y; w[v * 4 + 2] = x[v].z; w[v * 4 + 3] = x[v].w; }
+                    for (int v = 0; v < 48; ++v) w[v] = 0u;
+                } else if (aligned32_dev(args.q)) {      // six 32-byte loads (half a row is 192 bytes)
+#pragma unroll
+                    for (int v = 0; v < 6; ++v) ld_global_v8(src + 2 * v, w + 8 * v);
+                } else {
+                    uint4 x[12];
+#pragma unroll
+                    for (int v = 0; v < 12; ++v) x[v] = src[v];
+#pragma unroll
+                    for (int v = 0; v < 12; ++v) { w[v * 4] = x[v].x; w[v * 4 + 1] = x[v].y; w[v * 4 + 2] = x[v].z; w[v * 4 + 3] = x[v].w; }
+                }
                 __syncwarp();
                 tmem_st_x32(tmem_q + lane_addr + g * 48, w);
                 tmem_st_x16(tmem_q + lane_addr + g * 48 + 32, w + 32);

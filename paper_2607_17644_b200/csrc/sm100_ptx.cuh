@@ -457,6 +457,21 @@ __device__ __forceinline__ void mma_commit_pair(uint64_t* bar, uint16_t cta_mask
 // ------------------------------------------------------------------------------------------------
 // Small helpers
 // ------------------------------------------------------------------------------------------------
+// 256-bit global accesses (sm_100): a lane moves 32 contiguous bytes per instruction.  The row-per-lane epilogues
+// and operand stagings of the attention kernels touch 32 different lines per instruction whatever its width, so
+// halving the instruction count halves what they cost the load/store unit.  The address must be 32-byte aligned.
+__device__ __forceinline__ void st_global_v8(void* addr, const uint32_t* r) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]),
+                 "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void ld_global_v8(const void* addr, uint32_t* r) {
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "l"(addr));
+}
+__device__ __forceinline__ bool aligned32_dev(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0u; }
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), .y = hi
     return *reinterpret_cast<uint32_t*>(&v);
