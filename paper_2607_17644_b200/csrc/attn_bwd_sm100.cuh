@@ -293,32 +293,29 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             constexpr uint32_t idesc_st = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: both K-major
             constexpr uint32_t idesc_dv = make_idesc_bf16(128, 128, 0, 1);   // dV: A = P^T (TMEM), B = dO MN-major
             constexpr uint32_t idesc_dk = make_idesc_bf16(128, 192, 0, 1);   // dK: A = dS^T (TMEM), B = Q MN-major
-            const uint32_t sk = smem_u32(smem + L::kK), sv = smem_u32(smem + L::kV), sdo = smem_u32(smem + L::kDo);
-            auto stage_q = [&](uint32_t T) { return smem_u32(smem + L::kQ + (T % L::kQStages) * 3 * L::kSlab); };
+            // Every batch of MMAs is one asm chain (sm100_ptx.cuh): descriptors as a constant upper word and a lower
+            // word that steps by immediates, commits inside the chain.  This lane's instructions cost four to six
+            // clocks each beside the consumer warps and sit on the path S^T -> P^T -> dP^T -> dS^T of every tile.
+            const uint64_t dk_k = desc_k_major(smem_u32(smem + L::kK)), dk_v = desc_k_major(smem_u32(smem + L::kV));
+            const uint64_t dk_do = desc_k_major(smem_u32(smem + L::kDo)), dk_q0 = desc_k_major(smem_u32(smem + L::kQ));
+            const uint64_t dm_do = desc_mn_major(smem_u32(smem + L::kDo), L::kSlab), dm_q0 = desc_mn_major(smem_u32(smem + L::kQ), L::kSlab);
+            constexpr uint32_t kQStageLo = (3 * L::kSlab) >> 4;      // a Q stage further on, in descriptor units
+            const uint32_t bars_a = smem_u32(bars);
+            auto bar_a = [&](const uint64_t* b) { return bars_a + static_cast<uint32_t>(b - bars) * 8u; };
             auto issue_st = [&](uint32_t T, bool first_of_cta) -> bool {   // S^T(T) = K Q^T into X
                 if (!mbar_wait(&q_full[T % L::kQStages], (T / L::kQStages) & 1u, abort_flag, args.status, 0x52)) return false;
                 // X still holds dP^T of the previous tile until both groups have loaded it
                 if (!first_of_cta && !mbar_wait(dp_read, (T - 1) & 1u, abort_flag, args.status, 0x57)) return false;
                 tc_fence_after_sync();
-                const uint32_t sq = stage_q(T);
-#pragma unroll
-                for (int kk = 0; kk < 12; ++kk) {
-                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
-                    mma_ss(tmem_base, desc_k_major(sk + off), desc_k_major(sq + off), idesc_st, kk > 0 ? 1u : 0u);
-                }
-                mma_commit(st_full);
+                mma_ss_chain12_k128(tmem_base, desc_lo(dk_k), desc_hi(dk_k), desc_lo(dk_q0) + (T % L::kQStages) * kQStageLo, desc_hi(dk_q0),
+                                    idesc_st, bar_a(st_full));
                 return true;
             };
             auto issue_dp = [&](uint32_t T) -> bool {     // dP^T(T) = V dO^T over X once S^T(T) was read
                 if (!mbar_wait(st_read, T & 1u, abort_flag, args.status, 0x53)) return false;
                 if (!mbar_wait(do_full, T & 1u, abort_flag, args.status, 0x55)) return false;
                 tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
-                    mma_ss(tmem_base, desc_k_major(sv + off), desc_k_major(sdo + off), idesc_st, kk > 0 ? 1u : 0u);
-                }
-                mma_commit(dp_full);
+                mma_ss_chain8_k128(tmem_base, desc_lo(dk_v), desc_hi(dk_v), desc_lo(dk_do), desc_hi(dk_do), idesc_st, bar_a(dp_full));
                 return true;
             };
             uint32_t T0 = 0;
@@ -341,12 +338,8 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     if (ok && j == 0 && n > 0) ok = mbar_wait(acc_empty, (n - 1) & 1u, abort_flag, args.status, 0x56);
                     if (!ok) break;
                     tc_fence_after_sync();
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        mma_ts(tmem_dv, tmem_y + kk * 8, desc_mn_major(sdo + kk * 2048, L::kSlab), idesc_dv,
-                               (j > 0 || kk > 0) ? 1u : 0u);
-                    mma_commit(do_empty);
-                    mma_commit(dv_done);
+                    mma_ts_chain8_mn(tmem_dv, tmem_y, desc_lo(dm_do), desc_hi(dm_do), idesc_dv, static_cast<uint32_t>(j),
+                                     bar_a(do_empty), bar_a(dv_done));
                     if (j + 1 < n_iter) {
                         ok = issue_st(T + 1, false);
                         if (!ok) break;
@@ -355,13 +348,8 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     ok = mbar_wait(ds_full, T & 1u, abort_flag, args.status, 0x51);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t sq = stage_q(T);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        mma_ts(tmem_dk, tmem_y + kk * 8, desc_mn_major(sq + kk * 2048, L::kSlab), idesc_dk,
-                               (j > 0 || kk > 0) ? 1u : 0u);
-                    mma_commit(&q_empty[T % L::kQStages]);
-                    mma_commit(dk_done);
+                    mma_ts_chain8_mn(tmem_dk, tmem_y, desc_lo(dm_q0) + (T % L::kQStages) * kQStageLo, desc_hi(dm_q0), idesc_dk,
+                                     static_cast<uint32_t>(j), bar_a(&q_empty[T % L::kQStages]), bar_a(dk_done));
                     if (j + 1 < n_iter) {
                         ok = issue_dp(T + 1);
                         if (ok && j + 2 == n_iter) mma_commit(kv_empty);   // that was the item's last read of K and V
@@ -679,31 +667,24 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         if (elect_one()) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);    // S: both K-major; dP: A from TMEM
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, 192, 0, 1);   // dQ: A = dS (TMEM), B = K MN-major
-            const uint32_t sq = smem_u32(smem + L::kQ);
-            const uint32_t sv = smem_u32(smem + L::kV);
-            auto stage_k = [&](uint32_t T) { return smem_u32(smem + L::kK + (T % kDqKStages) * 3 * L::kSlab); };
+            // (one asm chain per batch of MMAs, as in the dK/dV kernel)
+            const uint64_t dk_q = desc_k_major(smem_u32(smem + L::kQ)), dk_v = desc_k_major(smem_u32(smem + L::kV));
+            const uint64_t dk_k0 = desc_k_major(smem_u32(smem + L::kK)), dm_k0 = desc_mn_major(smem_u32(smem + L::kK), L::kSlab);
+            constexpr uint32_t kKStageLo = (3 * L::kSlab) >> 4;      // a K stage further on, in descriptor units
+            const uint32_t bars_a = smem_u32(bars);
+            auto bar_a = [&](const uint64_t* b) { return bars_a + static_cast<uint32_t>(b - bars) * 8u; };
             auto issue_s = [&](uint32_t T) -> bool {      // S(T) = Q K^T
                 if (!mbar_wait(&k_full[T % kDqKStages], (T / kDqKStages) & 1u, abort_flag, args.status, 0x82)) return false;
                 if (T > 0 && !mbar_wait(s_read, (T - 1) & 1u, abort_flag, args.status, 0x83)) return false;
                 tc_fence_after_sync();
-                const uint32_t sk = stage_k(T);
-#pragma unroll
-                for (int kk = 0; kk < 12; ++kk) {
-                    const uint32_t off = (kk >> 2) * L::kSlab + (kk & 3) * 32;
-                    mma_ss(tmem_base, desc_k_major(sq + off), desc_k_major(sk + off), idesc_s, kk > 0 ? 1u : 0u);
-                }
-                mma_commit(s_full);
+                mma_ss_chain12_k128(tmem_base, desc_lo(dk_q), desc_hi(dk_q), desc_lo(dk_k0) + (T % kDqKStages) * kKStageLo, desc_hi(dk_k0),
+                                    idesc_s, bar_a(s_full));
                 return true;
             };
             auto issue_dp = [&](uint32_t T) -> bool {     // dP(T) = dO V^T; overwrites dS(T-1), whose reader was issued earlier
                 if (!mbar_wait(v_full, T & 1u, abort_flag, args.status, 0x84)) return false;
                 tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    mma_ts(tmem_dp, tmem_do + kk * 8, desc_k_major(sv + (kk >> 2) * L::kSlab + (kk & 3) * 32), idesc_s,
-                           kk > 0 ? 1u : 0u);
-                mma_commit(v_empty);
-                mma_commit(dp_full);
+                mma_ts_chain8_k128(tmem_dp, tmem_do, desc_lo(dk_v), desc_hi(dk_v), idesc_s, bar_a(v_empty), bar_a(dp_full));
                 return true;
             };
             uint32_t T0 = 0;
@@ -731,12 +712,8 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     if (ok && j == 0 && n > 0) ok = mbar_wait(acc_empty, (n - 1) & 1u, abort_flag, args.status, 0x86);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t sk = stage_k(T);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        mma_ts(tmem_dq, tmem_dp + (kk >> 2) * 64 + (kk & 3) * 8, desc_mn_major(sk + kk * 2048, L::kSlab),
-                               idesc_dq, (j > 0 || kk > 0) ? 1u : 0u);
-                    mma_commit(&k_empty[T % kDqKStages]);
+                    mma_ts_chain8_mn_split(tmem_dq, tmem_dp, desc_lo(dm_k0) + (T % kDqKStages) * kKStageLo, desc_hi(dm_k0), idesc_dq,
+                                           static_cast<uint32_t>(j), bar_a(&k_empty[T % kDqKStages]));
                     if (j + 1 < n_iter) ok = issue_dp(T + 1);
                 }
                 if (ok) mma_commit(acc_full);

@@ -211,15 +211,16 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             // while the MMAs block, and the bounded wait runs only when the probe came back false.
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, BK, 0, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, 0, 1);
+            const uint64_t desc_k0 = desc_k_major(smem_u32(smem + L::kK));
+            const uint64_t desc_v0 = desc_mn_major(smem_u32(smem + L::kV), L::kSlab);
+            const uint32_t k_lo0 = static_cast<uint32_t>(desc_k0), k_hi = static_cast<uint32_t>(desc_k0 >> 32);
+            const uint32_t v_lo0 = static_cast<uint32_t>(desc_v0), v_hi = static_cast<uint32_t>(desc_v0 >> 32);
+            constexpr uint32_t kKStageLo = (3 * L::kSlab) >> 4, kVStageLo = (2 * L::kSlab) >> 4;
+            const uint32_t bars_a = smem_u32(bars);
             auto qk_mmas = [&](uint32_t T) {
                 const uint32_t s = T % kFwdStages;
-                const uint32_t sk = smem_u32(smem + L::kK + s * 3 * L::kSlab);
-#pragma unroll
-                for (int kk = 0; kk < 12; ++kk)
-                    mma_ts(tmem_base + s * BK, tmem_q + kk * 8, desc_k_major(sk + (kk >> 2) * L::kSlab + (kk & 3) * 32),
-                           idesc_qk, kk > 0 ? 1u : 0u);
-                mma_commit(&k_empty[s]);
-                mma_commit(&s_full[s]);
+                mma_ts_chain_qk96_head(tmem_base + s * BK, tmem_q, k_lo0 + s * kKStageLo, k_hi, idesc_qk);
+                mma_ts_chain_qk96_tail(tmem_base + s * BK, tmem_q, k_lo0 + s * kKStageLo, k_hi, idesc_qk, bars_a + (4u + s) * 8u, bars_a + (13u + s) * 8u);
             };
             uint32_t T0 = 0;
             bool ok = true;
@@ -248,13 +249,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     tc_fence_after_sync();
                     const bool more = j + 3 < n_kv;
                     const bool k_ok = more && mbar_try_wait(&k_full[s], ph ^ 1u);   // K of tile T+3 lands in the stage tile T left
-                    const uint32_t sv = smem_u32(smem + L::kV + s * 2 * L::kSlab);
-#pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)   // A = P: packed bf16, 8 TMEM columns per 16 keys
-                        mma_ts(tmem_o, tmem_base + s * BK + kk * 8, desc_mn_major(sv + kk * 2048, L::kSlab), idesc_pv,
-                               (j > 0 || kk > 0) ? 1u : 0u);
-                    mma_commit(&v_empty[s]);
-                    mma_commit(&pv_done[g]);
+                    mma_ts_chain_pv96_head(tmem_o, tmem_base + s * BK, v_lo0 + s * kVStageLo, v_hi, idesc_pv, static_cast<uint32_t>(j));
+                    mma_ts_chain_pv96_tail(tmem_o, tmem_base + s * BK, v_lo0 + s * kVStageLo, v_hi, idesc_pv, bars_a + (10u + s) * 8u, bars_a + (19u + g) * 8u);
                     v_ok = p_ok = false;
                     if (more) {
                         if (!k_ok) ok = mbar_wait(&k_full[s], ph ^ 1u, abort_flag, args.status, 0x23);

@@ -292,6 +292,146 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Chains of MMAs from ONE asm block.  The issuing lane shares its scheduler with two busy softmax warps and runs at
+// four to six clocks per instruction, so the ten or so instructions that the compiler spends on every separately
+// written MMA (descriptor arithmetic in 64 bits, predicate set-up, operand moves) are time the tensor pipe
+// idles: measured, the lane's instruction count sets the tile period once it exceeds the MMAs' own time.  Here a
+// step costs two additions and the MMA: the descriptor's upper word is constant and its lower word (start
+// address in 16-byte units, below the leading-offset field) is advanced by an immediate.
+#define LAGA_MMA_TS_STEP(AOFF, BOFF, P)                                                       \
+    "add.u32 a, %1, " #AOFF ";\n\tadd.u32 lo, %2, " #BOFF ";\n\tmov.b64 desc, {lo, %3};\n\t"  \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], desc, %4, " #P ";\n\t"
+// Each chain comes in two parts, so that the lane can put the bookkeeping that follows a chain BEFORE the
+// chain's last MMAs: it then runs while the pipe still has those queued (the queue holds only two to four MMAs).
+#define LAGA_MMA_COMMIT2(B0, B1)                                                                               \
+    "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [" #B0 "];\n\t"                      \
+    "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [" #B1 "];\n\t"
+// S = Q K^T for one 96-key tile: twelve K steps, A = Q from TMEM (8 columns per step), B = a K-major key tile of
+// three slabs of 96 rows (12288 bytes = 768 descriptor units each; 32 bytes = 2 units per step inside a slab).
+// Head: the steps of slabs 0 and 1 (the first overwrites S).  Tail: slab 2, then commits to two mbarriers
+// (shared-memory addresses).
+__device__ __forceinline__ void mma_ts_chain_qk96_head(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 a, lo;\n\t.reg .b64 desc;\n\t"
+        "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_TS_STEP(0, 0, p0) LAGA_MMA_TS_STEP(8, 2, p1) LAGA_MMA_TS_STEP(16, 4, p1) LAGA_MMA_TS_STEP(24, 6, p1)
+        LAGA_MMA_TS_STEP(32, 768, p1) LAGA_MMA_TS_STEP(40, 770, p1) LAGA_MMA_TS_STEP(48, 772, p1) LAGA_MMA_TS_STEP(56, 774, p1)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_chain_qk96_tail(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                       uint32_t bar0, uint32_t bar1) {
+    asm volatile(
+        "{\n\t.reg .pred p1;\n\t.reg .b32 a, lo;\n\t.reg .b64 desc;\n\t"
+        "setp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_TS_STEP(64, 1536, p1) LAGA_MMA_TS_STEP(72, 1538, p1) LAGA_MMA_TS_STEP(80, 1540, p1) LAGA_MMA_TS_STEP(88, 1542, p1)
+        LAGA_MMA_COMMIT2(%5, %6)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(bar0), "r"(bar1)
+        : "memory");
+}
+// O (+)= P V for one 96-key tile: six K steps, A = P from TMEM (8 columns per step), B = an MN-major value tile
+// (16 key rows = 2048 bytes = 128 descriptor units per step).  Head: three steps, accumulate_first == 0
+// overwrites O.  Tail: three steps, then commits to two mbarriers.
+__device__ __forceinline__ void mma_ts_chain_pv96_head(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                       uint32_t accumulate_first) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 a, lo;\n\t.reg .b64 desc;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_TS_STEP(0, 0, p0) LAGA_MMA_TS_STEP(8, 128, p1) LAGA_MMA_TS_STEP(16, 256, p1)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_chain_pv96_tail(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                       uint32_t bar0, uint32_t bar1) {
+    asm volatile(
+        "{\n\t.reg .pred p1;\n\t.reg .b32 a, lo;\n\t.reg .b64 desc;\n\t"
+        "setp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_TS_STEP(24, 384, p1) LAGA_MMA_TS_STEP(32, 512, p1) LAGA_MMA_TS_STEP(40, 640, p1)
+        LAGA_MMA_COMMIT2(%5, %6)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(bar0), "r"(bar1)
+        : "memory");
+}
+
+// The chains of the backward kernels (128-row slabs: 16384 bytes = 1024 descriptor units per 64 elements of K).
+#define LAGA_MMA_SS_STEP(OFF, P)                                                                                  \
+    "add.u32 lo, %1, " #OFF ";\n\tmov.b64 da, {lo, %2};\n\tadd.u32 lo, %3, " #OFF ";\n\tmov.b64 db, {lo, %4};\n\t"  \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, " #P ";\n\t"
+#define LAGA_MMA_COMMIT1(B0) "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [" #B0 "];\n\t"
+// D = A B^T, both operands K-major tiles of 128 rows in shared memory, 192 deep (twelve steps); then one commit.
+__device__ __forceinline__ void mma_ss_chain12_k128(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                    uint32_t idesc, uint32_t bar0) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 lo;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_SS_STEP(0, p0) LAGA_MMA_SS_STEP(2, p1) LAGA_MMA_SS_STEP(4, p1) LAGA_MMA_SS_STEP(6, p1)
+        LAGA_MMA_SS_STEP(1024, p1) LAGA_MMA_SS_STEP(1026, p1) LAGA_MMA_SS_STEP(1028, p1) LAGA_MMA_SS_STEP(1030, p1)
+        LAGA_MMA_SS_STEP(2048, p1) LAGA_MMA_SS_STEP(2050, p1) LAGA_MMA_SS_STEP(2052, p1) LAGA_MMA_SS_STEP(2054, p1)
+        LAGA_MMA_COMMIT1(%6)
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(bar0)
+        : "memory");
+}
+// The same, 128 deep (eight steps).
+__device__ __forceinline__ void mma_ss_chain8_k128(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                   uint32_t idesc, uint32_t bar0) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 lo;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_SS_STEP(0, p0) LAGA_MMA_SS_STEP(2, p1) LAGA_MMA_SS_STEP(4, p1) LAGA_MMA_SS_STEP(6, p1)
+        LAGA_MMA_SS_STEP(1024, p1) LAGA_MMA_SS_STEP(1026, p1) LAGA_MMA_SS_STEP(1028, p1) LAGA_MMA_SS_STEP(1030, p1)
+        LAGA_MMA_COMMIT1(%6)
+        "}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(bar0)
+        : "memory");
+}
+// D (+)= A B: A = packed bf16 in TMEM (8 columns per step), B = an MN-major tile of 128 rows of K (16 rows = 2048
+// bytes = 128 units per step), eight steps; accumulate_first == 0 overwrites D; then two commits.
+__device__ __forceinline__ void mma_ts_chain8_mn(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                 uint32_t accumulate_first, uint32_t bar0, uint32_t bar1) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 a, lo;\n\t.reg .b64 desc;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_TS_STEP(0, 0, p0) LAGA_MMA_TS_STEP(8, 128, p1) LAGA_MMA_TS_STEP(16, 256, p1) LAGA_MMA_TS_STEP(24, 384, p1)
+        LAGA_MMA_TS_STEP(32, 512, p1) LAGA_MMA_TS_STEP(40, 640, p1) LAGA_MMA_TS_STEP(48, 768, p1) LAGA_MMA_TS_STEP(56, 896, p1)
+        LAGA_MMA_COMMIT2(%6, %7)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "r"(bar0), "r"(bar1)
+        : "memory");
+}
+// The same with A in two blocks of 32 columns that lie 64 columns apart (the dQ kernel's dS); then one commit.
+__device__ __forceinline__ void mma_ts_chain8_mn_split(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                       uint32_t accumulate_first, uint32_t bar0) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 a, lo;\n\t.reg .b64 desc;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_TS_STEP(0, 0, p0) LAGA_MMA_TS_STEP(8, 128, p1) LAGA_MMA_TS_STEP(16, 256, p1) LAGA_MMA_TS_STEP(24, 384, p1)
+        LAGA_MMA_TS_STEP(64, 512, p1) LAGA_MMA_TS_STEP(72, 640, p1) LAGA_MMA_TS_STEP(80, 768, p1) LAGA_MMA_TS_STEP(88, 896, p1)
+        LAGA_MMA_COMMIT1(%6)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "r"(bar0)
+        : "memory");
+}
+// D = A B^T: A = packed bf16 in TMEM (8 columns per step), B = a K-major tile of 128 rows, 128 deep (eight steps);
+// overwrites D; then two commits.
+__device__ __forceinline__ void mma_ts_chain8_k128(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                   uint32_t bar0, uint32_t bar1) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b32 a, lo;\n\t.reg .b64 desc;\n\t"
+        "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+        LAGA_MMA_TS_STEP(0, 0, p0) LAGA_MMA_TS_STEP(8, 2, p1) LAGA_MMA_TS_STEP(16, 4, p1) LAGA_MMA_TS_STEP(24, 6, p1)
+        LAGA_MMA_TS_STEP(32, 1024, p1) LAGA_MMA_TS_STEP(40, 1026, p1) LAGA_MMA_TS_STEP(48, 1028, p1) LAGA_MMA_TS_STEP(56, 1030, p1)
+        LAGA_MMA_COMMIT2(%5, %6)
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(bar0), "r"(bar1)
+        : "memory");
+}
+__device__ __forceinline__ uint32_t desc_lo(uint64_t desc) { return static_cast<uint32_t>(desc); }
+__device__ __forceinline__ uint32_t desc_hi(uint64_t desc) { return static_cast<uint32_t>(desc >> 32); }
+
 // Arrive (count 1) on `bar` once every MMA this thread issued so far has completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
