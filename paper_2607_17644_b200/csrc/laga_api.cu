@@ -111,6 +111,7 @@ void init_device(DeviceInfo* info, int dev) {
     bool ok = allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, false, true, EPI_BF16>, G::kTotalBytes) &&
               allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, false, false, EPI_BF16>, G::kTotalBytes) &&
               allow_smem(gemm_pair_sm100_kernel<128, kGemmStages, false, false, EPI_BF16>, GemmPairSmem<128, kGemmStages>::kTotalBytes) &&
+              allow_smem(gemm_pair_sm100_kernel<128, kGemmStages, false, true, EPI_BF16>, GemmPairSmem<128, kGemmStages>::kTotalBytes) &&
               allow_smem(gemm_pair_sm100_kernel<256, kGemmStages, true, true, EPI_ATOMIC_F32>, G::kTotalBytes) &&
               allow_smem(gemm_sm100_kernel<128, 4, false, true, EPI_BF16>, GemmSmem<128, 4>::kTotalBytes) &&
               allow_smem(attn_absorbed_fwd_sm100_kernel<true>, AttnAbsorbedSmem::kTotalBytes) &&
@@ -300,9 +301,10 @@ WorkSchedule make_schedule(int n_tiles, int S, int h, unsigned* counter, const i
 
 // ---- y[M, N] = x[M, K] . W[K, N]: Algorithm 1 step 4 (KV = c_kv W, K = d_c) and the dense projections of
 // ---- steps 1 and 7 through laga_linear --------------------------------------------------------------
-int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
-                      cudaStream_t stream, bool overlap = false, int K = kDc) {
-    constexpr int BN = 256, STAGES = kGemmStages;
+template <int BN>
+int launch_up_project_bn(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
+                         cudaStream_t stream, bool overlap, int K) {
+    constexpr int STAGES = kGemmStages;
     auto kernel = gemm_pair_sm100_kernel<BN, STAGES, false, true, EPI_BF16>;
     using L = GemmPairSmem<BN, STAGES>;
     CUtensorMap ta, tb;
@@ -314,6 +316,15 @@ int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, u
     dim3 grid(pair_grid(((N + BN - 1) / BN) * ((S + 255) / 256)), 1, 1);
     { ScopedKernelEvents ev(LAGA_KERNEL_UP_PROJECT, stream); launch_kernel(kernel, grid, dim3(192), L::kTotalBytes, stream, overlap, ta, tb, tc, a); }
     return launch_status();
+}
+int launch_up_project(const void* c_kv, const void* w, int S, int N, void* kv, unsigned* status,
+                      cudaStream_t stream, bool overlap = false, int K = kDc) {
+    // As for dc_kv below: when 256-column tiles do not even give every CTA pair one tile, tiles of half the width
+    // do better (S = 512, N = 512: 12.7 -> 10.7 us).  Where they only fill the LAST wave better they lose: at
+    // S = 4096, N = 4096 (256 tiles on 74 pairs, four waves for 3.46) 26.8 us against 24.0.
+    const int tiles_256 = ((N + 255) / 256) * ((S + 255) / 256);
+    if (tiles_256 < sm_count() / 2) return launch_up_project_bn<128>(c_kv, w, S, N, kv, status, stream, overlap, K);
+    return launch_up_project_bn<256>(c_kv, w, S, N, kv, status, stream, overlap, K);
 }
 
 // ---- Section 5.2, back through step 4 -----------------------------------------------------------
