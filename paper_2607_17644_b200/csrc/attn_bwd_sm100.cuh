@@ -50,8 +50,13 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __r
                  const float* __restrict__ lse, int S, int h, int S_pad, float* __restrict__ stat_l2,
                  float* __restrict__ stat_delta, float4* __restrict__ zero_begin, size_t zero_count,
                  const int2* __restrict__ seqs, int n_seqs) {
+    // This kernel depends on nothing the kernel launched before it in the same call produces (that is the
+    // recomputed up-projection: it writes K/V, this reads out / dout / lse and writes the statistics and the
+    // rope-gradient accumulator), so it does not wait for it before working: launched with programmatic stream
+    // serialization it runs BESIDE the up-projection (bound by HBM, the other by the tensor pipe).  It waits at
+    // its END instead, so that its own completion still implies the completion of everything before it -- the
+    // kernels after it rely on that.
     grid_launch_dependents();
-    grid_dependency_wait();
     // Also clears the fp32 buffer the dK/dV kernel accumulates the rope-column key gradients into
     // (zero_count float4 elements): one launch less than a separate memset.
     for (size_t z = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; z < zero_count;
@@ -97,6 +102,7 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __r
         stat_l2[static_cast<size_t>(i) * S_pad + s] = valid ? lse[static_cast<size_t>(row) * h + i] * 1.4426950408889634f : INFINITY;
         stat_delta[static_cast<size_t>(i) * S_pad + s] = valid ? acc : 0.f;
     }
+    grid_dependency_wait();
 }
 
 // dk_pe[t, r] is the sum over heads of the rope-column key gradients (Section 5.3: the rope band is
@@ -104,15 +110,20 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __r
 // head's columns into an fp32 accumulator with atomics; this kernel rounds the sums to bf16.
 __global__ void __launch_bounds__(256)
 bwd_dkpe_convert_kernel(const float* __restrict__ dkpe_acc, int S, __nv_bfloat16* __restrict__ dk_pe) {
+    // Launched behind the dQ kernel, whose output it does not touch: what it reads is complete once the dQ
+    // kernel's CTAs have passed THEIR dependency wait (they signal their dependents only after it), so it starts
+    // beside them and, like the delta kernel, waits at its end.  The sums were written by another grid's atomics:
+    // they are read past L1.
     grid_launch_dependents();
-    grid_dependency_wait();
     const size_t idx = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
-    if (idx >= static_cast<size_t>(S) * 64) return;
-    const float4 v = *reinterpret_cast<const float4*>(dkpe_acc + idx);
-    uint2 o;
-    o.x = pack_bf16x2(v.x, v.y);
-    o.y = pack_bf16x2(v.z, v.w);
-    *reinterpret_cast<uint2*>(dk_pe + idx) = o;
+    if (idx < static_cast<size_t>(S) * 64) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(dkpe_acc + idx));
+        uint2 o;
+        o.x = pack_bf16x2(v.x, v.y);
+        o.y = pack_bf16x2(v.z, v.w);
+        *reinterpret_cast<uint2*>(dk_pe + idx) = o;
+    }
+    grid_dependency_wait();
 }
 
 // Deterministic alternative to the atomics: sum the per-head buffers in head order.
@@ -596,8 +607,9 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    grid_launch_dependents();
     grid_dependency_wait();          // set-up above overlaps the previous kernel's tail; global memory from here on
+    grid_launch_dependents();        // after the wait: the kernel launched behind this one starts beside it and relies on
+                                     // everything before this kernel being complete (bwd_dkpe_convert_kernel)
     if (threadIdx.x == 0 && abort_flag->value != 0u) atomicCAS(args.status, kStatusOk, kStatusCheck | 0xD1u);   // set-up found the shared memory misaligned
     clock_probe_begin(args.clock_probe);
     const uint32_t tmem_base = *tmem_slot;
