@@ -587,6 +587,24 @@ def run_cuda(args):
     kv_saved_ms = max_over_ranks(s0.elapsed_time(s1), world) / K
     laga.check_status(ws_b, where="kv-saved step")
 
+    # ---- variant: LAGA_FLAG_FUSED_KV_REBUILD, step 4 rebuilt inside the dK/dV kernel (reported, not the headline) ----
+    def step_kv_rebuild():
+        laga.fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_f)
+        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw_kv_b=dw, workspace=ws_b,
+                 flags=laga.FLAG_FUSED_KV_REBUILD)
+
+    for _ in range(2):
+        step_kv_rebuild()
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    r0.record()
+    for _ in range(K):
+        step_kv_rebuild()
+    r1.record()
+    barrier(world)
+    kv_rebuild_ms = max_over_ranks(r0.elapsed_time(r1), world) / K
+    laga.check_status(ws_b, where="kv-rebuild step")
+
     # ---- variant: LAGA_FLAG_FUSED_BWD, the one-pass CTA-pair backward (reported, not the headline) ---------
     one_pass_ms = None
     try:
@@ -780,6 +798,10 @@ def run_cuda(args):
                      "kv_saved": {"ms_per_step": kv_saved_ms, "value": world * total_flops / (kv_saved_ms * 1e-3) / 1e12,
                                   "note": "LAGA_FLAG_KV_SAVED: the backward reads the forward's K_nope/V from a shared "
                                           "workspace instead of recomputing step 4 (one launch less); not the headline"},
+                     "kv_rebuild": {"ms_per_step": kv_rebuild_ms, "value": world * total_flops / (kv_rebuild_ms * 1e-3) / 1e12,
+                                    "note": "LAGA_FLAG_FUSED_KV_REBUILD: the recomputation of step 4 fused into the dK/dV kernel's item "
+                                            "prologue (one launch less, K/V tiles built once per item); compare with no_kernel_events; "
+                                            "not the headline"},
                      "one_pass_bwd": {"ms_per_step": one_pass_ms,
                                       "note": "LAGA_FLAG_FUSED_BWD: backward attention that computes every score tile once on CTA "
                                               "pairs (1664 instead of 2304 executed FLOP per pair) with dQ summed by fp32 atomics; "

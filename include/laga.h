@@ -58,6 +58,7 @@ extern "C" {
 #define LAGA_FLAG_DETERMINISTIC 2u        /* laga_bwd: bitwise-repeatable dk_pe and dw_kv_b (see there) */
 #define LAGA_FLAG_KV_SAVED 4u             /* laga_bwd: the workspace still holds laga_fwd's K_nope/V (see there) */
 #define LAGA_FLAG_FUSED_BWD 8u            /* laga_bwd: one-pass backward attention on CTA pairs (see there)       */
+#define LAGA_FLAG_FUSED_KV_REBUILD 16u    /* laga_bwd: step 4 rebuilt inside the dK/dV kernel (see there)         */
 
 /* Library version (major*10000 + minor*100 + patch). */
 int laga_version(void);
@@ -113,6 +114,14 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
  * laga_bwd_workspace_bytes), so dq is then not repeatable bit for bit.  It executes 5 instead of 7 tile
  * products but is the SLOWER path on B200 as measured (its exponentials sit on one of the two SMs); it is
  * not the default and cannot be combined with LAGA_FLAG_DETERMINISTIC (LAGA_ERR_INVALID_ARG).
+ * LAGA_FLAG_FUSED_KV_REBUILD fuses the recomputation of step 4 into the dK/dV kernel (the open direction the
+ * paper names in Section 4.7: a fused up-projection -> attention kernel): every (key tile, head) item builds its
+ * own K_nope / V tile from c_kv and the head's block of w_kv_b with tensor-core MMAs in its prologue and stores
+ * it to the workspace for the dQ kernel; the separate up-projection launch is dropped.  Same results up to the
+ * summation order of the tensor cores; same workspace; one launch less.  Not combinable with LAGA_FLAG_KV_SAVED
+ * or LAGA_FLAG_FUSED_BWD (LAGA_ERR_INVALID_ARG).  Measured on B200: faster at S = 512, even at S = 4096 and at
+ * S = 16384, 4-14 % slower in between (the prologue is serial work per item: the accumulators it builds the tile in
+ * are free only between the previous item's drain and this item's first product); opt-in.
  */
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
              const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,

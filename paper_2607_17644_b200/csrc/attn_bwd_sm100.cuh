@@ -181,10 +181,22 @@ static_assert(AttnBwdDkvSmem::kTotalBytes <= 232448, "dkv kernel exceeds the 227
 // S^T(j) is issued as soon as the consumers have read dP^T(j-1) out of X, so the exponentials of tile j
 // run under dK(j-1) and dP^T(j); dS^T(j-1) is computed under dV(j-1) and S^T(j).  The two consumer
 // warpgroups split each tile's query columns (64 each).
-template <bool kCausal>
+//
+// kRebuild (LAGA_FLAG_FUSED_KV_REBUILD): the up-projection of Algorithm 1 step 4 is fused into this kernel's item
+// prologue instead of being recomputed by a GEMM launch of its own.  The item's K_nope / V tile
+// [128 keys x 256] = c_kv[128 keys x 512] . W_kv_b[512 x 256 of the head] is built by 32 MMAs (N = 256) into the
+// accumulator columns that dK / dV will occupy (they are free between items), from eight 64-deep chunks that the
+// producer streams through the Q stages (one chunk = one c_kv slab + a 64 x 256 block of W = exactly one stage;
+// eight chunks are four turns of the two-stage ring, so the Q tiles' stage and phase numbering is unchanged).  The
+// consumers round the tile to bf16 and write it into the K and V operand slabs in the swizzled layout a TMA load
+// would have produced; one of them also stores the four slabs to the K/V workspace, which the dQ kernel reads
+// afterwards.  Only the shared rope band still comes from memory.  The key-stationary loop is the one place where
+// this fusion costs no extra arithmetic (each K/V tile is built once).
+template <bool kCausal, bool kRebuild = false>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_do,
                           const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
+                          const __grid_constant__ CUtensorMap tmap_ckv, const __grid_constant__ CUtensorMap tmap_w,
                           const AttnBwdDkvArgs args) {
     using L = AttnBwdDkvSmem;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -207,13 +219,17 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     uint64_t* acc_empty = bars + 17;  // both groups have drained them
     ItemRing ring{bars + 18, bars + 20, reinterpret_cast<volatile int*>(bars + 22)};
     uint64_t* quiesce_bar = bars + 23;   // abort path only: the MMA lane's last commit
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
+    uint64_t* rb_full = bars + 24;       // kRebuild: the item's K_nope / V tile is in TMEM (fp32)
+    uint64_t* kv_built = bars + 25;      // kRebuild: both groups have written it to the operand slabs
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
     AbortFlag* abort_flag = reinterpret_cast<AbortFlag*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1); mbar_init(kv_empty, 1);
+        mbar_init(rb_full, 1); mbar_init(kv_built, 256);
+        if (kRebuild) { tma_prefetch_desc(&tmap_ckv); tma_prefetch_desc(&tmap_w); }
         for (int s = 0; s < L::kQStages; ++s) { mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); }
         mbar_init(do_full, 1); mbar_init(do_empty, 1);
         mbar_init(st_full, 1); mbar_init(st_read, 256); mbar_init(dp_full, 1); mbar_init(dp_read, 256);
@@ -269,13 +285,34 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 const int row_base = seq.seq_start;
                 ok = mbar_wait(kv_empty, (n & 1u) ^ 1u, abort_flag, args.status, 0x41);
                 if (!ok) break;
-                mbar_arrive_expect_tx(kv_full, 5 * L::kSlab);
-                armed.arm(kv_full, n & 1u);
-                tma_load_2d_chk(args.status, smem + L::kK, &tmap_kv, kv_full, head * 256, row_base + t0);
-                tma_load_2d_chk(args.status, smem + L::kK + L::kSlab, &tmap_kv, kv_full, head * 256 + 64, row_base + t0);
-                tma_load_2d_chk(args.status, smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, row_base + t0);
-                tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, row_base + t0);
-                tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, kv_full, head * 256 + 192, row_base + t0);
+                if (!kRebuild) {
+                    mbar_arrive_expect_tx(kv_full, 5 * L::kSlab);
+                    armed.arm(kv_full, n & 1u);
+                    tma_load_2d_chk(args.status, smem + L::kK, &tmap_kv, kv_full, head * 256, row_base + t0);
+                    tma_load_2d_chk(args.status, smem + L::kK + L::kSlab, &tmap_kv, kv_full, head * 256 + 64, row_base + t0);
+                    tma_load_2d_chk(args.status, smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, row_base + t0);
+                    tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, kv_full, head * 256 + 128, row_base + t0);
+                    tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, kv_full, head * 256 + 192, row_base + t0);
+                } else {
+                    // only the rope band is loaded; K_nope and V are built from eight chunks of the latent and the
+                    // head's weight block, streamed through the Q stages ahead of the item's Q tiles (chunk c takes
+                    // the ring position of tile T + c: eight positions are whole turns of the ring and of its phases)
+                    mbar_arrive_expect_tx(kv_full, L::kSlab);
+                    armed.arm(kv_full, n & 1u);
+                    tma_load_2d_chk(args.status, smem + L::kK + 2 * L::kSlab, &tmap_kpe, kv_full, 0, row_base + t0);
+                    for (uint32_t c = 0; c < 8u && ok; ++c) {
+                        const uint32_t Tc = T + c, sq = Tc % L::kQStages;
+                        ok = mbar_wait(&q_empty[sq], ((Tc / L::kQStages) & 1u) ^ 1u, abort_flag, args.status, 0x43);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&q_full[sq], 3 * L::kSlab);
+                        armed.arm(&q_full[sq], (Tc / L::kQStages) & 1u);
+                        uint8_t* dst = smem + L::kQ + sq * 3 * L::kSlab;
+                        tma_load_2d_chk(args.status, dst, &tmap_ckv, &q_full[sq], static_cast<int>(c) * 64, row_base + t0);
+                        for (int b = 0; b < 4; ++b)     // 64 latent rows x 64 columns each: 8 KB boxes
+                            tma_load_2d(dst + L::kSlab + b * 8192, &tmap_w, &q_full[sq], head * 256 + b * 64, static_cast<int>(c) * 64);
+                    }
+                    if (!ok) break;
+                }
                 for (int j = 0; j < n_iter; ++j, ++T) {
                     const uint32_t sq = T % L::kQStages;
                     const int q0 = (j_begin + j) * 128;
@@ -337,7 +374,26 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 int t0, head, j_begin, n_iter;
                 SeqTile seq;
                 item_geometry(item, t0, head, j_begin, n_iter, seq);
-                ok = mbar_wait(kv_full, n & 1u, abort_flag, args.status, 0x54);
+                if (kRebuild) {
+                    // the accumulator columns take the K/V tile first: the previous item's dK / dV must be drained
+                    if (n > 0) ok = mbar_wait(acc_empty, (n - 1) & 1u, abort_flag, args.status, 0x58);
+                    constexpr uint32_t idesc_rb = make_idesc_bf16(128, 256, 0, 1);   // A = c_kv K-major, B = W MN-major
+                    for (uint32_t c = 0; c < 8u && ok; ++c) {
+                        const uint32_t Tc = T0 + c, sq = Tc % L::kQStages;
+                        ok = mbar_wait(&q_full[sq], (Tc / L::kQStages) & 1u, abort_flag, args.status, 0x59);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t sa = smem_u32(smem + L::kQ + sq * 3 * L::kSlab), sb = sa + L::kSlab;
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_ss(tmem_dk, desc_k_major(sa + kk * 32), desc_mn_major(sb + kk * 2048, 8192), idesc_rb,
+                                   (c > 0u || kk > 0) ? 1u : 0u);
+                        mma_commit(&q_empty[sq]);
+                    }
+                    if (ok) mma_commit(rb_full);
+                    if (ok) ok = mbar_wait(kv_built, n & 1u, abort_flag, args.status, 0x5A);
+                }
+                if (ok) ok = mbar_wait(kv_full, n & 1u, abort_flag, args.status, 0x54);
                 if (ok) ok = issue_st(T0, T0 == 0);
                 if (ok) ok = issue_dp(T0);
                 if (ok && n_iter == 1) mma_commit(kv_empty);
@@ -395,6 +451,50 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             item_geometry(item, t0, head, j_begin, n_iter, seq);
             const int t_idx = t0 + row;                       // key index within the sequence
             const int t_row = seq.seq_start + t_idx;          // its row in the packed tensors
+            if (kRebuild) {
+                // The item's K_nope / V tile is in the accumulator columns as fp32.  Group 0 rounds K_nope (columns
+                // 0..127) into the two K slabs, group 1 V (128..255) into the two V slabs: row r of a slab at r * 128
+                // bytes, its 16-byte chunks XORed with r & 7 -- what a 128-byte-swizzled TMA load writes.
+                ok = mbar_wait_warp(rb_full, n & 1u, abort_flag, args.status, 0x66);
+                if (!ok) break;
+                tc_fence_after_sync();
+                uint8_t* dst_row = smem + (g == 0 ? L::kK : L::kV) + row * 128;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    __syncwarp();
+                    tmem_ld_x32(tmem_dk + lane_addr + g * 128 + c * 32, r);
+                    tmem_ld_wait();
+                    uint8_t* slab = dst_row + (c >> 1) * L::kSlab;
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const int chunk = (c & 1) * 4 + v;
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(r[8 * v]), __uint_as_float(r[8 * v + 1]));
+                        w.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+                        w.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+                        w.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+                        *reinterpret_cast<uint4*>(slab + ((chunk ^ (row & 7)) << 4)) = w;
+                    }
+                }
+                fence_async_shared();      // the MMAs and the TMA store below read the slabs through the async proxy
+                tc_fence_before_sync();
+                mbar_arrive(kv_built);
+                if (warp == 2) {           // one lane stores the tile to the K/V workspace for the dQ kernel
+                    ok = mbar_wait_warp(kv_built, n & 1u, abort_flag, args.status, 0x67);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        const int y = seq.seq_start + t0;
+                        tma_store_2d(&tmap_kv, smem + L::kK, head * 256, y);
+                        tma_store_2d(&tmap_kv, smem + L::kK + L::kSlab, head * 256 + 64, y);
+                        tma_store_2d(&tmap_kv, smem + L::kV, head * 256 + 128, y);
+                        tma_store_2d(&tmap_kv, smem + L::kV + L::kSlab, head * 256 + 192, y);
+                        tma_store_commit();
+                        tma_store_wait_read<0>();      // the slabs are rewritten by the next item's tile
+                    }
+                    __syncwarp();
+                }
+            }
             for (int j = 0; j < n_iter; ++j) {
                 const uint32_t T = T0 + j;
                 const uint32_t ph = T & 1u;
@@ -519,6 +619,7 @@ attn_bwd_dkv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             tc_fence_before_sync();
             mbar_arrive(acc_empty);
         }
+        if (kRebuild && warp == 2 && lane == 0) tma_store_wait_all();    // the K/V tiles this lane stored are in memory
     }
     tc_fence_before_sync();
     __syncthreads();

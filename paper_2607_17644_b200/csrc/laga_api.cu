@@ -120,6 +120,8 @@ void init_device(DeviceInfo* info, int dev) {
               allow_smem(attn_fwd_sm100_kernel<false>, AttnFwdSmem::kTotalBytes) &&
               allow_smem(attn_bwd_dkv_sm100_kernel<true>, AttnBwdDkvSmem::kTotalBytes) &&
               allow_smem(attn_bwd_dkv_sm100_kernel<false>, AttnBwdDkvSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_dkv_sm100_kernel<true, true>, AttnBwdDkvSmem::kTotalBytes) &&
+              allow_smem(attn_bwd_dkv_sm100_kernel<false, true>, AttnBwdDkvSmem::kTotalBytes) &&
               allow_smem(attn_bwd_dq_sm100_kernel<true>, AttnBwdDqSmem::kTotalBytes) &&
               allow_smem(attn_bwd_dq_sm100_kernel<false>, AttnBwdDqSmem::kTotalBytes) &&
               allow_smem(attn_bwd_fused_sm100_kernel<true>, AttnBwdFusedSmem::kTotalBytes) &&
@@ -529,7 +531,8 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
                     void* dk_pe, float* stat_l2, float* stat_delta, float* dkpe_acc, float* dk_rope_per_head, int S_pad,
                     float* dq_acc, int head_window, unsigned* status, cudaStream_t stream,
                     const int4* q_tiles = nullptr, const int4* k_tiles = nullptr, const int2* seqs = nullptr,
-                    int n_seqs = 0, int n_seq_tiles = 0, bool overlap = false) {
+                    int n_seqs = 0, int n_seq_tiles = 0, bool overlap = false,
+                    const void* rebuild_c_kv = nullptr, const void* rebuild_w = nullptr) {
     const int N = h * (kDn + kDv);
     const float scale_log2 = softmax_scale * 1.4426950408889634f;
     {   // delta and the transposed, padded softmax statistics; clears the rope-gradient accumulator on the way
@@ -584,8 +587,17 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
                         make_schedule(n_tiles, S, h, slot_counter(status, kSlotDq), q_tiles), slot_probe(status, kSlotDq)};
         {
             ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DKV, stream);
-            launch_kernel(causal ? attn_bwd_dkv_sm100_kernel<true> : attn_bwd_dkv_sm100_kernel<false>, grid, dim3(kBwdThreads),
-                          AttnBwdDkvSmem::kTotalBytes, stream, true, tq, tdo, tkv, tpe, a);
+            if (rebuild_c_kv != nullptr) {     // step 4 inside the kernel: boxes of the latent (64 x 128 rows) and of W (64 x 64 rows)
+                CUtensorMap tc, tw;
+                if (!cached_tmap_bf16(&tc, rebuild_c_kv, kDc, S, kDc * 2, 128) ||
+                    !cached_tmap_bf16(&tw, rebuild_w, N, kDc, static_cast<uint64_t>(N) * 2, 64))
+                    return LAGA_ERR_CUDA;
+                launch_kernel(causal ? attn_bwd_dkv_sm100_kernel<true, true> : attn_bwd_dkv_sm100_kernel<false, true>, grid,
+                              dim3(kBwdThreads), AttnBwdDkvSmem::kTotalBytes, stream, true, tq, tdo, tkv, tpe, tc, tw, a);
+            } else {
+                launch_kernel(causal ? attn_bwd_dkv_sm100_kernel<true, false> : attn_bwd_dkv_sm100_kernel<false, false>, grid,
+                              dim3(kBwdThreads), AttnBwdDkvSmem::kTotalBytes, stream, true, tq, tdo, tkv, tpe, tkv, tkv, a);
+            }
         }
         if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
         {
@@ -693,7 +705,7 @@ int zero_status_word(void* status_word, cudaStream_t stream) {
 
 extern "C" {
 
-int laga_version(void) { return 210; }
+int laga_version(void) { return 211; }
 
 const char* laga_status_string(int status) {
     switch (status) {
@@ -906,9 +918,12 @@ static int bwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
         !aligned16(lse) || !aligned16(dout) || !aligned16(dq) || !aligned16(dc_kv) || !aligned16(dk_pe) ||
         !aligned16(dw_kv_b) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return LAGA_ERR_INVALID_ARG;
-    if ((flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC | LAGA_FLAG_KV_SAVED | LAGA_FLAG_FUSED_BWD)) || !(softmax_scale > 0.f))
+    if ((flags & ~(LAGA_FLAG_ACCUM_DW | LAGA_FLAG_DETERMINISTIC | LAGA_FLAG_KV_SAVED | LAGA_FLAG_FUSED_BWD | LAGA_FLAG_FUSED_KV_REBUILD)) ||
+        !(softmax_scale > 0.f))
         return LAGA_ERR_INVALID_ARG;
     if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
+    const bool rebuild = (flags & LAGA_FLAG_FUSED_KV_REBUILD) != 0;
+    if (rebuild && (flags & (LAGA_FLAG_KV_SAVED | LAGA_FLAG_FUSED_BWD))) return LAGA_ERR_INVALID_ARG;
     const bool deterministic = (flags & LAGA_FLAG_DETERMINISTIC) != 0;
     const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
     const bool fused = (flags & LAGA_FLAG_FUSED_BWD) != 0;
@@ -940,13 +955,15 @@ static int bwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
     }
     // K_nope / V are recomputed from the latent (the forward keeps only out and lse) unless the caller
     // vouches that the forward's copy is still in this workspace: both layouts put it right after the status.
-    if (!(flags & LAGA_FLAG_KV_SAVED) && (rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
+    // (or the dK/dV kernel rebuilds them tile by tile: LAGA_FLAG_FUSED_KV_REBUILD)
+    const bool up_project = !(flags & LAGA_FLAG_KV_SAVED) && !rebuild;
+    if (up_project && (rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
     if ((rc = launch_attn_bwd(q, kv, k_pe, out, lse, dout, S, h, softmax_scale, causal, dq, dkv, dk_pe,
                               reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
                               reinterpret_cast<float*>(base + w.dkpe_acc),
                               deterministic ? reinterpret_cast<float*>(base + w.dk_rope_per_head) : nullptr, w.S_pad,
                               reinterpret_cast<float*>(base + w.dq_acc), w.head_window, status, st, q_tiles, k_tiles, seqs,
-                              plan.n_seqs, plan.n_tiles, /*overlap=*/!(flags & LAGA_FLAG_KV_SAVED))) != LAGA_OK)
+                              plan.n_seqs, plan.n_tiles, /*overlap=*/up_project, rebuild ? c_kv : nullptr, w_kv_b)) != LAGA_OK)
         return rc;
     // the two GEMMs of Section 5.2 are token-wise: one launch each over all the packed tokens
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,

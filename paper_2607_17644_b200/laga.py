@@ -22,6 +22,7 @@ FLAG_ACCUM_DW = 1
 FLAG_DETERMINISTIC = 2
 FLAG_KV_SAVED = 4
 FLAG_FUSED_BWD = 8
+FLAG_FUSED_KV_REBUILD = 16
 
 # LAGA_DEBUG=1 selects the checked build of the same kernels (liblaga_debug.so): every TMA issue and global
 # store verifies its index arithmetic first and reports LAGA_ERR_DEVICE_CHECK instead of a bad access.

@@ -89,6 +89,17 @@ def run_case(S, h, causal):
         assert err <= 5e-3, (name, err)
     assert float((lse.double().cpu() - ref["lse"]).abs().max()) <= 1e-3
     assert float((lse_a.double().cpu() - ref["lse"]).abs().max()) <= 5e-3
+    # step 4 rebuilt inside the dK/dV kernel (its TMA stores of the K/V tiles end at the last row): same buffers again
+    for t in (dq_1, dc_kv_1, dk_pe_1, dw_1):
+        t.fill_(float("nan"))
+    laga.bwd(q, c_kv, k_pe, w, out, lse, dout, causal=causal, dq=dq_1, dc_kv=dc_kv_1, dk_pe=dk_pe_1, dw_kv_b=dw_1,
+             workspace=ws_b, flags=laga.FLAG_FUSED_KV_REBUILD)
+    laga.check_status(ws_b, where="laga_bwd (K/V rebuilt in the dK/dV kernel)")
+    torch.cuda.synchronize()
+    assert arena.guards_intact(), f"a guard band was overwritten by the rebuild path (S={S}, h={h})"
+    for name, got in (("dq", dq_1), ("dc_kv", dc_kv_1), ("dk_pe", dk_pe_1), ("dw", dw_1)):
+        err = rel_l2(got, ref[name])
+        assert err <= 5e-3, ("rebuild", name, err)
 
 
 def run_packed_case(lengths, h, causal):

@@ -107,7 +107,9 @@ def test_argument_validation_happens_before_any_device_work(laga):
                             a["d_rope"], a["d_v"], 0.07, 1, dq, good, good, good, good, ws_bytes, flags, None)
 
     assert bwd(dq=None) == laga.ERR_INVALID_ARG
-    assert bwd(flags=16) == laga.ERR_INVALID_ARG    # 1, 2, 4 and 8 are defined
+    assert bwd(flags=32) == laga.ERR_INVALID_ARG    # 1, 2, 4, 8 and 16 are defined
+    assert bwd(flags=laga.FLAG_FUSED_KV_REBUILD | laga.FLAG_KV_SAVED) == laga.ERR_INVALID_ARG
+    assert bwd(flags=laga.FLAG_FUSED_KV_REBUILD | laga.FLAG_FUSED_BWD) == laga.ERR_INVALID_ARG
     assert bwd(flags=laga.FLAG_FUSED_BWD | laga.FLAG_DETERMINISTIC) == laga.ERR_INVALID_ARG
     assert bwd(d_v=64) == laga.ERR_UNSUPPORTED
     assert bwd(ws_bytes=4096) == laga.ERR_WORKSPACE_TOO_SMALL

@@ -142,6 +142,65 @@ def test_one_pass_backward_at_the_headline_size_agrees_with_the_default_path(lag
     assert float((a[3] - b[3]).norm() / b[3].norm()) < 1e-5                                   # dw (atomics)
 
 
+REBUILD_CASES = [(512, 2, True), (300, 3, True), (300, 3, False), (1, 1, True), (129, 2, True), (1024, 4, True),
+                 (700, 1, False), (2048, 5, True), (4096, 16, True)]
+
+
+@pytest.mark.parametrize("S,h,causal", REBUILD_CASES)
+def test_kv_rebuild_in_the_dkv_kernel_elementwise(laga, oracle, S, h, causal):
+    """LAGA_FLAG_FUSED_KV_REBUILD: step 4 is rebuilt tile by tile in the dK/dV kernel's prologue (and stored for
+    the dQ kernel) instead of by a GEMM launch.  Every gradient against the oracle with the default path's
+    tolerances, outputs prefilled with NaN."""
+    sh = LagaShape(S=S, h=h)
+    tensors = make_inputs(sh, 9000 + S + h)
+    g = run_gpu(laga, tensors, causal, bwd_flags=laga.FLAG_FUSED_KV_REBUILD)
+    q, c_kv, k_pe, w, dout = tensors
+    if S <= 2048:
+        r = oracle.bwd(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, causal=causal, kv_round_bf16=True, return_fwd=True)
+        if S > 1:
+            check_tensor("dq", g["dq"], r["dq"])
+            check_tensor("dk_pe", g["dk_pe"], r["dk_pe"])
+        else:
+            assert max_abs(g["dq"], r["dq"]) <= 1e-5 and max_abs(g["dk_pe"], r["dk_pe"]) <= 1e-5
+        check_tensor("dc_kv", g["dc_kv"], r["dc_kv"])
+        check_dw(g["dw"], r["dw"])
+        if S >= 64:
+            check_row_bands("dq", g["dq"], r["dq"])
+    # and against the default path: the K/V tiles come from the same products (tensor-core summation order aside)
+    d = run_gpu(laga, tensors, causal)
+    for name in ("dq", "dc_kv", "dk_pe"):
+        a, b = g[name].double(), d[name].double()
+        assert not torch.isnan(a).any(), name
+        assert float((a - b).norm() / b.norm().clamp_min(1e-30)) < 2e-3, name
+    assert float((g["dw"].double() - d["dw"].double()).norm() / d["dw"].double().norm().clamp_min(1e-30)) < 2e-3
+
+
+def test_kv_rebuild_with_packed_sequences(laga, oracle):
+    """The same flag through laga_bwd_varlen: ragged sequences whose key tiles read (and store) rows of the next
+    sequence, against the oracle applied sequence by sequence."""
+    lens = [130, 5, 384, 77, 256]
+    cu = [0]
+    for n in lens:
+        cu.append(cu[-1] + n)
+    sh = LagaShape(S=cu[-1], h=3)
+    q, c_kv, k_pe, w, dout = make_inputs(sh, 9100)
+    dev = [t.cuda() for t in (q, c_kv, k_pe, w, dout)]
+    out, lse, ws = laga.fwd(*dev[:4], cu_seqlens=cu)
+    laga.check_status(ws)
+    dq, dc, dk, dw, ws2 = laga.bwd(*dev[:4], out, lse, dev[4], cu_seqlens=cu, dq=nan_like(tuple(q.shape), torch.bfloat16),
+                                   dc_kv=nan_like(tuple(c_kv.shape), torch.bfloat16), flags=laga.FLAG_FUSED_KV_REBUILD)
+    laga.check_status(ws2)
+    dw_ref = torch.zeros(w.shape, dtype=torch.float64)
+    for a, b in zip(cu[:-1], cu[1:]):
+        r = oracle.bwd(q[a:b], c_kv[a:b], k_pe[a:b], w, dout[a:b], sh.d_v, sh.softmax_scale, causal=True, kv_round_bf16=True)
+        if b - a > 1:
+            check_tensor("dq", dq[a:b].cpu(), r["dq"])
+        check_tensor("dc_kv", dc[a:b].cpu(), r["dc_kv"])
+        check_tensor("dk_pe", dk[a:b].cpu(), r["dk_pe"])
+        dw_ref += r["dw"]
+    check_dw(dw.cpu(), dw_ref)
+
+
 def test_row_zero_and_head_shard_invariance(laga):
     """Properties that need no oracle: causal row 0 of O is V[0] (here: the bf16 up-projection row the
     library itself materialises), and a head shard's outputs do not depend on which other heads run
@@ -408,7 +467,7 @@ def test_kv_saved_flag_reuses_the_forwards_up_projection(laga):
     for a, b in zip(saved, recomputed):
         assert torch.equal(a, b)
     with pytest.raises(laga.LagaError):
-        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, flags=16)              # unknown flag bit
+        laga.bwd(q, c_kv, k_pe, w, out, lse, dout, flags=32)              # unknown flag bit
 
 
 def test_long_ragged_sequence_sampled(laga, oracle):
