@@ -119,9 +119,9 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
  * own K_nope / V tile from c_kv and the head's block of w_kv_b with tensor-core MMAs in its prologue and stores
  * it to the workspace for the dQ kernel; the separate up-projection launch is dropped.  Same results up to the
  * summation order of the tensor cores; same workspace; one launch less.  Not combinable with LAGA_FLAG_KV_SAVED
- * or LAGA_FLAG_FUSED_BWD (LAGA_ERR_INVALID_ARG).  Measured on B200: faster at S = 512, even at S = 4096 and at
- * S = 16384, 4-14 % slower in between (the prologue is serial work per item: the accumulators it builds the tile in
- * are free only between the previous item's drain and this item's first product); opt-in.
+ * or LAGA_FLAG_FUSED_BWD (LAGA_ERR_INVALID_ARG).  Measured on B200: within 3 % of the default path from S = 512 to
+ * S = 16384 (what the saved launch gains, the prologue -- serial work per item: the accumulators it builds the
+ * tile in are free only between the previous item's drain and this item's first product -- gives back); opt-in.
  */
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
              const float* lse, const void* dout, int S, int h, int d_c, int d_nope, int d_rope, int d_v,
