@@ -294,6 +294,71 @@ PACKED_MIXES = {
 }
 
 
+SWEEP_LENGTHS = (1024, 2048, 4096, 8192, 16384, 32768, 65536)
+
+
+def run_sweep(args):
+    """Sequence-length sweep at the headline head count (h_local = 16): forward and forward+backward of one
+    rank's shard from 1 K to 64 K tokens (the paper evaluates 4 K, 8 K and 16 K; the longer ones show where the
+    path settles once per-item and per-launch costs are amortised).  Device-timed, no per-kernel events."""
+    from paper_2607_17644_b200 import laga
+    laga.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    K, W = args.steps, max(args.warmup, 3)
+    rows = {}
+    for S in SWEEP_LENGTHS:
+        sh = LagaShape(S=S, h=16)
+        q, c_kv, k_pe, w, dout = (t.to(dev) for t in make_inputs(sh, 5000 + S))
+        out = torch.empty(sh.S, sh.h, sh.d_v, dtype=torch.bfloat16, device=dev)
+        lse = torch.empty(sh.S, sh.h, dtype=torch.float32, device=dev)
+        dq, dc_kv, dk_pe = torch.empty_like(q), torch.empty_like(c_kv), torch.empty_like(k_pe)
+        dw = torch.empty(sh.d_c, sh.n_cols, dtype=torch.float32, device=dev)
+        ws_f = laga.alloc_workspace(laga.fwd_workspace_bytes(sh.S, sh.h), dev)
+        ws_b = laga.alloc_workspace(laga.bwd_workspace_bytes(sh.S, sh.h), dev)
+
+        def fwd_only():
+            laga.fwd(q, c_kv, k_pe, w, out=out, lse=lse, workspace=ws_f)
+
+        def step():
+            fwd_only()
+            laga.bwd(q, c_kv, k_pe, w, out, lse, dout, dq=dq, dc_kv=dc_kv, dk_pe=dk_pe, dw_kv_b=dw, workspace=ws_b)
+
+        def timed(fn):
+            for _ in range(W):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(K):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / K
+
+        step_ms, fwd_ms = timed(step), timed(fwd_only)
+        laga.check_status(ws_f, where=f"sweep S={S} laga_fwd")
+        laga.check_status(ws_b, where=f"sweep S={S} laga_bwd")
+        fl = flops(sh)
+        total = fl["fwd"] + fl["bwd"]
+        rows[str(S)] = {"S": S, "h_local": 16, "ms_per_step": step_ms, "tflops": total / (step_ms * 1e-3) / 1e12,
+                        "frac_of_bf16_peak": total / (step_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                        "fwd_ms": fwd_ms, "fwd_tflops": fl["fwd"] / (fwd_ms * 1e-3) / 1e12, "flops_per_step": total}
+        del q, c_kv, k_pe, w, dout, out, lse, dq, dc_kv, dk_pe, dw, ws_f, ws_b
+        torch.cuda.empty_cache()
+    head = rows["16384"]
+    line = {"metric": METRIC, "value": head["tflops"], "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
+            "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "sweep: one rank's DeepSeek-V3 shard, h_local=16, causal, forward+backward, S from 1024 to 65536 "
+                                   "(the line's value is the S=16384 row)",
+                       "l2_policy": "inputs and workspaces larger than L2 from S=8192 on; the shorter rows fit in L2 (as they would "
+                                    "between the layers of a model this small)"},
+            "peak_source": peaks["source"] + " cuBLAS bf16, burst", "sweep": rows, "gpu_launches": 9 * K}
+    print(json.dumps(line), flush=True)
+
+
 def run_packed(args):
     """Batches and variable-length sequences (laga_fwd_varlen / laga_bwd_varlen): the same 16384 tokens of a
     16-head shard packed as one sequence, as a batch of four, as a ragged mix and as 64 short sequences.  Each
@@ -466,6 +531,8 @@ def run_cuda(args):
         return run_linear(args)
     if args.workload == "packed":
         return run_packed(args)
+    if args.workload == "sweep":
+        return run_sweep(args)
     world, rank, local_rank = dist_setup(args.gpus)
     dev = torch.device("cuda", torch.cuda.current_device())
     sh = CONFIGS[args.workload]
@@ -949,7 +1016,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing and parity leg")
-    ap.add_argument("--workload", choices=sorted(CONFIGS) + ["packed", "linear"], default=WORKLOAD,
+    ap.add_argument("--workload", choices=sorted(CONFIGS) + ["packed", "linear", "sweep"], default=WORKLOAD,
                     help="benchmark configuration (default c2, the headline; c4 = the absorbed form beside the LAGA "
                          "forward on c2's inputs; packed = batches / variable-length sequences through the varlen "
                          "entry points; linear = the dense projections of steps 1, 4 and 7; others are for profiling)")
