@@ -580,3 +580,10 @@ def test_autograd_wrapper_gives_the_oracles_gradients(laga, oracle):
         (o.float() * dout.float()).sum().backward()
         assert fresh[3].grad is None
     check_dw(acc / 2, ref["dw"])
+    # laga_bwd flags pass through: step 4 rebuilt inside the dK/dV kernel gives the same gradients
+    again = [t.clone().requires_grad_(True) for t in (q, c_kv, k_pe, w)]
+    o = laga_attention(*again, bwd_flags=laga.FLAG_FUSED_KV_REBUILD)
+    (o.float() * dout.float()).sum().backward()
+    check_tensor("dq (rebuild)", again[0].grad, ref["dq"])
+    check_tensor("dc_kv (rebuild)", again[1].grad, ref["dc_kv"])
+    check_tensor("dk_pe (rebuild)", again[2].grad, ref["dk_pe"])
