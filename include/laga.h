@@ -117,8 +117,8 @@ int laga_fwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv
  * LAGA_FLAG_FUSED_KV_REBUILD fuses the recomputation of step 4 into the dK/dV kernel (the open direction the
  * paper names in Section 4.7: a fused up-projection -> attention kernel): every (key tile, head) item builds its
  * own K_nope / V tile from c_kv and the head's block of w_kv_b with tensor-core MMAs in its prologue and stores
- * it to the workspace for the dQ kernel; the separate up-projection launch is dropped.  Same results up to the
- * summation order of the tensor cores; same workspace; one launch less.  Not combinable with LAGA_FLAG_KV_SAVED
+ * it to the workspace for the dQ kernel; the separate up-projection launch is dropped.  Same results (bit for bit
+ * with LAGA_FLAG_DETERMINISTIC on both sides); same workspace; one launch less.  Not combinable with LAGA_FLAG_KV_SAVED
  * or LAGA_FLAG_FUSED_BWD (LAGA_ERR_INVALID_ARG).  Measured on B200: within 3 % of the default path from S = 512 to
  * S = 16384 (what the saved launch gains, the prologue -- serial work per item: the accumulators it builds the
  * tile in are free only between the previous item's drain and this item's first product -- gives back); opt-in.

@@ -166,13 +166,13 @@ def test_kv_rebuild_in_the_dkv_kernel_elementwise(laga, oracle, S, h, causal):
         check_dw(g["dw"], r["dw"])
         if S >= 64:
             check_row_bands("dq", g["dq"], r["dq"])
-    # and against the default path: the K/V tiles come from the same products (tensor-core summation order aside)
-    d = run_gpu(laga, tensors, causal)
-    for name in ("dq", "dc_kv", "dk_pe"):
-        a, b = g[name].double(), d[name].double()
-        assert not torch.isnan(a).any(), name
-        assert float((a - b).norm() / b.norm().clamp_min(1e-30)) < 2e-3, name
-    assert float((g["dw"].double() - d["dw"].double()).norm() / d["dw"].double().norm().clamp_min(1e-30)) < 2e-3
+    # and against the default path: the K/V tiles are the same products accumulated in the same order, so with the
+    # ordered reductions on both sides every gradient is the same bit for bit
+    det = laga.FLAG_DETERMINISTIC
+    a = run_gpu(laga, tensors, causal, bwd_flags=det | laga.FLAG_FUSED_KV_REBUILD)
+    b = run_gpu(laga, tensors, causal, bwd_flags=det)
+    for name in ("dq", "dc_kv", "dk_pe", "dw"):
+        assert torch.equal(a[name], b[name]), name
 
 
 def test_kv_rebuild_with_packed_sequences(laga, oracle):
