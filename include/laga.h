@@ -29,9 +29,12 @@
  *   - The entry points may be called from several host threads at once (the library's per-device and
  *     tensor-map caches are locked); what the callers must keep apart is the memory: two calls that may
  *     overlap on the GPU must not share a workspace or an output.
- *   - This build is tuned for the DeepSeek-V3 head geometry: d_c = 512, d_nope = 128, d_rope = 64,
- *     d_v = 128.  Other values return LAGA_ERR_UNSUPPORTED.  S >= 1 and h >= 1 are arbitrary (S need
- *     not be a multiple of any tile).  Batch is a caller loop.
+ *   - This build is written for the DeepSeek-V3 head geometry: d_nope = 128, d_rope = 64, d_v = 128 (the
+ *     attention kernels' tiles and TMEM maps); other head dimensions return LAGA_ERR_UNSUPPORTED.  The latent
+ *     width d_c is free: any multiple of 8 from 8 to 8192 (it only enters the three token-wise GEMMs); 512 is
+ *     the tuned and benchmarked value.  The absorbed comparison form and LAGA_FLAG_FUSED_KV_REBUILD need
+ *     d_c = 512.  S >= 1 and h >= 1 are arbitrary (S need not be a multiple of any tile).  Batches: the
+ *     _varlen entry points.
  *   - `workspace` is caller-provided scratch of at least laga_*_workspace_bytes(...) bytes, 1024-byte
  *     aligned.  Its first 1024 bytes are the launch status slot (the status word laga_query_status reads,
  *     the work counters of the persistent kernels, their clock probes); every call clears what it needs.
@@ -47,7 +50,7 @@ extern "C" {
 
 #define LAGA_OK 0
 #define LAGA_ERR_INVALID_ARG (-1)         /* NULL or misaligned pointer, S < 1, h < 1, bad flag     */
-#define LAGA_ERR_UNSUPPORTED (-2)         /* head geometry other than 512/128/64/128, or not sm_100 */
+#define LAGA_ERR_UNSUPPORTED (-2)         /* head geometry other than 128/64/128 (see above), or not sm_100 */
 #define LAGA_ERR_WORKSPACE_TOO_SMALL (-3)
 #define LAGA_ERR_CUDA (-4)                /* a CUDA runtime/driver call or a launch failed          */
 #define LAGA_ERR_DEVICE_TIMEOUT (-5)      /* only from laga_query_status: a bounded device wait ran out */

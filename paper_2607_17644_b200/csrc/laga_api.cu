@@ -29,7 +29,13 @@ constexpr size_t kStatusBytes = 1024;   // the status word's slot; keeps what fo
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The head geometry is fixed (the attention kernels' tiles and TMEM maps are built for it); the latent width
+// is not: it only enters the three token-wise GEMMs, which take any multiple of 8 (16-byte rows).  The absorbed
+// comparison form and the fused K/V rebuild are written for d_c = 512 (geometry_is_v3).
 bool geometry_supported(int d_c, int d_nope, int d_rope, int d_v) {
+    return d_c >= 8 && d_c <= 8192 && d_c % 8 == 0 && d_nope == kDn && d_rope == kDr && d_v == kDv;
+}
+bool geometry_is_v3(int d_c, int d_nope, int d_rope, int d_v) {
     return d_c == kDc && d_nope == kDn && d_rope == kDr && d_v == kDv;
 }
 
@@ -740,7 +746,7 @@ int laga_up_project(const void* c_kv, const void* w_kv_b, int S, int h, int d_c,
     if ((rc = check_pointers({c_kv, w_kv_b, kv, status_word})) != LAGA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((rc = zero_status_word(status_word, st)) != LAGA_OK) return rc;
-    return launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, static_cast<unsigned*>(status_word), st);
+    return launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, static_cast<unsigned*>(status_word), st, false, d_c);
 }
 
 int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int S, int h, int d_c, int d_nope,
@@ -760,9 +766,9 @@ int laga_kv_backward(const void* dkv, const void* c_kv, const void* w_kv_b, int 
     const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
     if ((rc = zero_status_word(status_word, st)) != LAGA_OK) return rc;
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,
-                          accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st)) != LAGA_OK)
+                          accumulate ? 0 : static_cast<size_t>(d_c) * N, status, st, false, d_c)) != LAGA_OK)
         return rc;
-    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st);
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, (flags & LAGA_FLAG_DETERMINISTIC) != 0, status, st, false, d_c);
 }
 
 // laga_fwd and laga_fwd_varlen: cu_seqlens == nullptr means one sequence of S tokens.
@@ -798,7 +804,7 @@ static int fwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
         q_tiles = reinterpret_cast<const int4*>(base + kv_end + plan.q_tiles_offset());
     }
     // step 4 is token-wise: one GEMM over all the packed tokens
-    if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
+    if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st, false, d_c)) != LAGA_OK) return rc;
     return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st, q_tiles, plan.n_tiles, true);
 }
 
@@ -924,6 +930,7 @@ static int bwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
     if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
     const bool rebuild = (flags & LAGA_FLAG_FUSED_KV_REBUILD) != 0;
     if (rebuild && (flags & (LAGA_FLAG_KV_SAVED | LAGA_FLAG_FUSED_BWD))) return LAGA_ERR_INVALID_ARG;
+    if (rebuild && !geometry_is_v3(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;   // eight 64-deep chunks
     const bool deterministic = (flags & LAGA_FLAG_DETERMINISTIC) != 0;
     const bool accumulate = (flags & LAGA_FLAG_ACCUM_DW) != 0;
     const bool fused = (flags & LAGA_FLAG_FUSED_BWD) != 0;
@@ -957,7 +964,7 @@ static int bwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
     // vouches that the forward's copy is still in this workspace: both layouts put it right after the status.
     // (or the dK/dV kernel rebuilds them tile by tile: LAGA_FLAG_FUSED_KV_REBUILD)
     const bool up_project = !(flags & LAGA_FLAG_KV_SAVED) && !rebuild;
-    if (up_project && (rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st)) != LAGA_OK) return rc;
+    if (up_project && (rc = launch_up_project(c_kv, w_kv_b, S, N, kv, status, st, false, d_c)) != LAGA_OK) return rc;
     if ((rc = launch_attn_bwd(q, kv, k_pe, out, lse, dout, S, h, softmax_scale, causal, dq, dkv, dk_pe,
                               reinterpret_cast<float*>(base + w.stat_l2), reinterpret_cast<float*>(base + w.stat_delta),
                               reinterpret_cast<float*>(base + w.dkpe_acc),
@@ -967,9 +974,9 @@ static int bwd_impl(const void* q, const void* c_kv, const void* k_pe, const voi
         return rc;
     // the two GEMMs of Section 5.2 are token-wise: one launch each over all the packed tokens
     if ((rc = launch_dckv(dkv, w_kv_b, S, N, dc_kv, accumulate ? nullptr : dw_kv_b,
-                          accumulate ? 0 : static_cast<size_t>(kDc) * N, status, st, true)) != LAGA_OK)
+                          accumulate ? 0 : static_cast<size_t>(d_c) * N, status, st, true, d_c)) != LAGA_OK)
         return rc;
-    return launch_dw(c_kv, dkv, S, N, dw_kv_b, deterministic, status, st, true);
+    return launch_dw(c_kv, dkv, S, N, dw_kv_b, deterministic, status, st, true, d_c);
 }
 
 int laga_bwd(const void* q, const void* c_kv, const void* k_pe, const void* w_kv_b, const void* out,
@@ -1041,12 +1048,12 @@ int laga_fwd_builtin_scratch(const void* q, const void* c_kv, const void* k_pe, 
     // start at zero; KV rows [0, S) are fully overwritten by the up-projection before the attention kernel
     // reads them.
     if ((rc = zero_status(status, st)) != LAGA_OK) return rc;
-    if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st)) != LAGA_OK) return rc;
+    if ((rc = launch_up_project(c_kv, w_kv_b, S, h * (kDn + kDv), kv, status, st, false, d_c)) != LAGA_OK) return rc;
     return launch_attn_fwd(q, kv, k_pe, S, h, softmax_scale, causal, out, lse, status, st, nullptr, 0, true);
 }
 
 size_t laga_absorbed_fwd_workspace_bytes(int S, int h, int d_c, int d_nope, int d_rope, int d_v) {
-    if (S < 1 || h < 1 || !geometry_supported(d_c, d_nope, d_rope, d_v)) return 0;
+    if (S < 1 || h < 1 || !geometry_is_v3(d_c, d_nope, d_rope, d_v)) return 0;
     return kStatusBytes + 2 * align_up(static_cast<size_t>(S) * h * d_c * 2, 1024);
 }
 
@@ -1059,7 +1066,7 @@ int laga_absorbed_fwd(const void* q, const void* c_kv, const void* k_pe, const v
         !aligned16(lse) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return LAGA_ERR_INVALID_ARG;
     if (flags != 0 || !(softmax_scale > 0.f)) return LAGA_ERR_INVALID_ARG;
-    if (!geometry_supported(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
+    if (!geometry_is_v3(d_c, d_nope, d_rope, d_v)) return LAGA_ERR_UNSUPPORTED;
     if (workspace_bytes < laga_absorbed_fwd_workspace_bytes(S, h, d_c, d_nope, d_rope, d_v))
         return LAGA_ERR_WORKSPACE_TOO_SMALL;
     int rc = check_device();

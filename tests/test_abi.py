@@ -72,7 +72,9 @@ def test_workspace_sizes(laga):
     assert laga.bwd_workspace_bytes(512, 2, flags=laga.FLAG_FUSED_BWD) == laga.bwd_workspace_bytes(512, 2) + 512 * 2 * 192 * 4
     assert laga.fwd_workspace_bytes(300, 3) % 1024 == 0 and laga.bwd_workspace_bytes(300, 3) % 1024 == 0
     # unsupported geometry or empty problem: 0
-    assert laga.fwd_workspace_bytes(128, 2, d_c=256) == 0
+    assert laga.fwd_workspace_bytes(128, 2, d_c=256) == laga.fwd_workspace_bytes(128, 2)      # the latent width is free
+    assert laga.fwd_workspace_bytes(128, 2, d_c=260) == 0                                   # ... in multiples of 8
+    assert laga.fwd_workspace_bytes(128, 2, d_nope=64) == 0
     assert laga.bwd_workspace_bytes(128, 2, d_rope=32) == 0
     assert laga.fwd_workspace_bytes(0, 2) == 0 and laga.fwd_workspace_bytes(128, 0) == 0
 
@@ -97,7 +99,8 @@ def test_argument_validation_happens_before_any_device_work(laga):
     assert fwd(ws=p(1040)) == laga.ERR_INVALID_ARG   # workspace not 1024-byte aligned
     assert fwd(flags=8) == laga.ERR_INVALID_ARG
     assert fwd(scale=0.0) == laga.ERR_INVALID_ARG
-    assert fwd(d_c=256) == laga.ERR_UNSUPPORTED
+    assert fwd(d_c=260) == laga.ERR_UNSUPPORTED
+    assert fwd(d_nope=64) == laga.ERR_UNSUPPORTED
     assert fwd(d_rope=32) == laga.ERR_UNSUPPORTED
     assert fwd(ws_bytes=1024) == laga.ERR_WORKSPACE_TOO_SMALL
 

@@ -201,6 +201,28 @@ def test_kv_rebuild_with_packed_sequences(laga, oracle):
     check_dw(dw.cpu(), dw_ref)
 
 
+@pytest.mark.parametrize("d_c,S,h", [(256, 700, 3), (1024, 300, 2), (64, 513, 2), (1536, 260, 1), (520, 384, 2)])
+def test_other_latent_widths_elementwise(laga, oracle, d_c, S, h):
+    """The latent width only enters the three token-wise GEMMs (step 4, dc_kv, dW): any multiple of 8 runs through
+    the same kernels.  Forward and every gradient against the oracle, outputs prefilled with NaN; the fused K/V
+    rebuild, which is written for d_c = 512, must refuse."""
+    sh = LagaShape(S=S, h=h, d_c=d_c)
+    tensors = make_inputs(sh, 9500 + d_c + S)
+    g = run_gpu(laga, tensors, True)
+    q, c_kv, k_pe, w, dout = tensors
+    r = oracle.bwd(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, causal=True, kv_round_bf16=True, return_fwd=True)
+    check_tensor("out", g["out"], r["out"])
+    assert max_abs(g["lse"], r["lse"]) <= TOL_LSE
+    check_tensor("dq", g["dq"], r["dq"])
+    check_tensor("dc_kv", g["dc_kv"], r["dc_kv"])
+    check_tensor("dk_pe", g["dk_pe"], r["dk_pe"])
+    check_dw(g["dw"], r["dw"])
+    dev = [t.cuda() for t in tensors]
+    out, lse, _ = laga.fwd(*dev[:4])
+    with pytest.raises(laga.LagaError):
+        laga.bwd(*dev[:4], out, lse, dev[4], flags=laga.FLAG_FUSED_KV_REBUILD)
+
+
 def test_row_zero_and_head_shard_invariance(laga):
     """Properties that need no oracle: causal row 0 of O is V[0] (here: the bf16 up-projection row the
     library itself materialises), and a head shard's outputs do not depend on which other heads run
