@@ -492,6 +492,25 @@ def test_kv_saved_flag_reuses_the_forwards_up_projection(laga):
         laga.bwd(q, c_kv, k_pe, w, out, lse, dout, flags=32)              # unknown flag bit
 
 
+def test_quarter_million_tokens_sampled(laga, oracle):
+    """S = 262181 (sixteen times the headline length, two heads): 32-bit row counts times wide rows, thousands of
+    work items per CTA, three-digit tile counts per item.  Sampled query rows and late keys against the oracle."""
+    sh = LagaShape(S=262144 + 37, h=2)
+    tensors = make_inputs(sh, 4242)
+    q, c_kv, k_pe, w, dout = tensors
+    g = run_gpu(laga, tensors, True)
+    rows = sorted({0, 127, 128, 100000, 200001, sh.S - 1, sh.S - 38})
+    r = oracle.bwd_rows(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, rows, kv_round_bf16=True)
+    check_tensor("out[rows]", g["out"][rows], r["out"])
+    assert max_abs(g["lse"][rows], r["lse"]) <= TOL_LSE
+    check_tensor("dq[rows]", g["dq"][rows], r["dq"])
+    keys = sorted({sh.S - 1, sh.S - 2, sh.S - 37, sh.S - 101, sh.S - 300})
+    k = oracle.bwd_keys(q, c_kv, k_pe, w, dout, sh.d_v, sh.softmax_scale, keys, kv_round_bf16=True)
+    check_tensor("dk_pe[keys]", g["dk_pe"][keys], k["dk_pe"])
+    check_tensor("dc_kv[keys]", g["dc_kv"][keys], k["dc_kv"])
+    assert not torch.isnan(g["dw"]).any() and not torch.isnan(g["dc_kv"].float()).any()
+
+
 def test_long_ragged_sequence_sampled(laga, oracle):
     """A sequence longer than any benchmark configuration and a multiple of no tile size (40037 tokens, two
     heads): index arithmetic far from the origin and ragged tails in every kernel, checked on sampled query
