@@ -12,7 +12,7 @@
 //                             O += P V (6 tcgen05.mma of N=128).  Both read their A operand (Q, P) from TMEM:
 //                             an MMA with both operands in shared memory is bound by shared-memory
 //                             bandwidth (128 B/clk).
-//   warp 10     TMA producer: V tiles, three stages
+//   warp 10     TMA producer: V tiles, three stages; ahead of each item's tiles the item's query tile as three ring entries
 // Why 96 keys: the Q tile (96 columns of packed bf16), the O accumulator (128) and THREE score tiles
 // (3 x 96) fill the 512 TMEM columns exactly.  With three score tiles the tensor pipe computes S_{j+3}
 // while the two groups work on tiles j+1 and j+2, so neither side waits for the other; with 128-key
@@ -74,13 +74,12 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 // drained, so the next item's first score MMAs run under the drain.
 template <bool kCausal>
 __global__ void __launch_bounds__(kFwdThreads, 1)
-attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
-                      const AttnFwdArgs args) {
+attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
+                      const __grid_constant__ CUtensorMap tmap_kpe, const AttnFwdArgs args) {
     using L = AttnFwdSmem;
     constexpr int BK = kFwdKeys;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
-    uint64_t* q_ready = bars + 0;    // both warpgroups have put their halves of the item's Q tile into TMEM
     uint64_t* k_full = bars + 1;     // [3]
     uint64_t* k_empty = bars + 4;    // [3]
     uint64_t* v_full = bars + 7;     // [3]
@@ -107,7 +106,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        mbar_init(q_ready, 256);
         for (int s = 0; s < 3; ++s) {
             mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); mbar_init(&s_full[s], 1);
             mbar_init(&p_full[s], 128);
@@ -122,7 +120,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
         mbar_init(quiesce_bar, 1);
         abort_flag->value = 0;
         mbar_fence_init();
-        tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
+        tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_kv); tma_prefetch_desc(&tmap_kpe);
         if ((smem_u32(smem) & 1023u) != 0u) {   // the swizzled operand slabs need a 1024-byte aligned base
             abort_flag->value = 1;
         }
@@ -189,13 +187,29 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 if (!ok || item < 0) break;
                 int q0, head, n_kv, row_base, S_seq;
                 item_geometry(item, q0, head, n_kv, row_base, S_seq);
+                // The item's query tile travels through the V ring ahead of the item's value tiles: three slabs of
+                // 128 rows x 64 elements, one ring entry each (a stage holds 24 KB, a slab is 16 KB).  Three entries
+                // are one turn of the ring, so the value tiles keep their stages; every item shifts the barriers'
+                // phases by one.  The MMA lane copies the slabs to TMEM (tcgen05.cp): no thread's load/store unit
+                // sees the tile -- a lane reading its own row touches 32 lines per instruction, and done that way
+                // the staging cost four to seven thousand clocks per item on the softmax warps.
+                for (uint32_t c = 0; c < 3u && ok; ++c) {
+                    const uint32_t Tc = T + c, s = Tc % kFwdStages, ph = ((Tc / kFwdStages) + n) & 1u;
+                    ok = mbar_wait(&v_empty[s], ph ^ 1u, abort_flag, args.status, 0x12);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&v_full[s], 128 * 128);
+                    armed.arm(&v_full[s], ph);
+                    tma_load_2d_chk(args.status, smem + L::kV + s * 2 * L::kSlab, &tmap_q, &v_full[s], head * 192 + static_cast<int>(c) * 64,
+                                    row_base + q0);      // rows past the tensor's end read as zero
+                }
+                if (!ok) break;
                 for (int j = 0; j < n_kv; ++j, ++T) {
-                    const uint32_t s = T % kFwdStages;
-                    ok = mbar_wait(&v_empty[s], ((T / kFwdStages) & 1u) ^ 1u, abort_flag, args.status, 0x11);
+                    const uint32_t s = T % kFwdStages, phv = ((T / kFwdStages) + n + 1u) & 1u;
+                    ok = mbar_wait(&v_empty[s], phv ^ 1u, abort_flag, args.status, 0x11);
                     if (!ok) break;
                     uint8_t* dv = smem + L::kV + s * 2 * L::kSlab;
                     mbar_arrive_expect_tx(&v_full[s], 2 * L::kSlab);
-                    armed.arm(&v_full[s], (T / kFwdStages) & 1u);
+                    armed.arm(&v_full[s], phv);
                     tma_load_2d_chk(args.status, dv, &tmap_kv, &v_full[s], head * 256 + 128, row_base + j * BK);
                     tma_load_2d_chk(args.status, dv + L::kSlab, &tmap_kv, &v_full[s], head * 256 + 192, row_base + j * BK);
                 }
@@ -229,7 +243,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                 if (!ok || item < 0) break;
                 int q0, head, n_kv, row_base, S_seq;
                 item_geometry(item, q0, head, n_kv, row_base, S_seq);
-                ok = mbar_wait(q_ready, n & 1u, abort_flag, args.status, 0x22);
+                // The item's query tile: three entries of the V ring, copied to TMEM as the A operand of S.  (Every
+                // MMA that read the previous tile has completed: the previous item's last P V was issued after the
+                // softmax of its last score tile.)
+                for (uint32_t c = 0; c < 3u && ok; ++c) {
+                    const uint32_t Tc = T0 + c, s = Tc % kFwdStages;
+                    ok = mbar_wait(&v_full[s], ((Tc / kFwdStages) + n) & 1u, abort_flag, args.status, 0x22);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t src = smem_u32(smem + L::kV + s * 2 * L::kSlab);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) tmem_cp_128x256b(tmem_q + c * 32 + kk * 8, desc_k_major(src + kk * 32));
+                    mma_commit(&v_empty[s]);
+                }
+                const uint32_t vflip = (n + 1u) & 1u;     // phase shift of the V ring's barriers for this item's tiles
                 for (int j = 0; j < 3 && j < n_kv && ok; ++j) {
                     const uint32_t T = T0 + j;
                     ok = mbar_wait(&k_full[T % kFwdStages], (T / kFwdStages) & 1u, abort_flag, args.status, 0x23);
@@ -243,7 +270,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                     const uint32_t T = T0 + j;
                     const uint32_t s = T % kFwdStages, g = T & 1u;
                     const uint32_t ph = (T / kFwdStages) & 1u;
-                    if (!v_ok) ok = mbar_wait(&v_full[s], ph, abort_flag, args.status, 0x20);
+                    if (!v_ok) ok = mbar_wait(&v_full[s], ph ^ vflip, abort_flag, args.status, 0x20);
                     if (ok && !p_ok) ok = mbar_wait(&p_full[s], ph, abort_flag, args.status, 0x21);
                     if (!ok) break;
                     tc_fence_after_sync();
@@ -256,7 +283,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
                         if (!k_ok) ok = mbar_wait(&k_full[s], ph ^ 1u, abort_flag, args.status, 0x23);
                         if (!ok) break;
                         tc_fence_after_sync();
-                        v_ok = mbar_try_wait(&v_full[(T + 1) % kFwdStages], ((T + 1) / kFwdStages) & 1u);
+                        v_ok = mbar_try_wait(&v_full[(T + 1) % kFwdStages], (((T + 1) / kFwdStages) & 1u) ^ vflip);
                         p_ok = mbar_try_wait(&p_full[(T + 1) % kFwdStages], ((T + 1) / kFwdStages) & 1u);
                         qk_mmas(T + 3);
                     }
@@ -322,35 +349,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_kv, const __grid_
             int q0, head, n_kv, row_base, S_seq;
             item_geometry(item, q0, head, n_kv, row_base, S_seq);
             const int sq_idx = q0 + row;              // query index within the sequence
-            {   // The item's query tile goes to TMEM once, as the A operand of S (the previous item's MMAs, which read
-                // the old tile, are known complete).  Both groups own every TMEM lane (warps w and w + 4 address the same
-                // 32 lanes), so each takes half of the row: group g the 48 packed words [48g, 48g + 48).  A lane reads
-                // its own row and rows are kilobytes apart, so every 16-byte load is a round trip to L2 or HBM that
-                // touches 32 different lines per instruction: all of a thread's loads are issued before the first is
-                // used (three dependent rounds of eight cost 7.5 K clocks per item, one round far less).
-                const bool q_valid = sq_idx < S_seq;
-                const uint4* src = reinterpret_cast<const uint4*>(args.q + (static_cast<size_t>(row_base + sq_idx) * args.h + head) * 192) + g * 12;
-                uint32_t w[48];
-                if (!q_valid) {
-#pragma unroll
-                    for (int v = 0; v < 48; ++v) w[v] = 0u;
-                } else if (aligned32_dev(args.q)) {      // six 32-byte loads (half a row is 192 bytes)
-#pragma unroll
-                    for (int v = 0; v < 6; ++v) ld_global_v8(src + 2 * v, w + 8 * v);
-                } else {
-                    uint4 x[12];
-#pragma unroll
-                    for (int v = 0; v < 12; ++v) x[v] = src[v];
-#pragma unroll
-                    for (int v = 0; v < 12; ++v) { w[v * 4] = x[v].x; w[v * 4 + 1] = x[v].y; w[v * 4 + 2] = x[v].z; w[v * 4 + 3] = x[v].w; }
-                }
-                __syncwarp();
-                tmem_st_x32(tmem_q + lane_addr + g * 48, w);
-                tmem_st_x16(tmem_q + lane_addr + g * 48 + 32, w + 32);
-                tmem_st_wait();
-                tc_fence_before_sync();
-                mbar_arrive(q_ready);
-            }
             if (n > 0) drain(prev_sq_idx, prev_valid, prev_head, prev_m_fin, prev_l_run);
             float m_mine = -INFINITY;                     // reference max (scaled, log2 domain) l_part refers to
             float l_part = 0.f;                           // this group's part of the row sum

@@ -475,7 +475,9 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
                     const int4* q_tiles = nullptr, int n_seq_tiles = 0, bool overlap = false) {
     using L = AttnFwdSmem;
     const int N = h * (kDn + kDv);
-    CUtensorMap tkv, tpe;   // boxes of 64 columns x one key tile of rows
+    CUtensorMap tq, tkv, tpe;   // boxes of 64 columns x one query tile / one key tile of rows
+    const uint64_t q_row = static_cast<uint64_t>(h) * (kDn + kDr);
+    if (!cached_tmap_bf16(&tq, q, q_row, S, q_row * 2, 128)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tkv, kv, N, S, static_cast<uint64_t>(N) * 2, kFwdKeys)) return LAGA_ERR_CUDA;
     if (!cached_tmap_bf16(&tpe, k_pe, kDr, S, kDr * 2, kFwdKeys)) return LAGA_ERR_CUDA;
     const int n_tiles = q_tiles ? n_seq_tiles : (S + 127) / 128;
@@ -485,7 +487,7 @@ int launch_attn_fwd(const void* q, const void* kv, const void* k_pe, int S, int 
     dim3 grid(persistent_grid(n_tiles * h), 1, 1);
     ScopedKernelEvents ev(LAGA_KERNEL_ATTN_FWD, stream);
     launch_kernel(causal ? attn_fwd_sm100_kernel<true> : attn_fwd_sm100_kernel<false>, grid, dim3(kFwdThreads), L::kTotalBytes,
-                  stream, overlap, tkv, tpe, a);
+                  stream, overlap, tq, tkv, tpe, a);
     return launch_status();
 }
 

@@ -439,6 +439,15 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
                  : "memory");
 }
 
+// Shared memory -> TMEM, issued by ONE thread like an MMA (and executed in order with that thread's MMAs): row r
+// of a 128-row K-major swizzled slab, bytes [0, 32) from the descriptor's start address, lands in TMEM lane r,
+// columns [col, col + 8) -- the layout in which an MMA reads sixteen bf16 of its A operand from TMEM.  Advance
+// the start address by 32 bytes per eight columns inside a slab, exactly as for an MMA's K steps.  Completion is
+// observed through mma_commit.
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t desc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+}
+
 // Warp-collective TMEM loads.  Lane l of warp w (w % 4 selects the 32-lane quarter) receives, from
 // TMEM lane 32*(w%4)+l, the 32-bit columns [col, col+N).  `taddr` = (lane << 16) | column.
 __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t* r) {
