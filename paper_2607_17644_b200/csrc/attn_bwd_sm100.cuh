@@ -663,8 +663,9 @@ struct AttnBwdDqSmem {
 // MMAs of the next item run under the drain; the K ring simply keeps going across items.
 template <bool kCausal>
 __global__ void __launch_bounds__(kBwdThreads, 1)
-attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
-                         const __grid_constant__ CUtensorMap tmap_kpe, const AttnBwdDqArgs args) {
+attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_do,
+                         const __grid_constant__ CUtensorMap tmap_kv, const __grid_constant__ CUtensorMap tmap_kpe,
+                         const AttnBwdDqArgs args) {
     using L = AttnBwdDqSmem;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBar);
@@ -674,7 +675,6 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
     uint64_t* k_empty = bars + 5;     // [3]
     uint64_t* v_full = bars + 8;
     uint64_t* v_empty = bars + 9;
-    uint64_t* do_ready = bars + 10;   // the item's dO is in TMEM
     uint64_t* s_full = bars + 11;     // S is in TMEM
     uint64_t* s_read = bars + 12;     // both groups have loaded it
     uint64_t* dp_full = bars + 13;    // dP is in TMEM
@@ -692,7 +692,6 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
         mbar_init(q_full, 1); mbar_init(q_empty, 1);
         for (int s = 0; s < kDqKStages; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); }
         mbar_init(v_full, 1); mbar_init(v_empty, 1);
-        mbar_init(do_ready, 256);
         mbar_init(s_full, 1); mbar_init(s_read, 256); mbar_init(dp_full, 1); mbar_init(ds_full, 256);
         mbar_init(acc_full, 1); mbar_init(acc_empty, 256);
         for (int s = 0; s < 2; ++s) { mbar_init(&ring.full[s], 1); mbar_init(&ring.empty[s], 9); }
@@ -761,14 +760,27 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 for (int c = 0; c < 3; ++c)
                     tma_load_2d_chk(args.status, smem + L::kQ + c * L::kSlab, &tmap_q, q_full, head * 192 + c * 64, row_base + q0);
                 ok = load_k(T0, row_base, head);
+                if (!ok) break;
+                {   // The item's dO tile (the A operand of dP, kept in TMEM) goes through the single V stage ahead of the
+                    // item's V tiles: 128 rows x 128 elements are exactly its two slabs.  The MMA lane copies it to TMEM
+                    // (tcgen05.cp).  One more entry per item: the stage's barriers are counted on T + n.
+                    const uint32_t ph = (T0 + n) & 1u;
+                    ok = mbar_wait(v_empty, ph ^ 1u, abort_flag, args.status, 0x73);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
+                    armed.arm(v_full, ph);
+                    tma_load_2d_chk(args.status, smem + L::kV, &tmap_do, v_full, head * 128, row_base + q0);
+                    tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_do, v_full, head * 128 + 64, row_base + q0);
+                }
                 for (int j = 0; j < n_iter && ok; ++j) {
                     const uint32_t T = T0 + j;
                     if (j + 1 < n_iter) ok = load_k(T + 1, row_base + (j + 1) * 128, head);
                     if (!ok) break;
-                    ok = mbar_wait(v_empty, (T & 1u) ^ 1u, abort_flag, args.status, 0x71);
+                    const uint32_t phv = (T + n + 1u) & 1u;
+                    ok = mbar_wait(v_empty, phv ^ 1u, abort_flag, args.status, 0x71);
                     if (!ok) break;
                     mbar_arrive_expect_tx(v_full, 2 * L::kSlab);
-                    armed.arm(v_full, T & 1u);
+                    armed.arm(v_full, phv);
                     tma_load_2d_chk(args.status, smem + L::kV, &tmap_kv, v_full, head * 256 + 128, row_base + j * 128);
                     tma_load_2d_chk(args.status, smem + L::kV + L::kSlab, &tmap_kv, v_full, head * 256 + 192, row_base + j * 128);
                 }
@@ -794,8 +806,8 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                                     idesc_s, bar_a(s_full));
                 return true;
             };
-            auto issue_dp = [&](uint32_t T) -> bool {     // dP(T) = dO V^T; overwrites dS(T-1), whose reader was issued earlier
-                if (!mbar_wait(v_full, T & 1u, abort_flag, args.status, 0x84)) return false;
+            auto issue_dp = [&](uint32_t T, uint32_t n) -> bool {     // dP(T) = dO V^T; overwrites dS(T-1), whose reader was issued earlier
+                if (!mbar_wait(v_full, (T + n + 1u) & 1u, abort_flag, args.status, 0x84)) return false;
                 tc_fence_after_sync();
                 mma_ts_chain8_k128(tmem_dp, tmem_do, desc_lo(dk_v), desc_hi(dk_v), idesc_s, bar_a(v_empty), bar_a(dp_full));
                 return true;
@@ -811,8 +823,19 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                 ok = mbar_wait(q_full, n & 1u, abort_flag, args.status, 0x81);
                 if (ok) ok = issue_s(T0);
                 if (ok && n_iter == 1) mma_commit(q_empty);
-                if (ok) ok = mbar_wait(do_ready, n & 1u, abort_flag, args.status, 0x85);
-                if (ok) ok = issue_dp(T0);
+                if (ok) {     // the item's dO tile: from the V stage to TMEM (every dP MMA of the previous item has completed:
+                              // its last dS, which this lane has consumed, was computed from the last of them)
+                    ok = mbar_wait(v_full, (T0 + n) & 1u, abort_flag, args.status, 0x85);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        const uint32_t sv = smem_u32(smem + L::kV);
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            tmem_cp_128x256b(tmem_do + kk * 8, desc_k_major(sv + (kk >> 2) * L::kSlab + (kk & 3) * 32));
+                        mma_commit(v_empty);
+                    }
+                }
+                if (ok) ok = issue_dp(T0, n);
                 for (int j = 0; j < n_iter && ok; ++j) {
                     const uint32_t T = T0 + j;
                     if (j + 1 < n_iter) {
@@ -827,7 +850,7 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
                     tc_fence_after_sync();
                     mma_ts_chain8_mn_split(tmem_dq, tmem_dp, desc_lo(dm_k0) + (T % kDqKStages) * kKStageLo, desc_hi(dm_k0), idesc_dq,
                                            static_cast<uint32_t>(j), bar_a(&k_empty[T % kDqKStages]));
-                    if (j + 1 < n_iter) ok = issue_dp(T + 1);
+                    if (j + 1 < n_iter) ok = issue_dp(T + 1, n);
                 }
                 if (ok) mma_commit(acc_full);
                 T0 += static_cast<uint32_t>(n_iter);
@@ -892,32 +915,6 @@ attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gri
             const int s_idx = q0 + row;                       // query index within the sequence
             const int s_row = seq.seq_start + s_idx;          // its row in the packed tensors
             const bool valid = s_idx < S_seq;
-            {   // this thread's dO row, channels [64g, 64g+64), as 32 packed words into TMEM (the previous item's
-                // last dP MMA has completed: this group waited for it before writing its last dS)
-                uint32_t w[32];
-                if (valid) {
-                    const __nv_bfloat16* srcb = args.dout + (static_cast<size_t>(s_row) * args.h + head) * 128 + g * 64;
-                    if (aligned32_dev(args.dout)) {          // four 32-byte loads (rows are 256 bytes)
-#pragma unroll
-                        for (int v = 0; v < 4; ++v) ld_global_v8(srcb + v * 16, w + v * 8);
-                    } else {
-                        const uint4* src = reinterpret_cast<const uint4*>(srcb);
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            const uint4 x = src[v];
-                            w[v * 4] = x.x; w[v * 4 + 1] = x.y; w[v * 4 + 2] = x.z; w[v * 4 + 3] = x.w;
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int v = 0; v < 32; ++v) w[v] = 0u;
-                }
-                __syncwarp();
-                tmem_st_x32(tmem_do + lane_addr + g * 32, w);
-                tmem_st_wait();
-                tc_fence_before_sync();
-                mbar_arrive(do_ready);
-            }
             // Rows past the end of the sequence get LSE = +inf so that their P is exactly zero.
             const float l2 = valid ? args.lse[static_cast<size_t>(s_row) * args.h + head] * 1.4426950408889634f : INFINITY;
             const float delta = valid ? args.stat_delta[static_cast<size_t>(head) * args.S_pad + seq.pad_start + s_idx] : 0.f;

@@ -611,7 +611,7 @@ int launch_attn_bwd(const void* q, const void* kv, const void* k_pe, const void*
         {
             ScopedKernelEvents ev(LAGA_KERNEL_ATTN_BWD_DQ, stream);
             launch_kernel(causal ? attn_bwd_dq_sm100_kernel<true> : attn_bwd_dq_sm100_kernel<false>, grid, dim3(kBwdThreads),
-                          AttnBwdDqSmem::kTotalBytes, stream, true, tq, tkv, tpe, b);
+                          AttnBwdDqSmem::kTotalBytes, stream, true, tq, tdo, tkv, tpe, b);
         }
     }
     if (launch_status() != LAGA_OK) return LAGA_ERR_CUDA;
