@@ -658,9 +658,10 @@ struct AttnBwdDqSmem {
 // Persistent: one CTA per SM takes (query tile, head) items from the work counter.  dO of the query
 // tile is the A operand of dP = dO V^T for every key tile; it is kept in TMEM as packed bf16 (64
 // columns) instead of 32 KB of shared memory, which is what leaves room for a third stage of K: a K
-// tile lives from its score MMA to its dQ MMA, a whole tile period later.  Between items the
-// consumers first put the next tile's dO into TMEM and only then drain the finished dQ, so the score
-// MMAs of the next item run under the drain; the K ring simply keeps going across items.
+// tile lives from its score MMA to its dQ MMA, a whole tile period later.  Between items the next
+// tile's dO comes through the V stage and the MMA lane copies it to TMEM (tcgen05.cp) while the
+// consumers drain the finished dQ, so the score MMAs of the next item run under the drain; the K ring
+// simply keeps going across items.
 template <bool kCausal>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_do,

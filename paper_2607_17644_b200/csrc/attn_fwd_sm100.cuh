@@ -70,8 +70,9 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 // Persistent: one CTA per SM takes (query tile, head) items from the work counter.  The K, V and
 // score-tile rings and the alternation of the two softmax groups run on a tile count that continues
 // across items, so the producers prefetch the next item's first key tiles under the current item's
-// last ones; between items, the groups put the next query tile into TMEM before the finished O is
-// drained, so the next item's first score MMAs run under the drain.
+// last ones; between items, the next query tile comes through the V ring and the MMA lane copies it
+// to TMEM (tcgen05.cp) while the softmax groups drain the finished O, so the next item's first score
+// MMAs run under the drain.
 template <bool kCausal>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
